@@ -1,0 +1,180 @@
+"""TEST INFRASTRUCTURE -- not part of the product path.
+
+ctypes front end of the fp64 CPU oracle in ``tli_oracle.c`` (Algorithms 4 and 5
+of the paper).  Only tests, the smoke check and the benchmark's CPU-baseline
+legs may import this package; the CUDA library never does, and this package
+imports nothing from it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from concurrent.futures import ThreadPoolExecutor
+from typing import Dict, Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "tli_oracle.c")
+_LIB = os.path.join(_HERE, "liboracle.so")
+
+F32 = 0
+BF16 = 1
+
+FLAG_DRAFT_RANGE = 1
+FLAG_DRAFT_UNMAPPED = 2
+FLAG_NONFINITE = 4
+FLAG_FALLBACK = 8
+FLAG_BAD_TEMPERATURE = 32
+FLAG_SELFCHECK = 64
+
+
+class _Args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("V_t", ctypes.c_int32), ("V_d", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_k", ctypes.c_int64),
+        ("id_map", ctypes.c_void_p), ("draft_ids", ctypes.c_void_p),
+        ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("force_accept", ctypes.c_void_p), ("probe_token", ctypes.c_void_p),
+        ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("flags", ctypes.c_void_p),
+        ("thr", ctypes.c_void_p), ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
+        ("cdf_lo", ctypes.c_void_p), ("cdf_hi", ctypes.c_void_p), ("total", ctypes.c_void_p),
+        ("probe_lo", ctypes.c_void_p), ("probe_hi", ctypes.c_void_p), ("probe_w", ctypes.c_void_p),
+    ]
+
+
+def build(force: bool = False) -> str:
+    """Compile ``tli_oracle.c`` with gcc -O2 into ``liboracle.so`` beside it."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp.%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-fPIC", "-shared", "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        lib.oracle_tli_verify.argtypes = [ctypes.POINTER(_Args), ctypes.c_int32, ctypes.c_int32]
+        lib.oracle_tli_verify.restype = ctypes.c_int
+        lib.oracle_tli_distributions.argtypes = [ctypes.POINTER(_Args), ctypes.c_int32, ctypes.c_int32,
+                                                 ctypes.c_void_p, ctypes.c_void_p]
+        lib.oracle_tli_distributions.restype = ctypes.c_int
+        _lib = lib
+    return _lib
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data
+
+
+class _Call:
+    """Keeps the numpy arrays of one call alive next to the C struct."""
+
+    def __init__(self, target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
+                 force_accept=None, probe_token=None):
+        zt = np.asarray(target_logits)
+        zd = np.asarray(drafter_logits)
+        if zt.dtype == np.float32 and zd.dtype == np.float32:
+            dtype = F32
+        elif zt.dtype == np.uint16 and zd.dtype == np.uint16:
+            dtype = BF16
+        else:
+            raise TypeError("logits must both be float32 or both be uint16 bfloat16 bit patterns")
+        if zt.ndim != 3 or zd.ndim != 3:
+            raise ValueError("logits must be [B,K+1,V_t] and [B,K,V_d]")
+        B, K1, V_t = zt.shape
+        K = K1 - 1
+        if zd.shape[0] != B or zd.shape[1] != K:
+            raise ValueError("drafter logits must be [B,K,V_d]")
+        V_d = zd.shape[2]
+        if zt.strides[2] != zt.itemsize or zd.strides[2] != zd.itemsize:
+            raise ValueError("vocabulary axis must be contiguous")
+        self.zt, self.zd = zt, zd
+        self.id_map = np.ascontiguousarray(id_map, dtype=np.int32)
+        self.draft = np.ascontiguousarray(draft_ids, dtype=np.int32).reshape(B, K)
+        self.tau = np.ascontiguousarray(temperature, dtype=np.float32).reshape(B)
+        self.u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, K + 1)
+        if self.id_map.shape != (V_d,):
+            raise ValueError("id_map must be [V_d]")
+        self.force = None if force_accept is None else np.ascontiguousarray(force_accept, dtype=np.int8).reshape(B, K)
+        self.probe = None if probe_token is None else np.ascontiguousarray(probe_token, dtype=np.int32).reshape(B)
+        self.out: Dict[str, np.ndarray] = {
+            "accepted": np.zeros(B, np.int32), "next_token": np.zeros(B, np.int32),
+            "flags": np.zeros(B, np.int32),
+            "thr": np.zeros((B, K), np.float64), "p_draft": np.zeros((B, K), np.float64),
+            "q_draft": np.zeros((B, K), np.float64),
+            "cdf_lo": np.zeros(B, np.float64), "cdf_hi": np.zeros(B, np.float64),
+            "total": np.zeros(B, np.float64),
+        }
+        if self.probe is not None:
+            self.out.update(probe_lo=np.zeros(B, np.float64), probe_hi=np.zeros(B, np.float64),
+                            probe_w=np.zeros(B, np.float64))
+        o = self.out
+        self.B, self.K = B, K
+        self.args = _Args(
+            B, K, V_t, V_d, dtype,
+            zt.ctypes.data, zt.strides[0] // zt.itemsize, zt.strides[1] // zt.itemsize,
+            zd.ctypes.data, zd.strides[0] // zd.itemsize, zd.strides[1] // zd.itemsize,
+            _ptr(self.id_map), _ptr(self.draft), _ptr(self.tau), _ptr(self.u),
+            _ptr(self.force), _ptr(self.probe),
+            _ptr(o["accepted"]), _ptr(o["next_token"]), _ptr(o["flags"]),
+            _ptr(o["thr"]), _ptr(o["p_draft"]), _ptr(o["q_draft"]),
+            _ptr(o["cdf_lo"]), _ptr(o["cdf_hi"]), _ptr(o["total"]),
+            _ptr(o.get("probe_lo")), _ptr(o.get("probe_hi")), _ptr(o.get("probe_w")),
+        )
+
+
+def verify(target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
+           force_accept=None, probe_token=None, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Run the oracle on a whole batch.
+
+    Logits are float32 arrays or uint16 arrays holding bfloat16 bit patterns;
+    the batch axes may be strided (a zero batch stride broadcasts one set of
+    logits to every row).  ``threads`` > 1 splits the rows over that many host
+    threads; the arithmetic per row is unchanged.  Returns a dict with
+    ``accepted``, ``next_token``, ``flags`` (int32 [B]), ``thr``, ``p_draft``,
+    ``q_draft`` (float64 [B,K]), ``cdf_lo``, ``cdf_hi``, ``total`` (float64
+    [B]) and, when ``probe_token`` is given, ``probe_lo/hi/w``.
+    """
+    lib = _load()
+    call = _Call(target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
+                 force_accept, probe_token)
+    B = call.B
+    threads = max(1, min(int(threads), B))
+
+    def run(lo_hi):
+        rc = lib.oracle_tli_verify(ctypes.byref(call.args), lo_hi[0], lo_hi[1])
+        if rc != 0:
+            raise RuntimeError("oracle_tli_verify failed with code %d" % rc)
+
+    if threads == 1:
+        run((0, B))
+    else:
+        cuts = [(B * i) // threads for i in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(run, [(cuts[i], cuts[i + 1]) for i in range(threads)]))
+    return call.out
+
+
+def distributions(target_logits, drafter_logits, id_map, temperature, b: int, j: int):
+    """(p, q'_T) of row ``b`` position ``j`` as float64 [V_t] arrays, q' carried to target ids."""
+    lib = _load()
+    zt = np.asarray(target_logits)
+    B, K1, V_t = zt.shape
+    K = K1 - 1
+    call = _Call(target_logits, drafter_logits, id_map, np.zeros((B, K), np.int32), temperature,
+                 np.zeros((B, K + 1), np.float32))
+    p = np.zeros(V_t, np.float64)
+    qT = np.zeros(V_t, np.float64)
+    rc = lib.oracle_tli_distributions(ctypes.byref(call.args), b, j, p.ctypes.data, qT.ctypes.data)
+    if rc != 0:
+        raise RuntimeError("oracle_tli_distributions failed with code %d" % rc)
+    return p, qT

@@ -1,0 +1,373 @@
+/*
+ * TEST INFRASTRUCTURE -- NOT PART OF THE PRODUCT PATH.
+ *
+ * Plain, slow, fp64 CPU oracle for batched Token-Level Intersection (TLI)
+ * verification.  It exists so that tests can check the CUDA library and so that
+ * the benchmark can time a CPU baseline.  Nothing in the product may call it,
+ * and it shares no code, table or helper with the CUDA sources.
+ *
+ * What it computes, in the paper's notation (T target vocabulary, D drafter
+ * vocabulary, p target distribution, q drafter distribution):
+ *
+ *   - Algorithm 4 (TLI): q'(x) = q(x) / sum_{t in T cap D} q(t) on the
+ *     intersection and 0 elsewhere.  The algorithm box writes the sum over T;
+ *     q only lives on D, and the expected-acceptance table writes the same
+ *     denominator as a sum over T cap D, which is the reading used here (it
+ *     also reproduces the worked example q = 1/3,1/3,1/3 -> q' = 1/2,1/2,0).
+ *   - Algorithm 5 (standard speculative decoding) run with (p, q'): a draft
+ *     d_j is rejected with probability 1 - p(d_j)/q'(d_j) when p <= q', i.e.
+ *     accepted iff u < min(1, p/q') for a uniform u in [0,1); the number of
+ *     accepted drafts n is the index of the first rejection; the extra token
+ *     is drawn from r(t) = (p(t) - min{p(t), q'(t)}) / (1 - sum min{p, q'})
+ *     if a draft was rejected and from p otherwise.
+ *
+ * Readings where the paper is silent (each one is a documented choice):
+ *   - logits become distributions by softmax(z / tau), one tau per sequence,
+ *     the same for target and drafter; tau == 0 is the arg-max limit with the
+ *     lowest index winning ties, and then drafter logits and uniforms are not
+ *     read: a draft is accepted iff map[d_j] equals the arg-max of its row;
+ *   - draft ids are drafter-vocabulary ids; the id map sends a drafter id to
+ *     its target id or to -1;
+ *   - a draft id outside [0, V_d) or outside the intersection has q' = 0 and
+ *     is rejected with certainty (threshold 0);
+ *   - the extra token is found by inverse CDF in increasing target-id order
+ *     using one more uniform v = u[b, K]: the smallest t whose cumulative
+ *     weight exceeds v * (total weight);
+ *   - if the residual has zero total weight (only reachable through a draft
+ *     outside the intersection) it falls back to p of that position.
+ *
+ * Every sum runs in index order in double precision; there is no blocking,
+ * fusion or reordering.
+ *
+ * Parity status: every function here is pinned by tests that do not use this
+ * file's own formulas (worked example, brute-force losslessness on tiny
+ * vocabularies, chi-square losslessness, closed-form acceptance rate,
+ * reduction to single-vocabulary rejection sampling, q == p, disjoint and
+ * subset vocabularies).  At benchmark-scale vocabularies nothing beyond those
+ * pins is available: the same code is trusted there because it passed them.
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define ORACLE_F32 0
+#define ORACLE_BF16 1
+
+/* row flag bits, same meaning as the library's row_status */
+#define FLAG_DRAFT_RANGE 1
+#define FLAG_DRAFT_UNMAPPED 2
+#define FLAG_NONFINITE 4
+#define FLAG_FALLBACK 8
+#define FLAG_BAD_TEMPERATURE 32
+/* oracle-only: the two ways of forming q' disagree by more than 1e-12 */
+#define FLAG_SELFCHECK 64
+
+typedef struct {
+    int32_t B, K, V_t, V_d, dtype;
+    const void *target_logits;  /* [B, K+1, V_t], strides in elements */
+    int64_t t_stride_b, t_stride_k;
+    const void *drafter_logits; /* [B, K, V_d] */
+    int64_t d_stride_b, d_stride_k;
+    const int32_t *id_map;      /* [V_d] drafter id -> target id or -1 */
+    const int32_t *draft_ids;   /* [B, K] drafter ids */
+    const float *temperature;   /* [B] */
+    const float *uniforms;      /* [B, K+1] */
+    const int8_t *force_accept; /* [B, K] or NULL: -1 natural, 0 reject, 1 accept */
+    const int32_t *probe_token; /* [B] or NULL: report this token's CDF interval */
+    /* outputs */
+    int32_t *accepted;          /* [B] */
+    int32_t *next_token;        /* [B] */
+    int32_t *flags;             /* [B] */
+    double *thr;                /* [B, K] min(1, p/q') (0 for drafts outside the intersection) */
+    double *p_draft;            /* [B, K] p(map[d_j]) */
+    double *q_draft;            /* [B, K] q'(d_j) */
+    double *cdf_lo;             /* [B] normalised CDF just below next_token */
+    double *cdf_hi;             /* [B] normalised CDF at next_token */
+    double *total;              /* [B] total weight R of the sampled distribution */
+    double *probe_lo;           /* [B] (only if probe_token) */
+    double *probe_hi;           /* [B] */
+    double *probe_w;            /* [B] normalised weight of the probed token */
+} oracle_args;
+
+static double load_logit(const void *base, int dtype, int64_t idx)
+{
+    if (dtype == ORACLE_F32) {
+        return (double)((const float *)base)[idx];
+    } else {
+        uint32_t bits = ((uint32_t)((const uint16_t *)base)[idx]) << 16;
+        float f;
+        memcpy(&f, &bits, sizeof f);
+        return (double)f;
+    }
+}
+
+/* softmax(z / tau) of one row of V logits into out[V]; returns 0 if a logit is not finite */
+static int softmax_row(const void *base, int dtype, int64_t off, int V, double tau, double *out)
+{
+    double m = -INFINITY;
+    for (int i = 0; i < V; ++i) {
+        double z = load_logit(base, dtype, off + i);
+        if (!isfinite(z)) return 0;
+        if (z > m) m = z;
+    }
+    double Z = 0.0;
+    for (int i = 0; i < V; ++i) {
+        out[i] = exp((load_logit(base, dtype, off + i) - m) / tau);
+        Z += out[i];
+    }
+    for (int i = 0; i < V; ++i) out[i] /= Z;
+    return 1;
+}
+
+/* lowest index attaining the maximum of one row */
+static int argmax_row(const void *base, int dtype, int64_t off, int V)
+{
+    int best = 0;
+    double m = load_logit(base, dtype, off);
+    for (int i = 1; i < V; ++i) {
+        double z = load_logit(base, dtype, off + i);
+        if (z > m) { m = z; best = i; }
+    }
+    return best;
+}
+
+/*
+ * Algorithm 4's q' for one drafter row: softmax over all of D, then divide by
+ * the mass on the intersection.  qp[x] = 0 for x outside the intersection.
+ * Also forms q' by a softmax restricted to the intersection and reports
+ * whether the two agree to 1e-12.  Returns 0 on a non-finite logit.
+ */
+static int qprime_row(const oracle_args *a, int64_t off, double tau, double *q, double *qp,
+                      int *selfcheck_ok, int *empty)
+{
+    const int V_d = a->V_d;
+    *selfcheck_ok = 1;
+    *empty = 0;
+    if (!softmax_row(a->drafter_logits, a->dtype, off, V_d, tau, q)) return 0;
+    double M = 0.0;
+    int n_in = 0;
+    for (int x = 0; x < V_d; ++x)
+        if (a->id_map[x] >= 0) { M += q[x]; ++n_in; }
+    if (n_in == 0 || !(M > 0.0)) {
+        /* empty intersection, or all its mass underflowed */
+        *empty = 1;
+        for (int x = 0; x < V_d; ++x) qp[x] = 0.0;
+        if (n_in == 0) return 1;
+    } else {
+        for (int x = 0; x < V_d; ++x) qp[x] = (a->id_map[x] >= 0) ? q[x] / M : 0.0;
+    }
+    /* second route: softmax over the intersection only */
+    double m = -INFINITY;
+    for (int x = 0; x < V_d; ++x)
+        if (a->id_map[x] >= 0) {
+            double z = load_logit(a->drafter_logits, a->dtype, off + x);
+            if (z > m) m = z;
+        }
+    double Z = 0.0;
+    for (int x = 0; x < V_d; ++x)
+        if (a->id_map[x] >= 0) Z += exp((load_logit(a->drafter_logits, a->dtype, off + x) - m) / tau);
+    for (int x = 0; x < V_d; ++x)
+        if (a->id_map[x] >= 0) {
+            double alt = exp((load_logit(a->drafter_logits, a->dtype, off + x) - m) / tau) / Z;
+            if (*empty) { qp[x] = alt; }
+            else if (fabs(alt - qp[x]) > 1e-12) *selfcheck_ok = 0;
+        }
+    if (*empty) *empty = 2; /* rescued by the restricted softmax */
+    return 1;
+}
+
+/*
+ * Verify rows [row_begin, row_end).  Returns 0, or -1 on bad arguments, -2 if
+ * the id map is not injective / out of range, -3 on allocation failure.
+ */
+int oracle_tli_verify(const oracle_args *a, int32_t row_begin, int32_t row_end)
+{
+    if (!a || a->B < 0 || a->K < 1 || a->V_t < 1 || a->V_d < 1) return -1;
+    if (a->dtype != ORACLE_F32 && a->dtype != ORACLE_BF16) return -1;
+    if (row_begin < 0 || row_end > a->B || row_begin > row_end) return -1;
+    const int K = a->K, V_t = a->V_t, V_d = a->V_d;
+
+    int32_t *inv = (int32_t *)malloc(sizeof(int32_t) * (size_t)V_t);
+    double *p = (double *)malloc(sizeof(double) * (size_t)V_t);
+    double *q = (double *)malloc(sizeof(double) * (size_t)V_d);
+    double *qp = (double *)malloc(sizeof(double) * (size_t)V_d);
+    double *w = (double *)malloc(sizeof(double) * (size_t)V_t);
+    int *acc = (int *)malloc(sizeof(int) * (size_t)K);
+    int rc = 0;
+    if (!inv || !p || !q || !qp || !w || !acc) { rc = -3; goto done; }
+
+    /* inverse of the id map: target id -> the one drafter id that maps to it */
+    for (int t = 0; t < V_t; ++t) inv[t] = -1;
+    for (int x = 0; x < V_d; ++x) {
+        int32_t t = a->id_map[x];
+        if (t == -1) continue;
+        if (t < 0 || t >= V_t || inv[t] != -1) { rc = -2; goto done; }
+        inv[t] = x;
+    }
+
+    for (int b = row_begin; b < row_end; ++b) {
+        const double tau = (double)a->temperature[b];
+        const int64_t t_off = (int64_t)b * a->t_stride_b;
+        const int64_t d_off = (int64_t)b * a->d_stride_b;
+        int flags = 0;
+        int n = K;
+        int next = 0;
+        double lo = 0.0, hi = 0.0, R = 0.0;
+        for (int j = 0; j < K; ++j) {
+            if (a->thr) a->thr[(int64_t)b * K + j] = 0.0;
+            if (a->p_draft) a->p_draft[(int64_t)b * K + j] = 0.0;
+            if (a->q_draft) a->q_draft[(int64_t)b * K + j] = 0.0;
+        }
+
+        if (!(tau >= 0.0) || !isfinite(tau)) {
+            flags |= FLAG_BAD_TEMPERATURE;
+            n = 0; next = 0;
+            goto row_done;
+        }
+
+        if (tau == 0.0) {
+            /* arg-max limit: exact match of map[d_j] with the row's arg-max */
+            for (int j = 0; j < K; ++j) {
+                int aj = argmax_row(a->target_logits, a->dtype, t_off + (int64_t)j * a->t_stride_k, V_t);
+                int32_t x = a->draft_ids[(int64_t)b * K + j];
+                int ok;
+                if (x < 0 || x >= V_d) { flags |= FLAG_DRAFT_RANGE; ok = 0; }
+                else if (a->id_map[x] < 0) { flags |= FLAG_DRAFT_UNMAPPED; ok = 0; }
+                else ok = (a->id_map[x] == aj);
+                if (a->force_accept && a->force_accept[(int64_t)b * K + j] >= 0)
+                    ok = a->force_accept[(int64_t)b * K + j];
+                acc[j] = ok;
+                if (a->thr) a->thr[(int64_t)b * K + j] = ok ? 1.0 : 0.0;
+            }
+            n = K;
+            for (int j = 0; j < K; ++j) if (!acc[j]) { n = j; break; }
+            next = argmax_row(a->target_logits, a->dtype, t_off + (int64_t)n * a->t_stride_k, V_t);
+            lo = 0.0; hi = 1.0; R = 1.0;
+            goto row_done;
+        }
+
+        /* acceptance tests, Algorithm 5 with (p, q') */
+        for (int j = 0; j < K; ++j) {
+            int ok_sc, empty;
+            if (!softmax_row(a->target_logits, a->dtype, t_off + (int64_t)j * a->t_stride_k, V_t, tau, p) ||
+                !qprime_row(a, d_off + (int64_t)j * a->d_stride_k, tau, q, qp, &ok_sc, &empty)) {
+                flags |= FLAG_NONFINITE;
+                break;
+            }
+            if (!ok_sc) flags |= FLAG_SELFCHECK;
+            if (empty == 1) flags |= FLAG_FALLBACK;
+            int32_t x = a->draft_ids[(int64_t)b * K + j];
+            double thr, pv = 0.0, qv = 0.0;
+            if (x < 0 || x >= V_d) { flags |= FLAG_DRAFT_RANGE; thr = 0.0; }
+            else if (a->id_map[x] < 0) { flags |= FLAG_DRAFT_UNMAPPED; thr = 0.0; }
+            else {
+                pv = p[a->id_map[x]];
+                qv = qp[x];
+                if (qv > 0.0) { thr = pv / qv; if (thr > 1.0) thr = 1.0; }
+                else thr = (pv > 0.0) ? 1.0 : 0.0;
+            }
+            int ok = ((double)a->uniforms[(int64_t)b * (K + 1) + j] < thr);
+            if (a->force_accept && a->force_accept[(int64_t)b * K + j] >= 0)
+                ok = a->force_accept[(int64_t)b * K + j];
+            acc[j] = ok;
+            if (a->thr) a->thr[(int64_t)b * K + j] = thr;
+            if (a->p_draft) a->p_draft[(int64_t)b * K + j] = pv;
+            if (a->q_draft) a->q_draft[(int64_t)b * K + j] = qv;
+        }
+        if (flags & FLAG_NONFINITE) { n = 0; next = 0; goto row_done; }
+
+        /* number of accepted drafts */
+        n = K;
+        for (int j = 0; j < K; ++j) if (!acc[j]) { n = j; break; }
+
+        /* distribution of the extra token */
+        if (!softmax_row(a->target_logits, a->dtype, t_off + (int64_t)n * a->t_stride_k, V_t, tau, p)) {
+            flags |= FLAG_NONFINITE; n = 0; next = 0; goto row_done;
+        }
+        if (n < K) {
+            int ok_sc, empty;
+            if (!qprime_row(a, d_off + (int64_t)n * a->d_stride_k, tau, q, qp, &ok_sc, &empty)) {
+                flags |= FLAG_NONFINITE; n = 0; next = 0; goto row_done;
+            }
+            R = 0.0;
+            for (int t = 0; t < V_t; ++t) {
+                double qt = (inv[t] >= 0) ? qp[inv[t]] : 0.0;
+                double mn = (p[t] < qt) ? p[t] : qt;   /* min{p, q'} */
+                w[t] = p[t] - mn;                      /* numerator of r(t) */
+                R += w[t];
+            }
+            if (!(R > 0.0)) {
+                flags |= FLAG_FALLBACK;
+                R = 0.0;
+                for (int t = 0; t < V_t; ++t) { w[t] = p[t]; R += w[t]; }
+            }
+        } else {
+            R = 0.0;
+            for (int t = 0; t < V_t; ++t) { w[t] = p[t]; R += w[t]; }
+        }
+        {
+            const double target = (double)a->uniforms[(int64_t)b * (K + 1) + K] * R;
+            double C = 0.0;
+            int found = -1, last_pos = 0;
+            double C_before = 0.0;
+            for (int t = 0; t < V_t; ++t) {
+                double Cn = C + w[t];
+                if (w[t] > 0.0) last_pos = t;
+                if (found < 0 && Cn > target) { found = t; C_before = C; hi = Cn / R; }
+                C = Cn;
+            }
+            if (found < 0) { found = last_pos; C_before = C - w[last_pos]; hi = 1.0; }
+            next = found;
+            lo = C_before / R;
+            if (a->probe_token) {
+                int g = a->probe_token[b];
+                double plo = 0.0, phi = 0.0, pw = 0.0;
+                if (g >= 0 && g < V_t) {
+                    double Cc = 0.0;
+                    for (int t = 0; t < g; ++t) Cc += w[t];
+                    plo = Cc / R; phi = (Cc + w[g]) / R; pw = w[g] / R;
+                }
+                if (a->probe_lo) a->probe_lo[b] = plo;
+                if (a->probe_hi) a->probe_hi[b] = phi;
+                if (a->probe_w) a->probe_w[b] = pw;
+            }
+        }
+row_done:
+        a->accepted[b] = n;
+        a->next_token[b] = next;
+        if (a->flags) a->flags[b] = flags;
+        if (a->cdf_lo) a->cdf_lo[b] = lo;
+        if (a->cdf_hi) a->cdf_hi[b] = hi;
+        if (a->total) a->total[b] = R;
+    }
+done:
+    free(inv); free(p); free(q); free(qp); free(w); free(acc);
+    return rc;
+}
+
+/*
+ * The two distributions of one (row, position) pair, for inspection by tests:
+ * p_out[V_t] = target softmax, qT_out[V_t] = q' carried to target ids
+ * (0 where no drafter id maps).  Returns 0 on success.
+ */
+int oracle_tli_distributions(const oracle_args *a, int32_t b, int32_t j, double *p_out, double *qT_out)
+{
+    if (!a || b < 0 || b >= a->B || j < 0 || j > a->K) return -1;
+    const double tau = (double)a->temperature[b];
+    if (!(tau > 0.0)) return -1;
+    if (!softmax_row(a->target_logits, a->dtype, (int64_t)b * a->t_stride_b + (int64_t)j * a->t_stride_k,
+                     a->V_t, tau, p_out)) return -4;
+    for (int t = 0; t < a->V_t; ++t) qT_out[t] = 0.0;
+    if (j == a->K) return 0;
+    double *q = (double *)malloc(sizeof(double) * (size_t)a->V_d);
+    double *qp = (double *)malloc(sizeof(double) * (size_t)a->V_d);
+    if (!q || !qp) { free(q); free(qp); return -3; }
+    int ok_sc, empty;
+    int ok = qprime_row(a, (int64_t)b * a->d_stride_b + (int64_t)j * a->d_stride_k, tau, q, qp, &ok_sc, &empty);
+    if (ok)
+        for (int x = 0; x < a->V_d; ++x)
+            if (a->id_map[x] >= 0 && a->id_map[x] < a->V_t) qT_out[a->id_map[x]] = qp[x];
+    free(q); free(qp);
+    return ok ? 0 : -4;
+}
