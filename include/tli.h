@@ -1,0 +1,161 @@
+/*
+ * tli.h -- C ABI of the Token-Level Intersection (TLI) verification library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * One call verifies K drafted tokens for each of B sequences when the drafter
+ * and the target model use different vocabularies: Algorithm 4 of the paper
+ * (project the drafter distribution onto the vocabulary intersection and
+ * renormalise it) followed by the verification half of Algorithm 5 (rejection
+ * test per draft, first rejection, residual or bonus sample).
+ *
+ * Conventions
+ *   - Pointers marked [device] are device pointers owned by the caller; the
+ *     library never frees or reallocates them.  Pointers marked [host] are
+ *     read during the call only.
+ *   - tli_verify() is asynchronous on the stream it is given, allocates
+ *     nothing and does not synchronise.
+ *   - Functions return TLI_OK or a negative tli error code.  Errors in the
+ *     data (a draft id outside the vocabulary, a NaN logit, a negative
+ *     temperature) never fault: they set bits in row_status.
+ */
+#ifndef TLI_H
+#define TLI_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tli_ctx tli_ctx; /* opaque, library-owned */
+
+/* logit storage types */
+enum { TLI_F32 = 0, TLI_BF16 = 1 };
+
+/* return codes */
+enum {
+    TLI_OK = 0,
+    TLI_ERR_ARG = -1,         /* null pointer, bad size, bad dtype, misaligned logits */
+    TLI_ERR_BAD_MAP = -2,     /* id map entry out of range, or two drafter ids on one target id */
+    TLI_ERR_CUDA = -3,        /* a CUDA runtime call failed (tli_last_cuda_error() says which) */
+    TLI_ERR_WORKSPACE = -4,   /* workspace missing, misaligned or too small */
+    TLI_ERR_UNSUPPORTED = -5  /* size beyond TLI_MAX_B / TLI_MAX_K / TLI_MAX_V */
+};
+
+/* row_status bits */
+enum {
+    TLI_ROW_DRAFT_RANGE = 1,      /* a draft id outside [0, V_d): treated as rejected */
+    TLI_ROW_DRAFT_UNMAPPED = 2,   /* a draft id outside the intersection: rejected (q' = 0 there) */
+    TLI_ROW_NONFINITE = 4,        /* NaN or +inf logit seen: accepted = 0, next_token = 0 */
+    TLI_ROW_FALLBACK = 8,         /* empty intersection or zero residual mass: sampled from p instead */
+    TLI_ROW_BAD_TEMPERATURE = 32  /* temperature negative or not finite: accepted = 0, next_token = 0 */
+};
+
+#define TLI_MAX_B 65535    /* sequences per call */
+#define TLI_MAX_K 64       /* drafts per sequence */
+#define TLI_MAX_V 1048576  /* vocabulary size (either side) */
+
+/*
+ * Create a context for one (target vocabulary, drafter vocabulary) pair on one
+ * device.  Implements the "T cap D" of Algorithm 4 as data: id_map[x] is the
+ * target id of drafter token x, or -1 when x is not in the target vocabulary.
+ *
+ *   out          [host]  receives the context
+ *   device               CUDA device ordinal; made current during the call and
+ *                        restored afterwards
+ *   V_t, V_d             vocabulary sizes, 1 .. TLI_MAX_V
+ *   id_map_host  [host]  int32[V_d]; every entry -1 or in [0, V_t); vocabularies
+ *                        are sets of strings, so no two drafter ids may share a
+ *                        target id (TLI_ERR_BAD_MAP otherwise).  Validated
+ *                        before any CUDA call is made.
+ *
+ * The context owns device copies of the map, its inverse (target id -> drafter
+ * id), a bit mask of mapped drafter ids, and per-sequence completion counters.
+ * Because of those counters a context serves one tli_verify() at a time: calls
+ * on the same context must be ordered on one stream (or by events).
+ */
+int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_t *id_map_host);
+
+/* Free a context.  The caller makes sure no call using it is still running. */
+int tli_destroy(tli_ctx *ctx);
+
+/* Bytes of device scratch tli_verify() needs for (B, K, dtype); 0 on bad arguments. */
+size_t tli_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype);
+
+typedef struct {
+    int32_t B;      /* sequences, 1 .. TLI_MAX_B */
+    int32_t K;      /* drafts per sequence, 1 .. TLI_MAX_K */
+    int32_t dtype;  /* TLI_F32 or TLI_BF16, for both logit tensors */
+
+    /* [device] target logits [B, K+1, V_t]: row j is the target distribution
+     * for the token at draft position j, row K the bonus position
+     * (Algorithm 5's single batched target pass).  Strides in elements; the
+     * vocabulary axis is contiguous.  The base pointer is aligned to the
+     * element size; rows need no further alignment. */
+    const void *target_logits;
+    int64_t t_stride_b, t_stride_k;
+
+    /* [device] drafter logits [B, K, V_d], the distributions the drafts were
+     * sampled from.  Not read for temperature-0 sequences. */
+    const void *drafter_logits;
+    int64_t d_stride_b, d_stride_k;
+
+    const int32_t *draft_ids;   /* [device] int32[B, K], drafter-vocabulary ids */
+    const float *temperature;   /* [device] float[B]; softmax(z / tau) on both sides; 0 = arg-max */
+    const float *uniforms;      /* [device] float[B, K+1] in [0, 1): column j < K drives the
+                                 * acceptance test of draft j, column K the one extra token */
+
+    int32_t *accepted;          /* [device] out int32[B]: accepted drafts n, 0 .. K */
+    int32_t *next_token;        /* [device] out int32[B]: target-vocabulary id of the token after
+                                 * the accepted drafts (residual sample if n < K, bonus sample
+                                 * from row K otherwise) */
+    int32_t *row_status;        /* [device] out int32[B] of TLI_ROW_* bits; may be NULL */
+    float *p_draft;             /* [device] out float[B, K]: p(map[d_j]); may be NULL */
+    float *q_draft;             /* [device] out float[B, K]: q'(d_j); may be NULL.  Both are 0
+                                 * for temperature-0 sequences and invalid drafts */
+
+    void *workspace;            /* [device] scratch, 256-byte aligned, >= tli_workspace_bytes();
+                                 * contents need no initialisation and are garbage afterwards */
+    size_t workspace_bytes;
+} tli_verify_args;
+
+/*
+ * Verify one batch (Algorithm 4, then Algorithm 5's acceptance loop, count and
+ * final sample), per sequence b with tau = temperature[b]:
+ *
+ *   tau > 0:  p_j = softmax(target row j / tau);  q_j = softmax(drafter row j / tau);
+ *             q'_j(x) = q_j(x) / sum_{map[y] >= 0} q_j(y) if map[x] >= 0, else 0;
+ *             draft j is accepted iff uniforms[b,j] < min(1, p_j(map[d_j]) / q'_j(d_j));
+ *             n = index of the first rejected draft, K if none;
+ *             n < K:  next_token ~ max(0, p_n - q'_n) normalised (q' carried to target ids);
+ *             n == K: next_token ~ p_K;
+ *             both by inverse CDF in increasing target-id order with v = uniforms[b,K]:
+ *             the smallest t whose cumulative weight exceeds v * total.
+ *   tau == 0: a_j = lowest index attaining the maximum of target row j; draft j is
+ *             accepted iff map[d_j] == a_j; next_token = a_n.
+ *
+ * All arithmetic on the vocabulary rows is fp32 with fp64 combination of
+ * partial sums; temperature-0 rows are exact comparisons on the stored values.
+ * A logit of -inf is a token of probability zero; NaN or +inf flags the row.
+ *
+ * Returns TLI_ERR_ARG / TLI_ERR_WORKSPACE / TLI_ERR_UNSUPPORTED for
+ * host-detectable argument errors (nothing is launched) and TLI_ERR_CUDA if a
+ * launch fails.  `cuda_stream` is a cudaStream_t (NULL = default stream); the
+ * context's device must be current.
+ */
+int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
+
+/* Vocabulary sizes and number of mapped drafter ids of a context. */
+int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped);
+
+/* Static, human-readable name of a return code. */
+const char *tli_status_string(int code);
+
+/* Text of the last CUDA runtime error seen by this library on the calling thread ("" if none). */
+const char *tli_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TLI_H */
