@@ -1,0 +1,904 @@
+// TLI verification for sm_100a: kernels and the C ABI declared in include/tli.h.
+//
+// Two launches per call, both streaming and HBM-bound (no dense contraction,
+// hence no tensor cores):
+//
+//   tli_stats_kernel   one CTA per 16 KB chunk of a logit row.  Target rows:
+//                      (reference, sum of 2^(z*s - reference)) with s = log2(e)/tau;
+//                      drafter rows: the same over ids inside the intersection
+//                      only (Algorithm 4's renormalisation: the full-softmax
+//                      denominator cancels in q' = q / sum_{T cap D} q);
+//                      temperature-0 rows: (max, lowest index).  The last CTA to
+//                      finish a sequence (atomic ticket, nobody waits) combines
+//                      the partials in fp64, runs Algorithm 5's acceptance tests
+//                      and first-rejection count, and records which row the
+//                      extra token is drawn from.
+//   tli_sample_kernel  one CTA per 16 KB tile of that one target row: tile sums
+//                      of max(0, p - q'_T) (or of p for the bonus row); the last
+//                      CTA of a sequence walks tile -> 16-byte vector -> element
+//                      to invert the CDF.
+//
+// Softmax terms are formed as ex2(fma(z, s, -c)) with a per-warp reference c in
+// log2 units, so the only per-term rounding is the one in the fma.
+
+#include <cuda_runtime.h>
+#include <float.h>
+#include <limits.h>
+#include <math.h>
+#include <stdint.h>
+#include <stdio.h>
+#include <string.h>
+#include <new>
+#include <vector>
+
+#include "tli.h"
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int kWarps = kThreads / 32;
+constexpr int kVecPerThread = 4;
+constexpr int kVecPerChunk = kThreads * kVecPerThread;      // 1024 16-byte vectors
+constexpr int kChunkBytes = kVecPerChunk * 16;              // 16 KB
+constexpr int kMaxTiles = (TLI_MAX_V * 4 + 15) / kChunkBytes + 2;
+constexpr float kNegBig = -FLT_MAX;
+
+enum : int { MODE_SKIP = 0, MODE_RESIDUAL = 1, MODE_TARGET_ONLY = 2 };
+
+struct RowSel {          // what the sampling pass needs for one sequence
+    int n;               // accepted drafts = row to sample from
+    int mode;            // MODE_*
+    float s;             // log2(e) / tau
+    float c_t;           // reference of target row n (log2 units)
+    float rs_t;          // 1 / sum of target row n
+    float c_d;           // reference of drafter row n
+    float rs_d;          // 1 / intersection sum of drafter row n (0 if empty)
+    float v;             // uniforms[b, K]
+};
+
+struct Params {
+    int B, K, V_t, V_d;
+    const void *zt; long long t_sb, t_sk;
+    const void *zd; long long d_sb, d_sk;
+    const int *map; const int *inv; const uint32_t *maskbits; int n_mapped;
+    const int *draft; const float *tau; const float *u;
+    int *accepted; int *next_token; int *status; float *p_out; float *q_out;
+    float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
+    unsigned *cnt_stats; unsigned *cnt_sample;
+    int nct, ncd;
+};
+
+// ---------------------------------------------------------------------------
+// small device helpers
+// ---------------------------------------------------------------------------
+
+__device__ __forceinline__ float ex2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+__device__ __forceinline__ int float_order(float f) {       // monotone float -> int
+    int i = __float_as_int(f);
+    return i ^ ((i >> 31) & 0x7fffffff);
+}
+__device__ __forceinline__ float order_float(int i) {
+    return __int_as_float(i ^ ((i >> 31) & 0x7fffffff));
+}
+__device__ __forceinline__ float warp_max(float m) {
+    return order_float(__reduce_max_sync(0xffffffffu, float_order(m)));
+}
+__device__ __forceinline__ float warp_sum(float s) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
+}
+__device__ __forceinline__ double warp_sum(double s) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
+    return s;
+}
+
+template <int DT> struct Elt;
+template <> struct Elt<TLI_F32> {
+    static constexpr int kBytes = 4;
+    static constexpr int kPerVec = 4;
+    static constexpr uint32_t kNegInfWord = 0xff800000u;
+};
+template <> struct Elt<TLI_BF16> {
+    static constexpr int kBytes = 2;
+    static constexpr int kPerVec = 8;
+    static constexpr uint32_t kNegInfWord = 0xff80ff80u;
+};
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+template <int DT> __device__ __forceinline__ float load_elt(const void *row, long long i) {
+    if (DT == TLI_F32) return __ldg(reinterpret_cast<const float *>(row) + i);
+    return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short *>(row) + i)) << 16);
+}
+
+template <int DT> __device__ __forceinline__ void unpack(const uint4 &r, float (&z)[Elt<DT>::kPerVec]) {
+    if constexpr (DT == TLI_F32) {
+        z[0] = __uint_as_float(r.x); z[1] = __uint_as_float(r.y);
+        z[2] = __uint_as_float(r.z); z[3] = __uint_as_float(r.w);
+    } else {
+        z[0] = bf16_lo(r.x); z[1] = bf16_hi(r.x); z[2] = bf16_lo(r.y); z[3] = bf16_hi(r.y);
+        z[4] = bf16_lo(r.z); z[5] = bf16_hi(r.z); z[6] = bf16_lo(r.w); z[7] = bf16_hi(r.w);
+    }
+}
+
+// A logit row seen as 16-byte vectors on the aligned address grid.  Vector v
+// holds elements [v*EPV - head, v*EPV - head + EPV); elements outside [0, V)
+// read as -inf.
+template <int DT> struct RowView {
+    const uint4 *vec0;   // 16-byte aligned address at or below the row start
+    const void *row;     // the row itself
+    int head;            // elements of vector 0 that precede the row
+    int V;
+    __device__ RowView(const void *base, long long elem_off, int V_) {
+        const char *p = reinterpret_cast<const char *>(base) + elem_off * Elt<DT>::kBytes;
+        uintptr_t a = reinterpret_cast<uintptr_t>(p);
+        uintptr_t a0 = a & ~static_cast<uintptr_t>(15);
+        vec0 = reinterpret_cast<const uint4 *>(a0);
+        row = p;
+        head = static_cast<int>(a - a0) / Elt<DT>::kBytes;
+        V = V_;
+    }
+    __device__ __forceinline__ int first_elem(int v) const { return v * Elt<DT>::kPerVec - head; }
+    __device__ __forceinline__ int nvec() const { return (V + head + Elt<DT>::kPerVec - 1) / Elt<DT>::kPerVec; }
+    // Whole vectors with one 128-bit load; the two ragged ends element by element.
+    __device__ __forceinline__ uint4 load(int v) const {
+        const int e0 = first_elem(v);
+        if (e0 >= 0 && e0 + Elt<DT>::kPerVec <= V) return __ldg(vec0 + v);
+        uint32_t w[4] = {Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord};
+        if constexpr (DT == TLI_F32) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                int e = e0 + i;
+                if (e >= 0 && e < V) w[i] = __ldg(reinterpret_cast<const uint32_t *>(row) + e);
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                int e = e0 + i;
+                if (e >= 0 && e < V) {
+                    uint32_t h = __ldg(reinterpret_cast<const unsigned short *>(row) + e);
+                    w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | (h << 16)) : ((w[i >> 1] & 0xffff0000u) | h);
+                }
+            }
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// bit i = 1 iff drafter id e0 + i is inside the intersection (ids outside [0, V_d) read 0;
+// the bit array is zero padded by two words).
+__device__ __forceinline__ uint32_t mask_bits(const uint32_t *maskbits, int e0) {
+    if (e0 < 0) return __ldg(maskbits) << (-e0);
+    const uint32_t lo = __ldg(maskbits + (e0 >> 5));
+    const uint32_t hi = __ldg(maskbits + (e0 >> 5) + 1);
+    return __funnelshift_r(lo, hi, e0 & 31);
+}
+
+// (reference, sum) pairs: value = sum * 2^reference.
+__device__ __forceinline__ void combine_pair(float &c, float &s, float c2, float s2) {
+    const float cn = fmaxf(c, c2);
+    s = s * ex2(c - cn) + s2 * ex2(c2 - cn);
+    c = cn;
+}
+
+// ---------------------------------------------------------------------------
+// pass 1: per-chunk statistics
+// ---------------------------------------------------------------------------
+
+// softmax statistics of one chunk; MASKED restricts to drafter ids inside the intersection
+template <int DT, bool MASKED>
+__device__ __forceinline__ float2 chunk_softmax_stats(const RowView<DT> &rv, int chunk, float s,
+                                                      const uint32_t *maskbits, float2 *sm_pairs) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = rv.nvec();
+    uint4 raw[kVecPerThread];
+    uint32_t bits[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = chunk * kVecPerChunk + k * kThreads + tid;
+        if (v < nvec) {
+            raw[k] = rv.load(v);
+            bits[k] = MASKED ? mask_bits(maskbits, rv.first_elem(v)) : 0xffffffffu;
+        } else {
+            raw[k] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+            bits[k] = 0;
+        }
+    }
+    float z[kVecPerThread][EPV];
+    float m = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        unpack<DT>(raw[k], z[k]);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+            if (MASKED) z[k][i] = ((bits[k] >> i) & 1u) ? z[k][i] : -INFINITY;
+            m = fmaxf(m, z[k][i]);
+        }
+    }
+    m = warp_max(m);
+    const float c = fmaxf(m * s, kNegBig);      // -inf (nothing here) -> most negative finite reference
+    const float nc = -c;
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) acc[i & 3] += ex2(fmaf(z[k][i], s, nc));
+    }
+    float sum = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
+    if (lane == 0) sm_pairs[warp] = make_float2(c, sum);
+    __syncthreads();
+    float2 out = make_float2(kNegBig, 0.f);
+    if (warp == 0) {
+        float2 pr = (lane < kWarps) ? sm_pairs[lane] : make_float2(kNegBig, 0.f);
+#pragma unroll
+        for (int o = kWarps / 2; o > 0; o >>= 1) {
+            float c2 = __shfl_xor_sync(0xffffffffu, pr.x, o);
+            float s2 = __shfl_xor_sync(0xffffffffu, pr.y, o);
+            combine_pair(pr.x, pr.y, c2, s2);
+        }
+        out = pr;
+    }
+    return out;      // valid in warp 0
+}
+
+// (max, lowest index attaining it) of one chunk, as (value, index bits)
+template <int DT>
+__device__ __forceinline__ float2 chunk_argmax(const RowView<DT> &rv, int chunk, float2 *sm_pairs) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = rv.nvec();
+    uint4 raw[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = chunk * kVecPerChunk + k * kThreads + tid;
+        raw[k] = (v < nvec) ? rv.load(v)
+                            : make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+    }
+    float best = -INFINITY;
+    int idx = INT_MAX;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {      // increasing index order, strict > keeps the lowest
+        float z[EPV];
+        unpack<DT>(raw[k], z);
+        const int e0 = rv.first_elem(chunk * kVecPerChunk + k * kThreads + tid);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i)
+            if (z[i] > best) { best = z[i]; idx = e0 + i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+        int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+        if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
+    }
+    if (lane == 0) sm_pairs[warp] = make_float2(best, __int_as_float(idx));
+    __syncthreads();
+    float2 out = make_float2(-INFINITY, __int_as_float(INT_MAX));
+    if (warp == 0) {
+        float2 pr = (lane < kWarps) ? sm_pairs[lane] : out;
+        best = pr.x; idx = __float_as_int(pr.y);
+#pragma unroll
+        for (int o = kWarps / 2; o > 0; o >>= 1) {
+            float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+            int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
+        }
+        out = make_float2(best, __int_as_float(idx));
+    }
+    return out;
+}
+
+// Last CTA of a sequence: fp64 combination of the chunk partials, Algorithm 5's
+// acceptance tests and count, hand-over to the sampling pass.
+template <int DT>
+__device__ void finalize_sequence(const Params &P, int b, float tau) {
+    __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
+    __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
+    __shared__ int sm_accept[TLI_MAX_K];
+    __shared__ int sm_flags;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int K = P.K;
+    const bool greedy = (tau == 0.f);
+    const int nrows = greedy ? (K + 1) : (2 * K + 1);
+    if (tid == 0) sm_flags = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+
+    for (int r = warp; r < nrows; r += kWarps) {
+        const bool is_t = r <= K;
+        const int nchunk = is_t ? P.nct : P.ncd;
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nct
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.ncd;
+        if (greedy) {
+            float best = -INFINITY; int idx = INT_MAX;
+            for (int i = lane; i < nchunk; i += 32) {
+                float2 pr = __ldcg(part + i);
+                int i2 = __float_as_int(pr.y);
+                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+                int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
+            }
+            if (lane == 0) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
+        } else {
+            float c = kNegBig;
+            for (int i = lane; i < nchunk; i += 32) c = fmaxf(c, __ldcg(part + i).x);
+            c = warp_max(c);
+            double s = 0.0;
+            for (int i = lane; i < nchunk; i += 32) {
+                float2 pr = __ldcg(part + i);
+                s += static_cast<double>(pr.y) * exp2(static_cast<double>(pr.x) - static_cast<double>(c));
+            }
+            s = warp_sum(s);
+            if (lane == 0) { sm_c[r] = c; sm_s[r] = s; }
+        }
+    }
+    __syncthreads();
+
+    const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
+    if (tid < K) {
+        const int j = tid;
+        const int x = P.draft[static_cast<size_t>(b) * K + j];
+        int ok = 0, fl = 0;
+        float pv = 0.f, qv = 0.f;
+        int t = -1;
+        if (x < 0 || x >= P.V_d) fl |= TLI_ROW_DRAFT_RANGE;
+        else { t = __ldg(P.map + x); if (t < 0) fl |= TLI_ROW_DRAFT_UNMAPPED; }
+        if (greedy) {
+            ok = (t >= 0 && t == static_cast<int>(sm_s[j]));
+        } else {
+            const double S_t = sm_s[j], S_d = sm_s[K + 1 + j];
+            if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
+            else if (t >= 0) {
+                const double sd = static_cast<double>(s_f);
+                const double zt = static_cast<double>(load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk + t));
+                const double zd = static_cast<double>(load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk + x));
+                const double p = exp2(zt * sd - static_cast<double>(sm_c[j])) / S_t;
+                const double q = (S_d > 0.0) ? exp2(zd * sd - static_cast<double>(sm_c[K + 1 + j])) / S_d : 0.0;
+                double thr;
+                if (q > 0.0) thr = fmin(1.0, p / q);
+                else thr = (p > 0.0) ? 1.0 : 0.0;
+                ok = static_cast<double>(P.u[static_cast<size_t>(b) * (K + 1) + j]) < thr;
+                pv = static_cast<float>(p); qv = static_cast<float>(q);
+            }
+        }
+        sm_accept[j] = ok;
+        if (fl) atomicOr(&sm_flags, fl);
+        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
+        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+    }
+    // the bonus row's sum must be usable too
+    if (tid == K && !greedy) {
+        const double S_t = sm_s[K];
+        if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n = K;
+        for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
+        int fl = sm_flags;
+        RowSel sel;
+        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
+        sel.v = P.u[static_cast<size_t>(b) * (K + 1) + K];
+        if (greedy) {
+            P.next_token[b] = static_cast<int>(sm_s[n]);
+        } else if (fl & TLI_ROW_NONFINITE) {
+            n = 0;
+            P.next_token[b] = 0;
+        } else {
+            sel.c_t = sm_c[n];
+            sel.rs_t = static_cast<float>(1.0 / sm_s[n]);
+            if (n < K) {
+                const double S_d = sm_s[K + 1 + n];
+                sel.mode = MODE_RESIDUAL;
+                sel.c_d = sm_c[K + 1 + n];
+                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
+            } else {
+                sel.mode = MODE_TARGET_ONLY;
+            }
+        }
+        sel.n = n;
+        P.accepted[b] = n;
+        if (P.status) P.status[b] = fl;
+        P.sel[b] = sel;
+        P.cnt_stats[b] = 0;        // leave the ticket counter ready for the next call
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_stats_kernel(const Params P) {
+    __shared__ float2 sm_pairs[kWarps];
+    __shared__ int sm_last;
+    asm volatile("griddepcontrol.launch_dependents;");
+    const int b = blockIdx.y;
+    const int item = blockIdx.x;
+    const int K = P.K;
+    const float tau = __ldg(P.tau + b);
+    if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
+        if (item == 0 && threadIdx.x == 0) {
+            P.accepted[b] = 0; P.next_token[b] = 0;
+            if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
+            RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            P.sel[b] = sel;
+        }
+        if (item == 0 && threadIdx.x < K) {
+            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + threadIdx.x] = 0.f;
+            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + threadIdx.x] = 0.f;
+        }
+        return;
+    }
+    const bool greedy = (tau == 0.f);
+    const int n_target_items = (K + 1) * P.nct;
+    const float s = 1.4426950408889634f / tau;
+    float2 partial;
+    float2 *dst;
+    if (item < n_target_items) {
+        const int j = item / P.nct, chunk = item - j * P.nct;
+        RowView<DT> rv(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk, P.V_t);
+        partial = greedy ? chunk_argmax<DT>(rv, chunk, sm_pairs)
+                         : chunk_softmax_stats<DT, false>(rv, chunk, s, nullptr, sm_pairs);
+        dst = P.part_t + (static_cast<size_t>(b) * (K + 1) + j) * P.nct + chunk;
+    } else {
+        if (greedy) return;                        // drafter logits are not read at temperature 0
+        const int it = item - n_target_items;
+        const int j = it / P.ncd, chunk = it - j * P.ncd;
+        RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk, P.V_d);
+        partial = chunk_softmax_stats<DT, true>(rv, chunk, s, P.maskbits, sm_pairs);
+        dst = P.part_d + (static_cast<size_t>(b) * K + j) * P.ncd + chunk;
+    }
+    if (threadIdx.x == 0) {
+        __stcg(dst, partial);
+        __threadfence();
+        const unsigned total = greedy ? n_target_items : n_target_items + K * P.ncd;
+        const unsigned ticket = atomicAdd(P.cnt_stats + b, 1u);
+        sm_last = (ticket == total - 1);
+    }
+    __syncthreads();
+    if (sm_last) {
+        __threadfence();
+        finalize_sequence<DT>(P, b, tau);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// pass 2: the extra token
+// ---------------------------------------------------------------------------
+
+// Weights of the elements of vector v of the sampled target row:
+// p(t), or max(0, p(t) - q'(inv[t])) for the residual.  The same code feeds the
+// tile sums and every rescan, so the levels of the CDF walk agree bit for bit.
+template <int DT>
+__device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
+                                               const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const uint4 raw = rt.load(v);
+    const int e0 = rt.first_elem(v);
+    float z[EPV];
+    unpack<DT>(raw, z);
+    int x[EPV];
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) x[i] = -1;
+    if (sel.mode == MODE_RESIDUAL) {
+        if (e0 >= 0 && e0 + EPV <= P.V_t && (e0 & 3) == 0) {
+#pragma unroll
+            for (int i = 0; i < EPV; i += 4) {
+                const int4 q = __ldg(reinterpret_cast<const int4 *>(P.inv + e0 + i));
+                x[i] = q.x; x[i + 1] = q.y; x[i + 2] = q.z; x[i + 3] = q.w;
+            }
+        } else {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                const int t = e0 + i;
+                x[i] = (t >= 0 && t < P.V_t) ? __ldg(P.inv + t) : -1;
+            }
+        }
+    }
+    const float nct = -sel.c_t, ncd = -sel.c_d;
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) {
+        const float et = ex2(__fmaf_rn(z[i], sel.s, nct));
+        float q = 0.f;
+        if (x[i] >= 0) {
+            const float zdv = load_elt<DT>(zd_row, x[i]);
+            q = __fmul_rn(ex2(__fmaf_rn(zdv, sel.s, ncd)), sel.rs_d);
+        }
+        w[i] = fmaxf(0.f, __fmaf_rn(et, sel.rs_t, -q));
+    }
+}
+
+template <int N> __device__ __forceinline__ float ordered_sum(const float (&w)[N]) {
+    float s = w[0];
+#pragma unroll
+    for (int i = 1; i < N; ++i) s = __fadd_rn(s, w[i]);
+    return s;
+}
+
+// sum of one tile's weights (fp64 over fp32 vector sums); result valid in thread 0
+template <int DT>
+__device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel &sel, const RowView<DT> &rt,
+                                                  const void *zd_row, int tile, double *sm_red) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nvec = rt.nvec();
+    double acc = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = tile * kVecPerChunk + k * kThreads + tid;
+        if (v < nvec) {
+            float w[EPV];
+            vector_weights<DT>(P, sel, rt, zd_row, v, w);
+            acc += static_cast<double>(ordered_sum(w));
+        }
+    }
+    acc = warp_sum(acc);
+    __syncthreads();                   // sm_red may still be in use by the previous tile
+    if (lane == 0) sm_red[warp] = acc;
+    __syncthreads();
+    double tot = 0.0;
+    if (tid == 0) {
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) tot += sm_red[i];
+    }
+    return tot;
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    __shared__ double sm_red[kWarps];
+    __shared__ double sm_tiles[kMaxTiles];
+    __shared__ float sm_seg[kVecPerChunk];
+    __shared__ double sm_warp_tot[kWarps];
+    __shared__ int sm_last, sm_tile, sm_found, sm_lastpos, sm_retry;
+    __shared__ double sm_rem;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int b = blockIdx.y, tile = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    RowSel sel = P.sel[b];
+    if (sel.mode == MODE_SKIP) return;
+    const int ntile = P.nct;
+    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
+        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
+
+    const double tot = tile_weight_sum<DT>(P, sel, rt, zd_row, tile, sm_red);
+    if (tid == 0) {
+        __stcg(P.tilesum + static_cast<size_t>(b) * ntile + tile, tot);
+        __threadfence();
+        const unsigned ticket = atomicAdd(P.cnt_sample + b, 1u);
+        sm_last = (ticket == static_cast<unsigned>(ntile) - 1);
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+
+    // ---- last CTA of the sequence: invert the CDF, tile -> vector -> element ----
+    for (int i = tid; i < ntile; i += kThreads) sm_tiles[i] = __ldcg(P.tilesum + static_cast<size_t>(b) * ntile + i);
+    __syncthreads();
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        if (tid == 0) {
+            double R = 0.0;
+            for (int i = 0; i < ntile; ++i) R += sm_tiles[i];
+            sm_retry = 0;
+            if (!(R > 0.0) || !isfinite(R)) {
+                sm_retry = 1;
+            } else {
+                const double target = static_cast<double>(sel.v) * R;
+                double run = 0.0;
+                int T = -1, lastpos = 0;
+                double before = 0.0;
+                for (int i = 0; i < ntile; ++i) {
+                    const double nx = run + sm_tiles[i];
+                    if (sm_tiles[i] > 0.0) lastpos = i;
+                    if (T < 0 && nx > target) { T = i; before = run; }
+                    run = nx;
+                }
+                if (T < 0) { T = lastpos; before = R - sm_tiles[lastpos]; }
+                sm_tile = T;
+                sm_rem = target - before;
+            }
+        }
+        __syncthreads();
+        if (!sm_retry) break;
+        if (attempt == 1) {                      // no usable mass even from p: give up on the row
+            if (tid == 0) {
+                P.next_token[b] = 0;
+                if (P.status) P.status[b] |= TLI_ROW_NONFINITE;
+                P.cnt_sample[b] = 0;
+            }
+            return;
+        }
+        // zero residual mass: sample from p of the same position instead
+        sel.mode = MODE_TARGET_ONLY;
+        if (tid == 0 && P.status) P.status[b] |= TLI_ROW_FALLBACK;
+        for (int i = 0; i < ntile; ++i) {
+            const double t2 = tile_weight_sum<DT>(P, sel, rt, zd_row, i, sm_red);
+            if (tid == 0) sm_tiles[i] = t2;
+        }
+        __syncthreads();
+    }
+
+    const int T = sm_tile;
+    const double rem = sm_rem;
+    const int nvec = rt.nvec();
+    // vector sums of tile T in address order
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int g = k * kThreads + tid;
+        const int v = T * kVecPerChunk + g;
+        float sseg = 0.f;
+        if (v < nvec) {
+            float w[EPV];
+            vector_weights<DT>(P, sel, rt, zd_row, v, w);
+            sseg = ordered_sum(w);
+        }
+        sm_seg[g] = sseg;
+    }
+    if (tid == 0) { sm_found = INT_MAX; sm_lastpos = -1; }
+    __syncthreads();
+    // thread i owns vectors 4i .. 4i+3: block-wide exclusive prefix in fp64
+    double loc[kVecPerThread];
+    double mine = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) { loc[k] = static_cast<double>(sm_seg[tid * kVecPerThread + k]); mine += loc[k]; }
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) sm_warp_tot[warp] = incl;
+    __syncthreads();
+    double base = 0.0;
+    for (int i = 0; i < warp; ++i) base += sm_warp_tot[i];
+    double run = base + incl - mine;               // mass before this thread's first vector
+    int cand = INT_MAX, lastpos = -1;
+    double cand_before = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const double nx = run + loc[k];
+        if (loc[k] > 0.0) lastpos = tid * kVecPerThread + k;
+        if (cand == INT_MAX && nx > rem) { cand = tid * kVecPerThread + k; cand_before = run; }
+        run = nx;
+    }
+    if (cand != INT_MAX) atomicMin(&sm_found, cand);
+    if (lastpos >= 0) atomicMax(&sm_lastpos, lastpos);
+    __syncthreads();
+    const int found = sm_found;
+    const int G = (found != INT_MAX) ? found : sm_lastpos;
+    if (G < 0) {                                   // cannot happen when the tile has positive mass
+        if (tid == 0) { P.next_token[b] = 0; P.cnt_sample[b] = 0; }
+        return;
+    }
+    if (tid == G / kVecPerThread) {
+        // walk the elements of vector G with the same running fp32 sum that formed its total;
+        // when rounding left no vector above the target, take the last positive element instead
+        double before = 0.0;
+        if (found != INT_MAX) {
+            before = base + incl - mine;
+            for (int k = 0; k < G - tid * kVecPerThread; ++k) before += loc[k];
+        }
+        const double rem2 = (found != INT_MAX) ? (rem - before) : INFINITY;
+        float w[EPV];
+        const int v = T * kVecPerChunk + G;
+        vector_weights<DT>(P, sel, rt, zd_row, v, w);
+        float runf = 0.f;
+        int pick = -1, lastw = 0;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+            runf = (i == 0) ? w[0] : __fadd_rn(runf, w[i]);
+            if (w[i] > 0.f) lastw = i;
+            if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
+        }
+        if (pick < 0) pick = lastw;
+        int token = rt.first_elem(v) + pick;
+        token = min(max(token, 0), P.V_t - 1);
+        P.next_token[b] = token;
+        P.cnt_sample[b] = 0;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// host side
+// ---------------------------------------------------------------------------
+
+thread_local char g_cuda_error[256] = "";
+
+int cuda_fail(cudaError_t e, const char *what) {
+    snprintf(g_cuda_error, sizeof g_cuda_error, "%s: %s", what, cudaGetErrorString(e));
+    return TLI_ERR_CUDA;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+int chunks_per_row(int V, int dtype) {
+    const long long epv = dtype == TLI_F32 ? 4 : 8;
+    return static_cast<int>((static_cast<long long>(V) + epv - 1 + epv * kVecPerChunk - 1) / (epv * kVecPerChunk));
+}
+
+struct Layout {
+    size_t part_t, part_d, sel, tilesum, total;
+    int nct, ncd;
+};
+
+Layout make_layout(int B, int K, int V_t, int V_d, int dtype) {
+    Layout L;
+    L.nct = chunks_per_row(V_t, dtype);
+    L.ncd = chunks_per_row(V_d, dtype);
+    size_t off = 0;
+    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nct, 256);
+    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.ncd, 256);
+    L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
+    L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.nct, 256);
+    L.total = off;
+    return L;
+}
+
+}  // namespace
+
+struct tli_ctx {
+    int device;
+    int32_t V_t, V_d, n_mapped;
+    int *d_map;
+    int *d_inv;
+    uint32_t *d_mask;
+    unsigned *d_counters;       // [2 * (TLI_MAX_B + 1)], zero between calls
+};
+
+extern "C" {
+
+int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_t *id_map_host) {
+    if (!out) return TLI_ERR_ARG;
+    *out = nullptr;
+    if (!id_map_host || device < 0) return TLI_ERR_ARG;
+    if (V_t < 1 || V_d < 1) return TLI_ERR_ARG;
+    if (V_t > TLI_MAX_V || V_d > TLI_MAX_V) return TLI_ERR_UNSUPPORTED;
+    // host-side validation and derived tables, before any CUDA call
+    std::vector<int32_t> inv(static_cast<size_t>(V_t), -1);
+    const size_t mask_words = (static_cast<size_t>(V_d) + 31) / 32 + 2;
+    std::vector<uint32_t> mask(mask_words, 0u);
+    int32_t n_mapped = 0;
+    for (int32_t x = 0; x < V_d; ++x) {
+        const int32_t t = id_map_host[x];
+        if (t == -1) continue;
+        if (t < 0 || t >= V_t || inv[t] != -1) return TLI_ERR_BAD_MAP;
+        inv[t] = x;
+        mask[x >> 5] |= 1u << (x & 31);
+        ++n_mapped;
+    }
+    int prev = -1;
+    cudaError_t e = cudaGetDevice(&prev);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    e = cudaSetDevice(device);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaSetDevice");
+    tli_ctx *c = new (std::nothrow) tli_ctx();
+    if (!c) { cudaSetDevice(prev); return TLI_ERR_ARG; }
+    c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
+    c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
+    int rc = TLI_OK;
+    do {
+        if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
+        if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
+        if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
+        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * 2 * (TLI_MAX_B + 1))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
+        if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
+        if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
+        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * 2 * (TLI_MAX_B + 1))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
+    } while (0);
+    if (rc != TLI_OK) {
+        cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
+        delete c;
+        cudaSetDevice(prev);
+        return rc;
+    }
+    cudaSetDevice(prev);
+    *out = c;
+    return TLI_OK;
+}
+
+int tli_destroy(tli_ctx *ctx) {
+    if (!ctx) return TLI_ERR_ARG;
+    int prev = -1;
+    cudaGetDevice(&prev);
+    cudaSetDevice(ctx->device);
+    cudaFree(ctx->d_map); cudaFree(ctx->d_inv); cudaFree(ctx->d_mask); cudaFree(ctx->d_counters);
+    if (prev >= 0) cudaSetDevice(prev);
+    delete ctx;
+    return TLI_OK;
+}
+
+size_t tli_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype) {
+    if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    return make_layout(B, K, ctx->V_t, ctx->V_d, dtype).total;
+}
+
+int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped) {
+    if (!ctx) return TLI_ERR_ARG;
+    if (V_t) *V_t = ctx->V_t;
+    if (V_d) *V_d = ctx->V_d;
+    if (n_mapped) *n_mapped = ctx->n_mapped;
+    return TLI_OK;
+}
+
+int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
+    if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->target_logits || !a->drafter_logits || !a->draft_ids || !a->temperature || !a->uniforms ||
+        !a->accepted || !a->next_token)
+        return TLI_ERR_ARG;
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
+        return TLI_ERR_ARG;
+    if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
+    const Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype);
+    if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
+        return TLI_ERR_WORKSPACE;
+
+    Params P;
+    P.B = a->B; P.K = a->K; P.V_t = ctx->V_t; P.V_d = ctx->V_d;
+    P.zt = a->target_logits; P.t_sb = a->t_stride_b; P.t_sk = a->t_stride_k;
+    P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sk = a->d_stride_k;
+    P.map = ctx->d_map; P.inv = ctx->d_inv; P.maskbits = ctx->d_mask; P.n_mapped = ctx->n_mapped;
+    P.draft = a->draft_ids; P.tau = a->temperature; P.u = a->uniforms;
+    P.accepted = a->accepted; P.next_token = a->next_token; P.status = a->row_status;
+    P.p_out = a->p_draft; P.q_out = a->q_draft;
+    char *ws = reinterpret_cast<char *>(a->workspace);
+    P.part_t = reinterpret_cast<float2 *>(ws + L.part_t);
+    P.part_d = reinterpret_cast<float2 *>(ws + L.part_d);
+    P.sel = reinterpret_cast<RowSel *>(ws + L.sel);
+    P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
+    P.cnt_stats = ctx->d_counters;
+    P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
+    P.nct = L.nct; P.ncd = L.ncd;
+
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const dim3 grid1(static_cast<unsigned>((a->K + 1) * L.nct + a->K * L.ncd), static_cast<unsigned>(a->B));
+    const dim3 grid2(static_cast<unsigned>(L.nct), static_cast<unsigned>(a->B));
+    if (a->dtype == TLI_F32) tli_stats_kernel<TLI_F32><<<grid1, kThreads, 0, stream>>>(P);
+    else tli_stats_kernel<TLI_BF16><<<grid1, kThreads, 0, stream>>>(P);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
+
+    // the sampling pass may be scheduled while the statistics pass drains
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cfg.gridDim = grid2; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_F32>, P);
+    else e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_BF16>, P);
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
+    return TLI_OK;
+}
+
+const char *tli_status_string(int code) {
+    switch (code) {
+        case TLI_OK: return "ok";
+        case TLI_ERR_ARG: return "bad argument";
+        case TLI_ERR_BAD_MAP: return "id map out of range or not injective";
+        case TLI_ERR_CUDA: return "CUDA runtime error";
+        case TLI_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case TLI_ERR_UNSUPPORTED: return "size beyond the library's limits";
+        default: return "unknown code";
+    }
+}
+
+const char *tli_last_cuda_error(void) { return g_cuda_error; }
+
+}  // extern "C"

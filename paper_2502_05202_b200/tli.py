@@ -1,0 +1,206 @@
+"""Thin ctypes binding of the C ABI in include/tli.h.
+
+Argument marshalling only: every step of the verification runs in the CUDA
+library.  torch is used for device memory and streams.  There is no CPU
+fallback: if ``libtli.so`` is missing or cannot be loaded, importing a function
+from here raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Dict, Optional
+
+import numpy as np
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtli.so")
+
+TLI_F32 = 0
+TLI_BF16 = 1
+TLI_OK = 0
+TLI_ERR_ARG = -1
+TLI_ERR_BAD_MAP = -2
+TLI_ERR_CUDA = -3
+TLI_ERR_WORKSPACE = -4
+TLI_ERR_UNSUPPORTED = -5
+TLI_ROW_DRAFT_RANGE = 1
+TLI_ROW_DRAFT_UNMAPPED = 2
+TLI_ROW_NONFINITE = 4
+TLI_ROW_FALLBACK = 8
+TLI_ROW_BAD_TEMPERATURE = 32
+TLI_MAX_B = 65535
+TLI_MAX_K = 64
+TLI_MAX_V = 1048576
+
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_ctx_info",
+           "tli_status_string", "tli_last_cuda_error")
+
+
+class tli_verify_args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_k", ctypes.c_int64),
+        ("draft_ids", ctypes.c_void_p), ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
+        ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+class TLIError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        lib = load()
+        msg = lib.tli_status_string(code).decode()
+        detail = lib.tli_last_cuda_error().decode() if code == TLI_ERR_CUDA else ""
+        super().__init__("%s failed: %s (%d)%s" % (where, msg, code, (": " + detail) if detail else ""))
+        self.code = code
+
+
+_lib = None
+
+
+def load() -> ctypes.CDLL:
+    """Load libtli.so (built by ``python -m paper_2502_05202_b200.build``); raises if absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError("CUDA library %s is missing; run `python -m paper_2502_05202_b200.build`" % LIB_PATH)
+        lib = ctypes.CDLL(LIB_PATH)
+        lib.tli_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_int32, ctypes.c_int32,
+                                   ctypes.c_void_p]
+        lib.tli_create.restype = ctypes.c_int
+        lib.tli_destroy.argtypes = [ctypes.c_void_p]
+        lib.tli_destroy.restype = ctypes.c_int
+        lib.tli_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_workspace_bytes.restype = ctypes.c_size_t
+        lib.tli_verify.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p]
+        lib.tli_verify.restype = ctypes.c_int
+        lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
+        lib.tli_ctx_info.restype = ctypes.c_int
+        lib.tli_status_string.argtypes = [ctypes.c_int]
+        lib.tli_status_string.restype = ctypes.c_char_p
+        lib.tli_last_cuda_error.argtypes = []
+        lib.tli_last_cuda_error.restype = ctypes.c_char_p
+        _lib = lib
+    return _lib
+
+
+def tli_create(device: int, V_t: int, V_d: int, id_map) -> int:
+    """tli_create(): returns the context handle; ``id_map`` is a host int32 array [V_d]."""
+    m = np.ascontiguousarray(id_map, dtype=np.int32)
+    if m.shape != (V_d,):
+        raise ValueError("id_map must have V_d entries")
+    h = ctypes.c_void_p()
+    rc = load().tli_create(ctypes.byref(h), int(device), int(V_t), int(V_d), m.ctypes.data)
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_create")
+    return h.value
+
+
+def tli_destroy(ctx: int) -> None:
+    rc = load().tli_destroy(ctx)
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_destroy")
+
+
+def tli_workspace_bytes(ctx: int, B: int, K: int, dtype: int) -> int:
+    return int(load().tli_workspace_bytes(ctx, B, K, dtype))
+
+
+def _logit_dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return TLI_F32
+    if t.dtype == torch.bfloat16:
+        return TLI_BF16
+    raise TypeError("logits must be float32 or bfloat16")
+
+
+def make_args(target_logits: torch.Tensor, drafter_logits: torch.Tensor, draft_ids: torch.Tensor,
+              temperature: torch.Tensor, uniforms: torch.Tensor, accepted: torch.Tensor,
+              next_token: torch.Tensor, workspace: torch.Tensor, row_status: Optional[torch.Tensor] = None,
+              p_draft: Optional[torch.Tensor] = None, q_draft: Optional[torch.Tensor] = None) -> tli_verify_args:
+    """Fill a tli_verify_args from device tensors (no copies; the tensors must outlive the call)."""
+    B, K1, _ = target_logits.shape
+    K = K1 - 1
+    dt = _logit_dtype(target_logits)
+    if _logit_dtype(drafter_logits) != dt:
+        raise TypeError("both logit tensors must have the same dtype")
+    if target_logits.stride(2) != 1 or drafter_logits.stride(2) != 1:
+        raise ValueError("the vocabulary axis must be contiguous")
+    if drafter_logits.shape[0] != B or drafter_logits.shape[1] != K:
+        raise ValueError("drafter logits must be [B, K, V_d]")
+    for name, t, dtype, shape in (("draft_ids", draft_ids, torch.int32, (B, K)),
+                                  ("temperature", temperature, torch.float32, (B,)),
+                                  ("uniforms", uniforms, torch.float32, (B, K + 1)),
+                                  ("accepted", accepted, torch.int32, (B,)),
+                                  ("next_token", next_token, torch.int32, (B,))):
+        if t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous %s tensor of shape %s" % (name, dtype, shape))
+    opt = lambda t: None if t is None else t.data_ptr()
+    return tli_verify_args(
+        B, K, dt,
+        target_logits.data_ptr(), target_logits.stride(0), target_logits.stride(1),
+        drafter_logits.data_ptr(), drafter_logits.stride(0), drafter_logits.stride(1),
+        draft_ids.data_ptr(), temperature.data_ptr(), uniforms.data_ptr(),
+        accepted.data_ptr(), next_token.data_ptr(), opt(row_status), opt(p_draft), opt(q_draft),
+        workspace.data_ptr(), workspace.numel() * workspace.element_size())
+
+
+def tli_verify(ctx: int, args: tli_verify_args, stream: Optional[int] = None) -> None:
+    """tli_verify() on ``stream`` (a cudaStream_t as int; default: torch's current stream)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_verify(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_verify")
+
+
+class Verifier:
+    """Convenience owner of one context plus its scratch and output tensors."""
+
+    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0):
+        self.device = torch.device("cuda", device)
+        self.V_t, self.V_d = int(V_t), int(V_d)
+        self.ctx = tli_create(device, V_t, V_d, id_map)
+        self._ws: Optional[torch.Tensor] = None
+
+    def close(self) -> None:
+        if self.ctx:
+            tli_destroy(self.ctx)
+            self.ctx = 0
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def workspace(self, B: int, K: int, dtype: int) -> torch.Tensor:
+        need = tli_workspace_bytes(self.ctx, B, K, dtype)
+        if need == 0:
+            raise TLIError(TLI_ERR_UNSUPPORTED, "tli_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
+        return self._ws
+
+    def verify(self, target_logits, drafter_logits, draft_ids, temperature, uniforms,
+               diagnostics: bool = True) -> Dict[str, torch.Tensor]:
+        """One call on torch's current stream; returns device tensors (no synchronisation)."""
+        B, K1, _ = target_logits.shape
+        K = K1 - 1
+        dev = self.device
+        out = {"accepted": torch.empty(B, dtype=torch.int32, device=dev),
+               "next_token": torch.empty(B, dtype=torch.int32, device=dev),
+               "row_status": torch.empty(B, dtype=torch.int32, device=dev)}
+        if diagnostics:
+            out["p_draft"] = torch.empty(B, K, dtype=torch.float32, device=dev)
+            out["q_draft"] = torch.empty(B, K, dtype=torch.float32, device=dev)
+        ws = self.workspace(B, K, _logit_dtype(target_logits))
+        args = make_args(target_logits, drafter_logits, draft_ids, temperature, uniforms,
+                         out["accepted"], out["next_token"], ws, out["row_status"],
+                         out.get("p_draft"), out.get("q_draft"))
+        tli_verify(self.ctx, args)
+        return out
