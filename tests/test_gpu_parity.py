@@ -1,0 +1,275 @@
+"""Parity of the CUDA library with the fp64 oracle, element by element, through the C ABI."""
+import ctypes
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2502_05202_b200 import tli, workload as wl
+from parity_util import check, compare, run_gpu, run_oracle, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+def bf16(x):
+    return wl.f32_to_bf16_bits(np.asarray(x, np.float32))
+
+
+# --------------------------------------------------------------------------
+# small and medium sizes: several tiles, ragged tails, both storage types
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+@pytest.mark.parametrize("V_t,V_d,K,B", [(3, 4, 1, 5), (11, 13, 3, 9), (64, 50, 2, 7), (257, 300, 5, 6),
+                                         (1000, 999, 4, 4)])
+def test_tiny_vocabularies(dtype, V_t, V_d, K, B):
+    cfg = wl.tiny_config(B=B, K=K, V_t=V_t, V_d=V_d, dtype=dtype, f_mapped=0.6,
+                         temperatures=(0.5, 1.0, 1.3), seed=11 + V_t)
+    rep = check(wl.make_batch(cfg))
+    assert rep.exact + rep.excused_sampler + rep.excused_threshold >= B
+
+
+@pytest.mark.parametrize("dtype,V_t,V_d", [
+    (wl.F32, 3 * 4096 + 37, 2 * 4096 + 5),      # 16 KB chunks of fp32: three full + ragged
+    (wl.BF16, 2 * 8192 + 13, 8192 + 8191),      # odd lengths: bf16 rows start off 16-byte alignment
+    (wl.BF16, 20001, 9999),
+    (wl.F32, 4096, 8192),                       # exact multiples
+])
+def test_several_tiles_and_ragged_tails(dtype, V_t, V_d):
+    cfg = wl.tiny_config(B=6, K=3, V_t=V_t, V_d=V_d, dtype=dtype, f_mapped=0.5,
+                         temperatures=(0.7, 1.0), greedy_rows="interleaved", seed=5)
+    rep = check(wl.make_batch(cfg))
+    print(rep)
+
+
+@pytest.mark.parametrize("mode", ["intersection", "raw"])
+def test_draft_modes_and_low_overlap(mode):
+    cfg = wl.tiny_config(B=16, K=6, V_t=5000, V_d=7001, dtype=wl.BF16, f_mapped=0.12, sigma_d=0.5,
+                         temperatures=(0.8, 1.0), seed=21)
+    batch = wl.make_batch(cfg, draft_mode=mode)
+    rep = check(batch)
+    if mode == "raw":
+        assert (run_oracle(batch)["flags"] & oracle.FLAG_DRAFT_UNMAPPED).any()
+
+
+def test_strided_and_offset_inputs():
+    """Rows padded to odd strides and a base pointer one element into the buffer."""
+    cfg = wl.tiny_config(B=5, K=3, V_t=4100, V_d=3001, dtype=wl.BF16, f_mapped=0.7, seed=31)
+    batch = wl.make_batch(cfg)
+    B, K = cfg.B, cfg.K
+    dev = to_device(batch)
+    big_t = torch.zeros(B, K + 2, cfg.V_t + 3, dtype=torch.bfloat16, device="cuda")
+    big_d = torch.zeros(B, K + 1, cfg.V_d + 5, dtype=torch.bfloat16, device="cuda")
+    big_t[:, :K + 1, 1:cfg.V_t + 1] = dev["target_logits"]
+    big_d[:, :K, 1:cfg.V_d + 1] = dev["drafter_logits"]
+    dev2 = dict(dev, target_logits=big_t[:, :K + 1, 1:cfg.V_t + 1], drafter_logits=big_d[:, :K, 1:cfg.V_d + 1])
+    assert dev2["target_logits"].data_ptr() % 16 != 0
+    gpu = run_gpu(batch, dev=dev2)
+    rep = compare(batch, gpu)
+    assert rep.ok(), str(rep)
+    ref = run_gpu(batch)
+    for k in ("accepted", "next_token", "row_status"):
+        np.testing.assert_array_equal(gpu[k], ref[k])
+
+
+# --------------------------------------------------------------------------
+# the five workloads at full size, every row, in the benchmark's launch configuration
+# --------------------------------------------------------------------------
+
+@pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
+def test_full_size_workloads(name):
+    cfg = wl.config_by_name(name)
+    batch = wl.make_batch(cfg)
+    rep = check(batch)
+    print(name, rep)
+    assert rep.rows == cfg.B
+    # near-ties are rare: almost every row must match exactly
+    assert rep.exact >= cfg.B - max(2, cfg.B // 16)
+
+
+def test_interleaved_greedy_rows_and_raw_drafts_on_cfg4_shape():
+    cfg = dataclasses.replace(wl.config_by_name("cfg4"), B=8, K=6, greedy_rows="interleaved", seed=77)
+    rep = check(wl.make_batch(cfg, draft_mode="raw"))
+    print(rep)
+
+
+# --------------------------------------------------------------------------
+# degenerate cases of the method
+# --------------------------------------------------------------------------
+
+def test_empty_intersection_rejects_everything():
+    cfg = wl.tiny_config(B=6, K=3, V_t=700, V_d=500, f_mapped=0.0, seed=3)
+    batch = wl.make_batch(cfg)
+    assert (batch["id_map"] < 0).all()
+    gpu = run_gpu(batch)
+    assert (gpu["accepted"] == 0).all()
+    assert (gpu["row_status"] == (tli.TLI_ROW_DRAFT_UNMAPPED | tli.TLI_ROW_FALLBACK)).all()
+    assert compare(batch, gpu).ok()
+
+
+def test_identity_map_with_equal_logits_accepts_everything():
+    rng = np.random.default_rng(0)
+    V, K, B = 9000, 4, 5
+    zt = rng.normal(0, 3, (B, K + 1, V)).astype(np.float32)
+    batch = {"target_logits": zt, "drafter_logits": zt[:, :K].copy(), "id_map": np.arange(V, dtype=np.int32),
+             "draft_ids": rng.integers(0, V, (B, K)).astype(np.int32), "temperature": np.ones(B, np.float32),
+             "uniforms": np.full((B, K + 1), 1 - 2.0 ** -24, np.float32)}
+    gpu = run_gpu(batch)
+    assert (gpu["accepted"] == K).all()
+    assert compare(batch, gpu).ok()
+
+
+def test_zero_residual_falls_back_to_target_distribution():
+    """p == q' everywhere and a draft id out of range: rejected, residual mass 0, sample from p."""
+    rng = np.random.default_rng(1)
+    V, K, B = 5000, 2, 4
+    zt = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
+    d = rng.integers(0, V, (B, K)).astype(np.int32)
+    d[:, 0] = V + 3
+    d[1, 0] = -1
+    batch = {"target_logits": zt, "drafter_logits": zt[:, :K].copy(), "id_map": np.arange(V, dtype=np.int32),
+             "draft_ids": d, "temperature": np.full(B, 0.9, np.float32),
+             "uniforms": rng.random((B, K + 1)).astype(np.float32)}
+    gpu = run_gpu(batch)
+    assert (gpu["accepted"] == 0).all()
+    assert (gpu["row_status"] == (tli.TLI_ROW_DRAFT_RANGE | tli.TLI_ROW_FALLBACK)).all()
+    assert compare(batch, gpu).ok()
+
+
+def test_minus_infinity_logits_are_zero_probability_tokens():
+    cfg = wl.tiny_config(B=6, K=3, V_t=6000, V_d=5000, dtype=wl.F32, f_mapped=0.5, seed=41)
+    batch = wl.make_batch(cfg)
+    rng = np.random.default_rng(2)
+    kill_t = rng.random(batch["target_logits"].shape) < 0.3
+    kill_d = rng.random(batch["drafter_logits"].shape) < 0.3
+    # keep the drafted tokens alive on both sides
+    for b in range(cfg.B):
+        for j in range(cfg.K):
+            x = batch["draft_ids"][b, j]
+            kill_d[b, j, x] = False
+            kill_t[b, j, batch["id_map"][x]] = False
+    gpu_in = dict(batch, target_logits=np.where(kill_t, -np.inf, batch["target_logits"]).astype(np.float32),
+                  drafter_logits=np.where(kill_d, -np.inf, batch["drafter_logits"]).astype(np.float32))
+    ref_in = dict(batch, target_logits=np.where(kill_t, -1e30, batch["target_logits"]).astype(np.float32),
+                  drafter_logits=np.where(kill_d, -1e30, batch["drafter_logits"]).astype(np.float32))
+    gpu = run_gpu(gpu_in)
+    assert (gpu["row_status"] == 0).all()
+    rep = compare(ref_in, gpu)
+    assert rep.ok(), str(rep)
+    dead = kill_t[np.arange(cfg.B), gpu["accepted"], gpu["next_token"]]
+    assert not dead.any()
+
+
+def test_nan_and_plus_infinity_flag_the_row():
+    cfg = wl.tiny_config(B=6, K=3, V_t=6000, V_d=5000, dtype=wl.BF16, f_mapped=0.5, seed=42)
+    batch = wl.make_batch(cfg)
+    zt = wl.bf16_bits_to_f32(batch["target_logits"]).copy()
+    zd = wl.bf16_bits_to_f32(batch["drafter_logits"]).copy()
+    zt[1, 2, 4097] = np.nan
+    zt[3, 0, 17] = np.inf
+    mapped = np.flatnonzero(batch["id_map"] >= 0)
+    zd[4, 1, mapped[5]] = np.nan
+    bad = dict(batch, target_logits=bf16(zt), drafter_logits=bf16(zd))
+    gpu = run_gpu(bad)
+    flagged = (gpu["row_status"] & tli.TLI_ROW_NONFINITE) != 0
+    assert flagged.tolist() == [False, True, False, True, True, False]
+    assert (gpu["accepted"][flagged] == 0).all() and (gpu["next_token"][flagged] == 0).all()
+    clean = run_gpu(batch)
+    for k in ("accepted", "next_token"):
+        np.testing.assert_array_equal(gpu[k][~flagged], clean[k][~flagged])
+
+
+def test_bad_temperature_flags_the_row():
+    cfg = wl.tiny_config(B=5, K=2, V_t=500, V_d=400, seed=43)
+    batch = wl.make_batch(cfg)
+    batch["temperature"] = np.array([1.0, -0.5, np.nan, np.inf, 0.0], np.float32)
+    gpu = run_gpu(batch)
+    assert gpu["row_status"].tolist()[1:4] == [tli.TLI_ROW_BAD_TEMPERATURE] * 3
+    assert (gpu["accepted"][1:4] == 0).all()
+    orc = run_oracle(dict(batch, temperature=np.array([1.0, 1.0, 1.0, 1.0, 0.0], np.float32)))
+    for b in (0, 4):
+        assert gpu["accepted"][b] == orc["accepted"][b] and gpu["next_token"][b] == orc["next_token"][b]
+
+
+def test_greedy_ties_are_bit_exact():
+    """bf16 logits tie often; the lowest index must win in every reduction step."""
+    rng = np.random.default_rng(5)
+    V_t, V_d, K, B = 3 * 8192 + 100, 9000, 4, 12
+    zt = np.round(rng.normal(0, 1, (B, K + 1, V_t))).astype(np.float32)     # few distinct values -> many ties
+    zd = rng.normal(0, 1, (B, K, V_d)).astype(np.float32)
+    cfgm = wl.tiny_config(V_t=V_t, V_d=V_d, f_mapped=0.8, seed=9)
+    id_map = wl.make_id_map(cfgm)
+    first_max = zt.argmax(axis=2)
+    inv = np.full(V_t, -1)
+    inv[id_map[id_map >= 0]] = np.flatnonzero(id_map >= 0)
+    d = np.where(inv[first_max[:, :K]] >= 0, inv[first_max[:, :K]], 0).astype(np.int32)
+    d[::3, 1] = (d[::3, 1] + 1) % V_d
+    batch = {"target_logits": bf16(zt), "drafter_logits": bf16(zd), "id_map": id_map, "draft_ids": d,
+             "temperature": np.zeros(B, np.float32), "uniforms": np.zeros((B, K + 1), np.float32)}
+    gpu = run_gpu(batch)
+    orc = run_oracle(batch)
+    np.testing.assert_array_equal(gpu["accepted"], orc["accepted"])
+    np.testing.assert_array_equal(gpu["next_token"], orc["next_token"])
+    assert gpu["accepted"].max() == K
+
+
+@pytest.mark.parametrize("B,K", [(1, 1), (1, 64), (300, 1)])
+def test_extreme_batch_and_draft_counts(B, K):
+    cfg = wl.tiny_config(B=B, K=K, V_t=2000, V_d=1500, dtype=wl.BF16, f_mapped=0.6, sigma_d=0.3, seed=50 + K)
+    check(wl.make_batch(cfg))
+
+
+def test_large_vocabulary_near_the_limit():
+    cfg = wl.tiny_config(B=2, K=1, V_t=tli.TLI_MAX_V, V_d=tli.TLI_MAX_V - 7, dtype=wl.F32, f_mapped=0.5, seed=60)
+    check(wl.make_batch(cfg))
+
+
+def test_repeated_calls_reuse_the_context():
+    cfg = wl.tiny_config(B=7, K=3, V_t=9000, V_d=7000, dtype=wl.BF16, f_mapped=0.6, seed=61)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    first = run_gpu(batch, v)
+    for _ in range(3):
+        again = run_gpu(batch, v)
+        for k in first:
+            np.testing.assert_array_equal(first[k], again[k])
+    small = wl.make_batch(dataclasses.replace(cfg, B=2, K=2, seed=62))
+    assert compare(small, run_gpu(small, v)).ok()
+    v.close()
+
+
+# --------------------------------------------------------------------------
+# host-detectable argument errors
+# --------------------------------------------------------------------------
+
+def test_argument_errors_are_reported_not_launched():
+    cfg = wl.tiny_config(B=2, K=2, V_t=300, V_d=200, seed=70)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    dev = to_device(batch)
+    acc = torch.zeros(2, dtype=torch.int32, device="cuda")
+    nxt = torch.zeros(2, dtype=torch.int32, device="cuda")
+    ws = v.workspace(2, 2, tli.TLI_F32)
+    good = lambda: tli.make_args(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"], dev["temperature"],
+                                 dev["uniforms"], acc, nxt, ws)
+    lib = tli.load()
+    call = lambda a: lib.tli_verify(v.ctx, ctypes.byref(a), None)
+    a = good(); a.workspace_bytes = 16
+    assert call(a) == tli.TLI_ERR_WORKSPACE
+    a = good(); a.workspace = None
+    assert call(a) == tli.TLI_ERR_WORKSPACE
+    a = good(); a.K = 0
+    assert call(a) == tli.TLI_ERR_ARG
+    a = good(); a.K = tli.TLI_MAX_K + 1
+    assert call(a) == tli.TLI_ERR_UNSUPPORTED
+    a = good(); a.dtype = 7
+    assert call(a) == tli.TLI_ERR_ARG
+    a = good(); a.uniforms = None
+    assert call(a) == tli.TLI_ERR_ARG
+    assert lib.tli_verify(None, ctypes.byref(good()), None) == tli.TLI_ERR_ARG
+    assert tli.tli_workspace_bytes(v.ctx, 0, 1, 0) == 0
+    assert call(good()) == tli.TLI_OK
+    torch.cuda.synchronize()
+    v.close()
