@@ -512,7 +512,8 @@ __device__ __forceinline__ void vector_weights(const Params &P, const RowSel &se
             const float zdv = load_elt<DT>(zd_row, x[i]);
             q = __fmul_rn(ex2(__fmaf_rn(zdv, sel.s, ncd)), sel.rs_d);
         }
-        w[i] = fmaxf(0.f, __fmaf_rn(et, sel.rs_t, -q));
+        // p and q' are each rounded before the subtraction, so that equal distributions leave exactly 0
+        w[i] = fmaxf(0.f, __fsub_rn(__fmul_rn(et, sel.rs_t), q));
     }
 }
 

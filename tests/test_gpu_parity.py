@@ -122,7 +122,10 @@ def test_identity_map_with_equal_logits_accepts_everything():
 
 
 def test_zero_residual_falls_back_to_target_distribution():
-    """p == q' everywhere and a draft id out of range: rejected, residual mass 0, sample from p."""
+    """p == q' bit for bit and a draft id out of range: rejected, residual mass exactly 0, sample from p.
+
+    The oracle forms q' as q / M with M = 1 +- 1e-16, so its own residual is rounding noise instead of 0;
+    the expected token is therefore the oracle's sample from p_0 (same logits, empty intersection)."""
     rng = np.random.default_rng(1)
     V, K, B = 5000, 2, 4
     zt = rng.normal(0, 2, (B, K + 1, V)).astype(np.float32)
@@ -135,7 +138,9 @@ def test_zero_residual_falls_back_to_target_distribution():
     gpu = run_gpu(batch)
     assert (gpu["accepted"] == 0).all()
     assert (gpu["row_status"] == (tli.TLI_ROW_DRAFT_RANGE | tli.TLI_ROW_FALLBACK)).all()
-    assert compare(batch, gpu).ok()
+    from_p = run_oracle(dict(batch, id_map=np.full(V, -1, np.int32), draft_ids=np.zeros((B, K), np.int32)))
+    assert (from_p["accepted"] == 0).all()
+    np.testing.assert_array_equal(gpu["next_token"], from_p["next_token"])
 
 
 def test_minus_infinity_logits_are_zero_probability_tokens():
@@ -196,7 +201,7 @@ def test_bad_temperature_flags_the_row():
 def test_greedy_ties_are_bit_exact():
     """bf16 logits tie often; the lowest index must win in every reduction step."""
     rng = np.random.default_rng(5)
-    V_t, V_d, K, B = 3 * 8192 + 100, 9000, 4, 12
+    V_t, V_d, K, B = 3 * 8192 + 100, 30000, 4, 12
     zt = np.round(rng.normal(0, 1, (B, K + 1, V_t))).astype(np.float32)     # few distinct values -> many ties
     zd = rng.normal(0, 1, (B, K, V_d)).astype(np.float32)
     cfgm = wl.tiny_config(V_t=V_t, V_d=V_d, f_mapped=0.8, seed=9)
@@ -235,7 +240,7 @@ def test_repeated_calls_reuse_the_context():
         again = run_gpu(batch, v)
         for k in first:
             np.testing.assert_array_equal(first[k], again[k])
-    small = wl.make_batch(dataclasses.replace(cfg, B=2, K=2, seed=62))
+    small = wl.make_batch(dataclasses.replace(cfg, B=2, K=2))      # same seed: same id map
     assert compare(small, run_gpu(small, v)).ok()
     v.close()
 
