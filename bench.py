@@ -1,0 +1,384 @@
+#!/usr/bin/env python
+"""Benchmark of TLI verification (draft positions verified per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl reference]
+
+A step is one tli_verify() call on one synthetic batch: both kernels, all
+sequences.  The headline workload is the largest of the five (cfg3: B=256, K=4,
+V_t=256000, V_d=128256, fp32 logits, 1.8 GB per call, larger than L2).  With N>1
+(under torchrun) every rank verifies its own copy of the batch -- sequences are
+independent, there is no collective on the data path -- and the value is the sum
+over ranks divided by the slowest rank's time.
+
+Prints ONE JSON line.  `--impl reference` times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "draft positions verified/s"
+UNIT = "positions/s"
+L2_ROTATE_BYTES = 400 << 20          # distinct input bytes cycled through when one batch fits in L2
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+def algorithmic_bytes(cfg, batch) -> int:
+    """All logits read once; temperature-0 sequences do not read drafter logits."""
+    import numpy as np
+    greedy = int((np.asarray(batch["temperature"]) == 0).sum())
+    return cfg.elt * (cfg.B * (cfg.K + 1) * cfg.V_t + (cfg.B - greedy) * cfg.K * cfg.V_d)
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons of one GPU, sampled every 200 ms in the background."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "200"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            threading.Thread(target=self._read, daemon=True).start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------
+# CPU oracle legs
+# ---------------------------------------------------------------------------
+
+def time_oracle(batch, positions, min_seconds=10.0, max_reps=50):
+    """The oracle as it stands, rows split over all host cores; returns (positions/s, cores, reps, seconds)."""
+    import oracle
+    cores = os.cpu_count() or 1
+    oracle.build()
+    run = lambda: oracle.verify(batch["target_logits"], batch["drafter_logits"], batch["id_map"], batch["draft_ids"],
+                                batch["temperature"], batch["uniforms"], threads=cores)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        run()
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds or reps >= max_reps:
+            break
+    return positions * reps / dt, min(cores, len(batch["temperature"])), reps, dt
+
+
+def reference_arm(args):
+    """`--impl reference`: the CPU oracle on the same workload, rank 0 only."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    from paper_2502_05202_b200 import workload as wl
+    import oracle
+    cfg = wl.config_by_name(args.config)
+    cores = os.cpu_count() or 1
+    rows = list(range(min(cfg.B, max(cores, 8) * 2)))          # bounded sample: a few rows per core
+    batch = wl.make_batch(cfg, rows=rows)
+    positions = len(rows) * cfg.K
+    oracle.build()
+    run = lambda: oracle.verify(batch["target_logits"], batch["drafter_logits"], batch["id_map"], batch["draft_ids"],
+                                batch["temperature"], batch["uniforms"], threads=cores)
+    for _ in range(args.warmup):
+        run()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        run()
+    dt = time.perf_counter() - t0
+    value = positions * args.steps / dt
+    used = min(cores, len(rows))
+    sample = "first %d of %d sequences of %s per step (%d positions), all rows in fp64" % (len(rows), cfg.B, cfg.name, positions)
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt / args.steps * 1e3,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": workload_config(cfg, None),
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_config(cfg, l2_note):
+    c = {"workload": cfg.name, "B": cfg.B, "K": cfg.K, "V_t": cfg.V_t, "V_d": cfg.V_d,
+         "logits": "f32" if cfg.elt == 4 else "bf16", "mapped_fraction": cfg.f_mapped,
+         "positions_per_step": cfg.positions, "logit_bytes_per_step": cfg.logit_bytes}
+    if l2_note:
+        c["l2"] = l2_note
+    return c
+
+
+# ---------------------------------------------------------------------------
+# GPU arm
+# ---------------------------------------------------------------------------
+
+class GpuCase:
+    """One workload resident on the device: enough copies of the inputs to defeat L2, outputs, scratch."""
+
+    def __init__(self, cfg, device, torch, tli, wl, want_host=False):
+        self.cfg, self.torch, self.tli = cfg, torch, tli
+        self.batch = wl.make_batch(cfg)
+        self.bytes = algorithmic_bytes(cfg, self.batch)
+        l2 = torch.cuda.get_device_properties(device).L2_cache_size
+        self.copies = 1 if cfg.logit_bytes > 2 * l2 else max(2, -(-L2_ROTATE_BYTES // cfg.logit_bytes))
+        self.l2_note = ("inputs larger than L2 (%d MB per step vs %d MB)" % (cfg.logit_bytes >> 20, l2 >> 20)
+                        if self.copies == 1 else
+                        "%d distinct input copies rotated (%d MB in all vs %d MB L2)" %
+                        (self.copies, (self.copies * cfg.logit_bytes) >> 20, l2 >> 20))
+        b = self.batch
+        zt = torch.from_numpy(b["target_logits"])
+        zd = torch.from_numpy(b["drafter_logits"])
+        if zt.dtype == torch.uint16:
+            zt, zd = zt.view(torch.bfloat16), zd.view(torch.bfloat16)
+        self.host = None
+        if want_host:
+            self.host = {"zt": zt.pin_memory(), "zd": zd.pin_memory(),
+                         "draft": torch.from_numpy(b["draft_ids"]).pin_memory(),
+                         "tau": torch.from_numpy(b["temperature"]).pin_memory(),
+                         "u": torch.from_numpy(b["uniforms"]).pin_memory(),
+                         "out": torch.empty(2, cfg.B, dtype=torch.int32).pin_memory()}
+        self.zt = [zt.to(device)]
+        self.zd = [zd.to(device)]
+        for _ in range(self.copies - 1):
+            self.zt.append(self.zt[0].clone())
+            self.zd.append(self.zd[0].clone())
+        self.draft = torch.from_numpy(b["draft_ids"]).to(device)
+        self.tau = torch.from_numpy(b["temperature"]).to(device)
+        self.u = torch.from_numpy(b["uniforms"]).to(device)
+        self.out = torch.empty(2, cfg.B, dtype=torch.int32, device=device)      # accepted, next_token
+        self.status = torch.empty(cfg.B, dtype=torch.int32, device=device)
+        self.ver = tli.Verifier(cfg.V_t, cfg.V_d, b["id_map"], device=device.index)
+        self.ws = self.ver.workspace(cfg.B, cfg.K, tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16)
+        self.args = [tli.make_args(self.zt[i], self.zd[i], self.draft, self.tau, self.u, self.out[0], self.out[1],
+                                   self.ws, self.status) for i in range(self.copies)]
+        self.stream = torch.cuda.current_stream().cuda_stream
+        self.calls = 0
+
+    def step(self):
+        self.tli.tli_verify(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
+        self.calls += 1
+
+    def step_e2e(self):
+        """Host buffers in, host results out: H2D of every input, the call, D2H of (accepted, next_token)."""
+        h = self.host
+        self.zt[0].copy_(h["zt"], non_blocking=True)
+        self.zd[0].copy_(h["zd"], non_blocking=True)
+        self.draft.copy_(h["draft"], non_blocking=True)
+        self.tau.copy_(h["tau"], non_blocking=True)
+        self.u.copy_(h["u"], non_blocking=True)
+        self.tli.tli_verify(self.ver.ctx, self.args[0], self.stream)
+        h["out"].copy_(self.out, non_blocking=True)
+
+    def e2e_bytes(self):
+        h = self.host
+        h2d = sum(h[k].numel() * h[k].element_size() for k in ("zt", "zd", "draft", "tau", "u"))
+        return h2d, h["out"].numel() * h["out"].element_size()
+
+    def profile(self, steps):
+        a = b = 0.0
+        for _ in range(steps):
+            ms1, ms2 = self.tli.tli_verify_profile(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
+            self.calls += 1
+            a += ms1; b += ms2
+        return a / steps, b / steps
+
+    def check(self):
+        st = self.status.cpu()
+        assert int(st.abs().sum()) == 0, "row_status not clean on benchmark inputs"
+
+    def close(self):
+        self.ver.close()
+
+
+def timed(torch, dist, steps, fn, world):
+    """K steps between two events, barrier + synchronize on both sides, max over ranks; returns ms in all."""
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    if world > 1:
+        dist.barrier()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    if world > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    return ms
+
+
+def gpu_arm(args):
+    import torch
+    from paper_2502_05202_b200 import tli, workload as wl
+    tli.load()                                   # fails loudly when the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus %d needs torchrun with that many ranks" % args.gpus)
+    torch.cuda.set_device(local)
+    device = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+    peak, peak_kind = load_peaks()
+    cfg = wl.config_by_name(args.config)
+    case = GpuCase(cfg, device, torch, tli, wl, want_host=True)
+
+    for _ in range(max(args.warmup, 3)):
+        case.step()
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ms = timed(torch, dist, args.steps, case.step, world)
+    # the dominant kernel alone, with events around it, on the same stream and workload
+    case.profile(3)
+    ms_stats, ms_sample = case.profile(args.steps)
+    clocks = sampler.stop() if rank == 0 else None
+    case.check()
+    # end to end: host buffers in, host results out
+    for _ in range(2):
+        case.step_e2e()
+    ms_e2e = timed(torch, dist, max(3, min(args.steps, 10)), case.step_e2e, world)
+    e2e_steps = max(3, min(args.steps, 10))
+    h2d, d2h = case.e2e_bytes()
+
+    ms_step = ms / args.steps
+    value = world * cfg.positions / (ms_step * 1e-3)
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": dict(workload_config(cfg, case.l2_note), parallelism="sequences replicated per GPU, no collective"),
+        "clocks": clocks,
+        "e2e": {"value": world * cfg.positions / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
+                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
+        "gpu_launches": 2 * args.steps,
+        "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
+        "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
+                     "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
+                     "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
+                     "traffic": None, "algorithmic_bytes": case.bytes,
+                     "ms_stats_kernel": ms_stats, "ms_sample_kernel": ms_sample},
+    }
+    headline_batch = case.batch
+    case.close()
+    del case
+    torch.cuda.empty_cache()
+
+    if rank == 0 and world == 1 and not args.no_per_config:
+        per = []
+        for c in wl.CONFIGS:
+            if c.name == cfg.name:
+                per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
+                            "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
+                            "ms_sample_kernel": ms_sample})
+                continue
+            k = GpuCase(c, device, torch, tli, wl)
+            for _ in range(max(args.warmup, 3) + k.copies):
+                k.step()
+            steps = max(args.steps, 2 * k.copies)
+            m = timed(torch, None, steps, k.step, 1) / steps
+            k.profile(3)
+            a, b = k.profile(min(steps, 50))
+            k.check()
+            per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
+                        "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
+                        "ms_stats_kernel": a, "ms_sample_kernel": b, "l2": k.l2_note})
+            k.close()
+            del k
+            torch.cuda.empty_cache()
+        out["per_config"] = per
+
+    if rank == 0 and world == 1:
+        v, cores, reps, secs = time_oracle(headline_batch, cfg.positions)
+        out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                               "sample": "all %d sequences of %s, %d repetitions in %.1f s" % (cfg.B, cfg.name, reps, secs)}
+    if rank == 0:
+        print(json.dumps(out))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--config", default="cfg3")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-per-config", action="store_true", help="skip the four other workloads")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        reference_arm(args)
+    else:
+        gpu_arm(args)
+
+
+if __name__ == "__main__":
+    main()

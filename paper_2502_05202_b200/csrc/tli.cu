@@ -833,7 +833,7 @@ int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapp
     return TLI_OK;
 }
 
-int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
+static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, cudaEvent_t *ev) {
     if (!ctx || !a) return TLI_ERR_ARG;
     if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
     if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
@@ -867,12 +867,14 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     P.nct = L.nct; P.ncd = L.ncd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (ev) cudaEventRecord(ev[0], stream);
     const dim3 grid1(static_cast<unsigned>((a->K + 1) * L.nct + a->K * L.ncd), static_cast<unsigned>(a->B));
     const dim3 grid2(static_cast<unsigned>(L.nct), static_cast<unsigned>(a->B));
     if (a->dtype == TLI_F32) tli_stats_kernel<TLI_F32><<<grid1, kThreads, 0, stream>>>(P);
     else tli_stats_kernel<TLI_BF16><<<grid1, kThreads, 0, stream>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
+    if (ev) cudaEventRecord(ev[1], stream);
 
     // the sampling pass may be scheduled while the statistics pass drains
     cudaLaunchConfig_t cfg;
@@ -885,7 +887,29 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_F32>, P);
     else e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_BF16>, P);
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
+    if (ev) cudaEventRecord(ev[2], stream);
     return TLI_OK;
+}
+
+int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
+    return verify_impl(ctx, a, cuda_stream, nullptr);
+}
+
+int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, float *ms_stats, float *ms_sample) {
+    if (!ms_stats || !ms_sample) return TLI_ERR_ARG;
+    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    cudaError_t e = cudaSuccess;
+    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaEventCreate(&ev[i]);
+    int rc = (e == cudaSuccess) ? verify_impl(ctx, a, cuda_stream, ev) : cuda_fail(e, "cudaEventCreate");
+    if (rc == TLI_OK) {
+        if ((e = cudaEventSynchronize(ev[2])) != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
+        else {
+            cudaEventElapsedTime(ms_stats, ev[0], ev[1]);
+            cudaEventElapsedTime(ms_sample, ev[1], ev[2]);
+        }
+    }
+    for (int i = 0; i < 3; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
+    return rc;
 }
 
 const char *tli_status_string(int code) {

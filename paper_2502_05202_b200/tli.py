@@ -34,7 +34,7 @@ TLI_MAX_B = 65535
 TLI_MAX_K = 64
 TLI_MAX_V = 1048576
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_ctx_info",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_profile", "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
 
@@ -78,6 +78,9 @@ def load() -> ctypes.CDLL:
         lib.tli_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_verify.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p]
         lib.tli_verify.restype = ctypes.c_int
+        lib.tli_verify_profile.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p,
+                                           ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+        lib.tli_verify_profile.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
         lib.tli_ctx_info.restype = ctypes.c_int
         lib.tli_status_string.argtypes = [ctypes.c_int]
@@ -156,6 +159,17 @@ def tli_verify(ctx: int, args: tli_verify_args, stream: Optional[int] = None) ->
     rc = load().tli_verify(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify")
+
+
+def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
+    """tli_verify_profile(): blocks; returns (ms of the statistics kernel, ms of the sampling kernel)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    a, b = ctypes.c_float(), ctypes.c_float()
+    rc = load().tli_verify_profile(ctx, ctypes.byref(args), ctypes.c_void_p(stream), ctypes.byref(a), ctypes.byref(b))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_verify_profile")
+    return a.value, b.value
 
 
 class Verifier:
