@@ -40,7 +40,8 @@ enum {
     TLI_ERR_BAD_MAP = -2,     /* id map entry out of range, or two drafter ids on one target id */
     TLI_ERR_CUDA = -3,        /* a CUDA runtime call failed (tli_last_cuda_error() says which) */
     TLI_ERR_WORKSPACE = -4,   /* workspace missing, misaligned or too small */
-    TLI_ERR_UNSUPPORTED = -5  /* size beyond TLI_MAX_B / TLI_MAX_K / TLI_MAX_V */
+    TLI_ERR_UNSUPPORTED = -5, /* size beyond TLI_MAX_B / TLI_MAX_K / TLI_MAX_V */
+    TLI_ERR_STATIC_SCRATCH = -6 /* tli_verify_static(): the batch needs more than TLI_STATIC_SCRATCH_BYTES */
 };
 
 /* row_status bits */
@@ -55,6 +56,7 @@ enum {
 #define TLI_MAX_B 65535    /* sequences per call */
 #define TLI_MAX_K 64       /* drafts per sequence */
 #define TLI_MAX_V 1048576  /* vocabulary size (either side) */
+#define TLI_STATIC_SCRATCH_BYTES 4194304 /* 4 MiB: scratch built into the library for tli_verify_static() */
 
 /*
  * Create a context for one (target vocabulary, drafter vocabulary) pair on one
@@ -145,6 +147,37 @@ typedef struct {
  * context's device must be current.
  */
 int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
+
+/*
+ * tli_verify() for callers that have no way to obtain device scratch.
+ * (The paper has no counterpart for this; it is a deployment convenience.)
+ *
+ * Some hosts of this library cannot allocate device memory at the moment they
+ * need a verification: an inference server that handed its whole HBM budget to
+ * the KV cache and weights at start-up, a decode loop where a cudaMalloc would
+ * stall the device, a plugin that is given tensors but no allocator.  For them
+ * this entry point does exactly what tli_verify() does, but ignores
+ * args->workspace / args->workspace_bytes and uses a fixed
+ * TLI_STATIC_SCRATCH_BYTES (4 MiB) array that is part of the library's device
+ * image.  Inputs and outputs are still the caller's.  It calls no cudaMalloc,
+ * cudaFree or other allocating routine.
+ *
+ * Cost and limits
+ *   - every GPU on which the library is loaded holds those 4 MiB until the
+ *     process exits, used or not;
+ *   - a batch whose scratch need (tli_workspace_bytes()) exceeds the array is
+ *     refused with TLI_ERR_STATIC_SCRATCH and nothing is launched; the five
+ *     benchmark workloads need at most about 1 MiB;
+ *   - the first call on each device looks up the array's device address (the
+ *     context's device must be current, as for tli_verify()).  Make that first
+ *     call outside any stream capture;
+ *   - all calls on one device share the one array.  Two calls that overlap on
+ *     the GPU (different streams, no ordering between them) corrupt each other;
+ *     order them on one stream or with events.  The array keeps whatever the
+ *     last call left in it; that is harmless, because each call writes every
+ *     word of it before reading that word, so nothing needs to be cleared.
+ */
+int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 
 /*
  * Measurement hook: the same work as tli_verify(), with CUDA events recorded on

@@ -28,6 +28,7 @@
 #include <stdint.h>
 #include <stdio.h>
 #include <string.h>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -912,6 +913,57 @@ int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     return rc;
 }
 
+// ---------------------------------------------------------------------------
+// tli_verify_static: the same verification with library-resident scratch
+// ---------------------------------------------------------------------------
+
+// Scratch for callers that cannot allocate.  It lives in the library's device image: every GPU
+// that loads the library carries these bytes until the process exits, whether or not it is used.
+static __device__ __align__(256) unsigned char g_static_scratch[TLI_STATIC_SCRATCH_BYTES];
+
+namespace {
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_ptr[kMaxDevices];       // device address of g_static_scratch, per device
+bool g_static_scratch_ready[kMaxDevices];
+std::mutex g_static_scratch_mutex;
+
+// In host code the name g_static_scratch is only a handle for the runtime, not an address a
+// kernel could use; the device address has to be asked for, once per device, with that device current.
+int static_scratch_address(int device, void **out) {
+    std::lock_guard<std::mutex> lock(g_static_scratch_mutex);
+    if (!g_static_scratch_ready[device]) {
+        void *ptr = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&ptr, g_static_scratch);
+        if (e != cudaSuccess) return cuda_fail(e, "cudaGetSymbolAddress(g_static_scratch)");
+        if (!ptr) return cuda_fail(cudaErrorInvalidSymbol, "cudaGetSymbolAddress(g_static_scratch)");
+        g_static_scratch_ptr[device] = ptr;
+        g_static_scratch_ready[device] = true;
+    }
+    *out = g_static_scratch_ptr[device];
+    return TLI_OK;
+}
+}  // namespace
+
+int tli_verify_static(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
+    if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype).total > TLI_STATIC_SCRATCH_BYTES)
+        return TLI_ERR_STATIC_SCRATCH;
+    int device = -1;
+    const cudaError_t e = cudaGetDevice(&device);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaGetDevice");
+    if (device != ctx->device || device < 0 || device >= kMaxDevices) return TLI_ERR_ARG;
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(device, &scratch);
+    if (rc != TLI_OK) return rc;
+    tli_verify_args b = *a;
+    b.workspace = scratch;
+    b.workspace_bytes = TLI_STATIC_SCRATCH_BYTES;
+    return verify_impl(ctx, &b, cuda_stream, nullptr);
+}
+
 const char *tli_status_string(int code) {
     switch (code) {
         case TLI_OK: return "ok";
@@ -920,6 +972,7 @@ const char *tli_status_string(int code) {
         case TLI_ERR_CUDA: return "CUDA runtime error";
         case TLI_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case TLI_ERR_UNSUPPORTED: return "size beyond the library's limits";
+        case TLI_ERR_STATIC_SCRATCH: return "batch needs more scratch than the built-in TLI_STATIC_SCRATCH_BYTES";
         default: return "unknown code";
     }
 }

@@ -25,6 +25,7 @@ TLI_ERR_BAD_MAP = -2
 TLI_ERR_CUDA = -3
 TLI_ERR_WORKSPACE = -4
 TLI_ERR_UNSUPPORTED = -5
+TLI_ERR_STATIC_SCRATCH = -6
 TLI_ROW_DRAFT_RANGE = 1
 TLI_ROW_DRAFT_UNMAPPED = 2
 TLI_ROW_NONFINITE = 4
@@ -33,8 +34,10 @@ TLI_ROW_BAD_TEMPERATURE = 32
 TLI_MAX_B = 65535
 TLI_MAX_K = 64
 TLI_MAX_V = 1048576
+TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_profile", "tli_ctx_info",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile",
+           "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
 
@@ -78,6 +81,8 @@ def load() -> ctypes.CDLL:
         lib.tli_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_verify.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p]
         lib.tli_verify.restype = ctypes.c_int
+        lib.tli_verify_static.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p]
+        lib.tli_verify_static.restype = ctypes.c_int
         lib.tli_verify_profile.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p,
                                            ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
         lib.tli_verify_profile.restype = ctypes.c_int
@@ -159,6 +164,19 @@ def tli_verify(ctx: int, args: tli_verify_args, stream: Optional[int] = None) ->
     rc = load().tli_verify(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify")
+
+
+def tli_verify_static(ctx: int, args: tli_verify_args, stream: Optional[int] = None) -> None:
+    """tli_verify_static(): like tli_verify() but on the library's built-in 4 MiB scratch.
+
+    For callers that cannot allocate device memory when they need to verify (all HBM already
+    committed, or an allocation would stall the device).  ``args.workspace`` is ignored.  Calls
+    that overlap on the GPU share the scratch and must be ordered by the caller."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_verify_static(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_verify_static")
 
 
 def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
