@@ -286,7 +286,12 @@ def gpu_arm(args):
         dist.init_process_group("nccl", device_id=device)
     peak, peak_kind = load_peaks()
     cfg = wl.config_by_name(args.config)
-    case = GpuCase(cfg, device, torch, tli, wl, want_host=True)
+    if args.batch:
+        import dataclasses
+        cfg = dataclasses.replace(cfg, B=args.batch)
+    if args.kernels_only:
+        args.no_per_config = True
+    case = GpuCase(cfg, device, torch, tli, wl, want_host=not args.kernels_only)
 
     for _ in range(max(args.warmup, 3)):
         case.step()
@@ -300,11 +305,14 @@ def gpu_arm(args):
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
-    for _ in range(2):
-        case.step_e2e()
-    ms_e2e = timed(torch, dist, max(3, min(args.steps, 10)), case.step_e2e, world)
     e2e_steps = max(3, min(args.steps, 10))
-    h2d, d2h = case.e2e_bytes()
+    if args.kernels_only:
+        ms_e2e, h2d, d2h = float("nan"), 0, 0
+    else:
+        for _ in range(2):
+            case.step_e2e()
+        ms_e2e = timed(torch, dist, e2e_steps, case.step_e2e, world)
+        h2d, d2h = case.e2e_bytes()
 
     ms_step = ms / args.steps
     value = world * cfg.positions / (ms_step * 1e-3)
@@ -354,7 +362,7 @@ def gpu_arm(args):
             torch.cuda.empty_cache()
         out["per_config"] = per
 
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.kernels_only:
         v, cores, reps, secs = time_oracle(headline_batch, cfg.positions)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                "sample": "all %d sequences of %s, %d repetitions in %.1f s" % (cfg.B, cfg.name, reps, secs)}
@@ -373,6 +381,9 @@ def main():
     ap.add_argument("--config", default="cfg3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-config", action="store_true", help="skip the four other workloads")
+    ap.add_argument("--batch", type=int, default=0, help="override the workload's B (profiling on a smaller case)")
+    ap.add_argument("--kernels-only", action="store_true",
+                    help="only the device-timed loop: no per-config, end-to-end or CPU legs (for profiler runs)")
     args = ap.parse_args()
     if args.impl == "reference":
         reference_arm(args)
