@@ -50,6 +50,7 @@ enum {
     TLI_ROW_DRAFT_UNMAPPED = 2,   /* a draft id outside the intersection: rejected (q' = 0 there) */
     TLI_ROW_NONFINITE = 4,        /* NaN or +inf logit seen: accepted = 0, next_token = 0 */
     TLI_ROW_FALLBACK = 8,         /* empty intersection or zero residual mass: sampled from p instead */
+    TLI_ROW_TIMEOUT = 16,         /* a bounded wait inside a kernel ran out (sticky for the context): results not to be trusted */
     TLI_ROW_BAD_TEMPERATURE = 32  /* temperature negative or not finite: accepted = 0, next_token = 0 */
 };
 

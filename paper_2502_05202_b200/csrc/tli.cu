@@ -3,7 +3,8 @@
 // Two launches per call, both streaming and HBM-bound (no dense contraction,
 // hence no tensor cores):
 //
-//   tli_stats_kernel   one CTA per 16 KB chunk of a logit row.  Target rows:
+//   tli_stats_kernel   persistent grid (two CTAs per SM); each CTA streams 16 KB chunks of
+//                      logit rows through a cp.async.bulk / mbarrier ring.  Target rows:
 //                      (reference, sum of 2^(z*s - reference)) with s = log2(e)/tau;
 //                      drafter rows: the same over ids inside the intersection
 //                      only (Algorithm 4's renormalisation: the full-softmax
@@ -41,6 +42,11 @@ constexpr int kWarps = kThreads / 32;
 constexpr int kVecPerThread = 4;
 constexpr int kVecPerChunk = kThreads * kVecPerThread;      // 1024 16-byte vectors
 constexpr int kChunkBytes = kVecPerChunk * 16;              // 16 KB
+constexpr int kStages = 6;                                  // 16 KB stages in the shared-memory ring
+constexpr int kCtasPerSm = 2;                               // persistent CTAs of the statistics kernel per SM
+constexpr int kSWarps = 16;                                 // consumer warps of the statistics kernel
+constexpr int kSThreads = kSWarps * 32;
+constexpr int kSVec = kVecPerChunk / kSThreads;             // 16-byte vectors per consumer thread per chunk
 constexpr int kMaxTiles = (TLI_MAX_V * 4 + 15) / kChunkBytes + 2;
 constexpr float kNegBig = -FLT_MAX;
 
@@ -66,7 +72,11 @@ struct Params {
     int *accepted; int *next_token; int *status; float *p_out; float *q_out;
     float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
     unsigned *cnt_stats; unsigned *cnt_sample;
-    int nct, ncd;
+    unsigned *error;     // sticky: set when a bounded wait ran out
+    unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
+    int nct, ncd;        // 16 KB chunks per target / drafter row
+    int cps;             // chunks per segment
+    int nst, nsd;        // segments per target / drafter row
 };
 
 // ---------------------------------------------------------------------------
@@ -183,143 +193,158 @@ __device__ __forceinline__ uint32_t mask_bits(const uint32_t *maskbits, int e0) 
     return __funnelshift_r(lo, hi, e0 & 31);
 }
 
-// (reference, sum) pairs: value = sum * 2^reference.
+// 2^d for an integer-valued d <= 0, exactly (0 below the normal range).
+__device__ __forceinline__ float pow2_neg(float d) {
+    return (d >= -126.f) ? __int_as_float((static_cast<int>(d) + 127) << 23) : 0.f;
+}
+__device__ __forceinline__ double pow2_neg_d(float d) {
+    return (d >= -1022.f) ? __hiloint2double((static_cast<int>(d) + 1023) << 20, 0) : 0.0;
+}
+// A softmax reference for values up to m*s: the next integer above, so that every later
+// change of reference is an exact power of two.  Nothing to refer to (-inf) gives kNegBig.
+__device__ __forceinline__ float reference_for(float ms) { return fmaxf(ceilf(ms), kNegBig); }
+
+// (reference, sum) pairs: value = sum * 2^reference, references integer valued.
 __device__ __forceinline__ void combine_pair(float &c, float &s, float c2, float s2) {
     const float cn = fmaxf(c, c2);
-    s = s * ex2(c - cn) + s2 * ex2(c2 - cn);
+    s = s * pow2_neg(c - cn) + s2 * pow2_neg(c2 - cn);
     c = cn;
 }
 
 // ---------------------------------------------------------------------------
-// pass 1: per-chunk statistics
+// pass 1: statistics of every row, persistent and pipelined
 // ---------------------------------------------------------------------------
+//
+// Work unit: a segment = up to `cps` consecutive 16 KB chunks of one logit row.  Segments are
+// numbered sequence-major and dealt round-robin to a fixed grid of CTAs.  In each CTA one thread
+// (the producer) streams the chunks into a ring of shared-memory stages with cp.async.bulk,
+// completion counted on an mbarrier per stage; eight consumer warps reduce a stage from shared
+// memory and hand it back through a second mbarrier as soon as its bytes are in registers.
 
-// softmax statistics of one chunk; MASKED restricts to drafter ids inside the intersection
-template <int DT, bool MASKED>
-__device__ __forceinline__ float2 chunk_softmax_stats(const RowView<DT> &rv, int chunk, float s,
-                                                      const uint32_t *maskbits, float2 *sm_pairs) {
-    constexpr int EPV = Elt<DT>::kPerVec;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nvec = rv.nvec();
-    uint4 raw[kVecPerThread];
-    uint32_t bits[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = chunk * kVecPerChunk + k * kThreads + tid;
-        if (v < nvec) {
-            raw[k] = rv.load(v);
-            bits[k] = MASKED ? mask_bits(maskbits, rv.first_elem(v)) : 0xffffffffu;
-        } else {
-            raw[k] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
-            bits[k] = 0;
-        }
+// ---- mbarrier and bulk-copy primitives ----
+
+__device__ __forceinline__ uint32_t smem_addr(const void *p) {
+    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, unsigned count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, unsigned bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_test(uint64_t *bar, unsigned parity) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kWaitLimit polls, records the fact and lets the caller go on
+// (results of that call are then flagged, never trusted).  Returns false on timeout.
+constexpr unsigned kWaitLimit = 1u << 22;
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, unsigned parity, int *sm_error, unsigned *g_error) {
+    if (*reinterpret_cast<volatile int *>(sm_error)) return false;
+    for (unsigned i = 0; i < kWaitLimit; ++i) {
+        if (mbar_test(bar, parity)) return true;
+        if (i > 64) __nanosleep(64);
     }
-    float z[kVecPerThread][EPV];
-    float m = -INFINITY;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        unpack<DT>(raw[k], z[k]);
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-            if (MASKED) z[k][i] = ((bits[k] >> i) & 1u) ? z[k][i] : -INFINITY;
-            m = fmaxf(m, z[k][i]);
-        }
-    }
-    m = warp_max(m);
-    const float c = fmaxf(m * s, kNegBig);      // -inf (nothing here) -> most negative finite reference
-    const float nc = -c;
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) acc[i & 3] += ex2(fmaf(z[k][i], s, nc));
-    }
-    float sum = warp_sum((acc[0] + acc[1]) + (acc[2] + acc[3]));
-    if (lane == 0) sm_pairs[warp] = make_float2(c, sum);
-    __syncthreads();
-    float2 out = make_float2(kNegBig, 0.f);
-    if (warp == 0) {
-        float2 pr = (lane < kWarps) ? sm_pairs[lane] : make_float2(kNegBig, 0.f);
-#pragma unroll
-        for (int o = kWarps / 2; o > 0; o >>= 1) {
-            float c2 = __shfl_xor_sync(0xffffffffu, pr.x, o);
-            float s2 = __shfl_xor_sync(0xffffffffu, pr.y, o);
-            combine_pair(pr.x, pr.y, c2, s2);
-        }
-        out = pr;
-    }
-    return out;      // valid in warp 0
+    *reinterpret_cast<volatile int *>(sm_error) = 1;
+    atomicOr(g_error, 1u);
+    return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity, int *sm_error, unsigned *g_error) {
+    if (mbar_test(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, sm_error, g_error);
+}
+__device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes, uint64_t *bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+__device__ __forceinline__ void consumer_sync() {            // the eight consumer warps only
+    asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory");
 }
 
-// (max, lowest index attaining it) of one chunk, as (value, index bits)
-template <int DT>
-__device__ __forceinline__ float2 chunk_argmax(const RowView<DT> &rv, int chunk, float2 *sm_pairs) {
-    constexpr int EPV = Elt<DT>::kPerVec;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int nvec = rv.nvec();
-    uint4 raw[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = chunk * kVecPerChunk + k * kThreads + tid;
-        raw[k] = (v < nvec) ? rv.load(v)
-                            : make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+// ---- the schedule both the producer and the consumers walk ----
+
+struct Segment {
+    int b;            // sequence
+    int row;          // 0..K target rows, K+1..2K drafter rows
+    int chunk0, chunk1;
+    int seg;          // index of the segment within its row
+    bool skip;        // nothing to read (bad temperature, or drafter row at temperature 0)
+    float tau;
+};
+
+__device__ __forceinline__ Segment decode_segment(const Params &P, long long id) {
+    Segment g;
+    const int per_b = (P.K + 1) * P.nst + P.K * P.nsd;
+    g.b = static_cast<int>(id / per_b);
+    int item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
+    g.tau = __ldg(P.tau + g.b);
+    const bool bad = !(g.tau >= 0.f) || isinf(g.tau);
+    int nchunk;
+    if (item < (P.K + 1) * P.nst) {
+        g.row = item / P.nst; g.seg = item - g.row * P.nst; nchunk = P.nct;
+        g.skip = bad;
+    } else {
+        item -= (P.K + 1) * P.nst;
+        const int j = item / P.nsd;
+        g.row = P.K + 1 + j; g.seg = item - j * P.nsd; nchunk = P.ncd;
+        g.skip = bad || g.tau == 0.f;
     }
-    float best = -INFINITY;
-    int idx = INT_MAX;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {      // increasing index order, strict > keeps the lowest
-        float z[EPV];
-        unpack<DT>(raw[k], z);
-        const int e0 = rv.first_elem(chunk * kVecPerChunk + k * kThreads + tid);
-#pragma unroll
-        for (int i = 0; i < EPV; ++i)
-            if (z[i] > best) { best = z[i]; idx = e0 + i; }
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        float b2 = __shfl_xor_sync(0xffffffffu, best, o);
-        int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
-        if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
-    }
-    if (lane == 0) sm_pairs[warp] = make_float2(best, __int_as_float(idx));
-    __syncthreads();
-    float2 out = make_float2(-INFINITY, __int_as_float(INT_MAX));
-    if (warp == 0) {
-        float2 pr = (lane < kWarps) ? sm_pairs[lane] : out;
-        best = pr.x; idx = __float_as_int(pr.y);
-#pragma unroll
-        for (int o = kWarps / 2; o > 0; o >>= 1) {
-            float b2 = __shfl_xor_sync(0xffffffffu, best, o);
-            int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
-            if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
-        }
-        out = make_float2(best, __int_as_float(idx));
-    }
-    return out;
+    g.chunk0 = g.seg * P.cps;
+    g.chunk1 = min(g.chunk0 + P.cps, nchunk);
+    return g;
 }
 
-// Last CTA of a sequence: fp64 combination of the chunk partials, Algorithm 5's
-// acceptance tests and count, hand-over to the sampling pass.
+template <int DT> __device__ __forceinline__ RowView<DT> segment_row(const Params &P, const Segment &g) {
+    if (g.row <= P.K)
+        return RowView<DT>(P.zt, static_cast<long long>(g.b) * P.t_sb + static_cast<long long>(g.row) * P.t_sk, P.V_t);
+    return RowView<DT>(P.zd, static_cast<long long>(g.b) * P.d_sb + static_cast<long long>(g.row - P.K - 1) * P.d_sk, P.V_d);
+}
+
+// Vectors of chunk `chunk` that lie wholly inside the row: [v0, v1).  Only these are bulk-copied;
+// the (at most two) ragged vectors of a row are read element by element by the consumers.
+template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT> &rv, int chunk, int &v0, int &v1) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int first_full = rv.head ? 1 : 0;
+    const int end_full = (rv.V + rv.head) / EPV;               // vectors [first_full, end_full) are whole
+    v0 = max(chunk * kVecPerChunk, first_full);
+    v1 = min((chunk + 1) * kVecPerChunk, end_full);
+    if (v1 < v0) v1 = v0;
+}
+
+// Last CTA of a sequence: fp64 combination of the segment partials, Algorithm 5's
+// acceptance tests and count, hand-over to the sampling pass.  Run by the consumer warps.
 template <int DT>
-__device__ void finalize_sequence(const Params &P, int b, float tau) {
+__device__ void finalize_sequence(const Params &P, int b, float tau, int tid) {
     __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
     __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
     __shared__ int sm_accept[TLI_MAX_K];
     __shared__ int sm_flags;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int lane = tid & 31, warp = tid >> 5;
     const int K = P.K;
     const bool greedy = (tau == 0.f);
     const int nrows = greedy ? (K + 1) : (2 * K + 1);
-    if (tid == 0) sm_flags = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+    if (tid == 0) {
+        int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+        if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
+        sm_flags = fl;
+    }
 
-    for (int r = warp; r < nrows; r += kWarps) {
+    for (int r = warp; r < nrows; r += kSWarps) {
         const bool is_t = r <= K;
-        const int nchunk = is_t ? P.nct : P.ncd;
-        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nct
-                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.ncd;
+        const int nseg = is_t ? P.nst : P.nsd;
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
         if (greedy) {
             float best = -INFINITY; int idx = INT_MAX;
-            for (int i = lane; i < nchunk; i += 32) {
+            for (int i = lane; i < nseg; i += 32) {
                 float2 pr = __ldcg(part + i);
                 int i2 = __float_as_int(pr.y);
                 if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
@@ -333,18 +358,18 @@ __device__ void finalize_sequence(const Params &P, int b, float tau) {
             if (lane == 0) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
         } else {
             float c = kNegBig;
-            for (int i = lane; i < nchunk; i += 32) c = fmaxf(c, __ldcg(part + i).x);
+            for (int i = lane; i < nseg; i += 32) c = fmaxf(c, __ldcg(part + i).x);
             c = warp_max(c);
             double s = 0.0;
-            for (int i = lane; i < nchunk; i += 32) {
+            for (int i = lane; i < nseg; i += 32) {
                 float2 pr = __ldcg(part + i);
-                s += static_cast<double>(pr.y) * exp2(static_cast<double>(pr.x) - static_cast<double>(c));
+                s += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
             }
             s = warp_sum(s);
             if (lane == 0) { sm_c[r] = c; sm_s[r] = s; }
         }
     }
-    __syncthreads();
+    consumer_sync();
 
     const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
     if (tid < K) {
@@ -383,7 +408,7 @@ __device__ void finalize_sequence(const Params &P, int b, float tau) {
         const double S_t = sm_s[K];
         if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
     }
-    __syncthreads();
+    consumer_sync();
     if (tid == 0) {
         int n = K;
         for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
@@ -414,60 +439,315 @@ __device__ void finalize_sequence(const Params &P, int b, float tau) {
         P.sel[b] = sel;
         P.cnt_stats[b] = 0;        // leave the ticket counter ready for the next call
     }
+    consumer_sync();               // the shared arrays above are reused by the next sequence this CTA finishes
+}
+
+// What the producer tells the consumers about the chunk it put into a stage.
+struct StageMeta {
+    long long id;     // segment
+    int chunk;        // chunk of the segment's row held by this stage
+    int flags;        // META_*
+};
+enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_NOTICE = 8 };
+
+struct StatsSmem {
+    uint64_t full[kStages];
+    uint64_t empty[kStages];
+    StageMeta meta[kStages];
+    float2 pairs[kSWarps];
+    int last;
+    int error;
+};
+
+constexpr int kStatsSmemBytes = kStages * kChunkBytes + static_cast<int>(sizeof(StatsSmem));
+
+// This thread's vectors of one chunk.  Chunks that lie wholly inside the row (all but the first
+// and last of a row) come straight from the stage; the others check every vector.
+template <int DT>
+__device__ __forceinline__ void load_chunk(const RowView<DT> &rv, int chunk, const uint4 *stage, int tid,
+                                           uint4 (&raw)[kSVec]) {
+    int v0, v1;
+    full_vectors<DT>(rv, chunk, v0, v1);
+    if (v0 == chunk * kVecPerChunk && v1 == (chunk + 1) * kVecPerChunk) {
+#pragma unroll
+        for (int q = 0; q < kSVec; ++q) raw[q] = stage[q * kSThreads + tid];
+    } else {
+        const int nvec = rv.nvec();
+#pragma unroll
+        for (int q = 0; q < kSVec; ++q) {
+            const int g_in = q * kSThreads + tid;
+            const int v = chunk * kVecPerChunk + g_in;
+            if (v >= v0 && v < v1) raw[q] = stage[g_in];
+            else if (v < nvec) raw[q] = rv.load(v);                      // ragged end of the row
+            else raw[q] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+        }
+    }
+}
+
+__device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
+    uint32_t d;
+    asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// One chunk of a softmax row into this thread's running (reference, sum).
+template <int DT, bool MASKED>
+__device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[kSVec], const uint32_t (&bits)[kSVec], float s,
+                                              float &c_run, float &acc) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    float z[kSVec][EPV];
+    float m;
+    if (DT == TLI_BF16 && !MASKED) {
+        uint32_t mm = bf16x2_max(bf16x2_max(raw[0].x, raw[0].y), bf16x2_max(raw[0].z, raw[0].w));
+#pragma unroll
+        for (int q = 1; q < kSVec; ++q)
+            mm = bf16x2_max(mm, bf16x2_max(bf16x2_max(raw[q].x, raw[q].y), bf16x2_max(raw[q].z, raw[q].w)));
+        m = fmaxf(bf16_lo(mm), bf16_hi(mm));
+#pragma unroll
+        for (int q = 0; q < kSVec; ++q) unpack<DT>(raw[q], z[q]);
+    } else {
+        m = -INFINITY;
+#pragma unroll
+        for (int q = 0; q < kSVec; ++q) {
+            unpack<DT>(raw[q], z[q]);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                if (MASKED) z[q][i] = ((bits[q] >> i) & 1u) ? z[q][i] : -INFINITY;
+                m = fmaxf(m, z[q][i]);
+            }
+        }
+    }
+    // raise the reference if this chunk tops it; the sum follows by an exact power of two
+    const float c_new = fmaxf(c_run, reference_for(m * s));
+    acc *= pow2_neg(c_run - c_new);
+    c_run = c_new;
+    const float nc = -c_run;
+    float a4[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int q = 0; q < kSVec; ++q) {
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) a4[i & 3] += ex2(fmaf(z[q][i], s, nc));
+    }
+    acc += (a4[0] + a4[1]) + (a4[2] + a4[3]);
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kThreads) tli_stats_kernel(const Params P) {
-    __shared__ float2 sm_pairs[kWarps];
-    __shared__ int sm_last;
+__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[kSVec], const RowView<DT> &rv, int chunk, int tid,
+                                             float &best, int &best_idx) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+#pragma unroll
+    for (int q = 0; q < kSVec; ++q) {                     // increasing index order, strict > keeps the lowest
+        float z[EPV];
+        unpack<DT>(raw[q], z);
+        const int e0 = rv.first_elem(chunk * kVecPerChunk + q * kSThreads + tid);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i)
+            if (z[i] > best) { best = z[i]; best_idx = e0 + i; }
+    }
+}
+
+// Segments are handed out by an atomic counter: a CTA that is busy closing a sequence simply takes
+// fewer of them.  The producer thread fetches the next segment number while it is still loading the
+// current one, streams the chunks through the stage ring and labels every stage for the consumers.
+template <int DT>
+__global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(const Params P) {
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw);                       // kStages * 16 KB
+    StatsSmem &sm = *reinterpret_cast<StatsSmem *>(smem_raw + static_cast<size_t>(kStages) * kChunkBytes);
     asm volatile("griddepcontrol.launch_dependents;");
-    const int b = blockIdx.y;
-    const int item = blockIdx.x;
-    const int K = P.K;
-    const float tau = __ldg(P.tau + b);
-    if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
-        if (item == 0 && threadIdx.x == 0) {
-            P.accepted[b] = 0; P.next_token[b] = 0;
-            if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
-            RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            P.sel[b] = sel;
-        }
-        if (item == 0 && threadIdx.x < K) {
-            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + threadIdx.x] = 0.f;
-            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + threadIdx.x] = 0.f;
-        }
-        return;
-    }
-    const bool greedy = (tau == 0.f);
-    const int n_target_items = (K + 1) * P.nct;
-    const float s = 1.4426950408889634f / tau;
-    float2 partial;
-    float2 *dst;
-    if (item < n_target_items) {
-        const int j = item / P.nct, chunk = item - j * P.nct;
-        RowView<DT> rv(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk, P.V_t);
-        partial = greedy ? chunk_argmax<DT>(rv, chunk, sm_pairs)
-                         : chunk_softmax_stats<DT, false>(rv, chunk, s, nullptr, sm_pairs);
-        dst = P.part_t + (static_cast<size_t>(b) * (K + 1) + j) * P.nct + chunk;
-    } else {
-        if (greedy) return;                        // drafter logits are not read at temperature 0
-        const int it = item - n_target_items;
-        const int j = it / P.ncd, chunk = it - j * P.ncd;
-        RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk, P.V_d);
-        partial = chunk_softmax_stats<DT, true>(rv, chunk, s, P.maskbits, sm_pairs);
-        dst = P.part_d + (static_cast<size_t>(b) * K + j) * P.ncd + chunk;
-    }
     if (threadIdx.x == 0) {
-        __stcg(dst, partial);
-        __threadfence();
-        const unsigned total = greedy ? n_target_items : n_target_items + K * P.ncd;
-        const unsigned ticket = atomicAdd(P.cnt_stats + b, 1u);
-        sm_last = (ticket == total - 1);
+#pragma unroll
+        for (int i = 0; i < kStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
+        sm.error = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    if (sm_last) {
-        __threadfence();
-        finalize_sequence<DT>(P, b, tau);
+    const long long nseg_total = static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
+
+    if (threadIdx.x < 32) {
+        // ---------------- producer ----------------
+        if (threadIdx.x == 0) {
+            unsigned it = 0;
+            bool ok = true;
+            long long next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));
+            while (ok) {
+                const long long id = next;
+                if (id >= nseg_total) break;
+                next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));     // used one segment later
+                const Segment g = decode_segment(P, id);
+                if (g.skip) {
+                    // a bad temperature is answered once per sequence, by the consumers of whoever meets its first segment
+                    if (g.row == 0 && g.seg == 0) {
+                        const unsigned st = it % kStages, k = it / kStages;
+                        ok = mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error);
+                        if (!ok) break;
+                        sm.meta[st].id = id; sm.meta[st].chunk = 0; sm.meta[st].flags = META_NOTICE;
+                        mbar_arrive(&sm.full[st]);
+                        ++it;
+                    }
+                    continue;
+                }
+                const RowView<DT> rv = segment_row<DT>(P, g);
+                for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk, ++it) {
+                    const unsigned st = it % kStages, k = it / kStages;
+                    ok = mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error);
+                    if (!ok) break;
+                    sm.meta[st].id = id; sm.meta[st].chunk = chunk;
+                    sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0);
+                    int v0, v1;
+                    full_vectors<DT>(rv, chunk, v0, v1);
+                    const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
+                    mbar_arrive_expect_tx(&sm.full[st], bytes);
+                    if (bytes)
+                        bulk_load(stage_base + static_cast<size_t>(st) * kVecPerChunk + (v0 - chunk * kVecPerChunk),
+                                  rv.vec0 + v0, bytes, &sm.full[st]);
+                }
+            }
+            if (ok) {                                    // tell the consumers there is nothing more
+                const unsigned st = it % kStages, k = it / kStages;
+                if (mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error)) {
+                    sm.meta[st].id = -1; sm.meta[st].chunk = 0; sm.meta[st].flags = META_END;
+                    mbar_arrive(&sm.full[st]);
+                    ++it;
+                }
+            }
+            // After a timeout nobody may be waiting for the copies still in flight: let them land
+            // (bounded) before this CTA's shared memory goes away.
+            if (*reinterpret_cast<volatile int *>(&sm.error)) {
+                const unsigned lo = it > kStages ? it - kStages : 0;
+                for (unsigned j = lo; j < it; ++j) {
+                    const unsigned st = j % kStages, k = j / kStages;
+                    for (unsigned i = 0; i < kWaitLimit && !mbar_test(&sm.full[st], k & 1u); ++i) __nanosleep(64);
+                }
+            }
+        }
+    } else {
+        // ---------------- consumers ----------------
+        constexpr int EPV = Elt<DT>::kPerVec;
+        const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
+        Segment g;
+        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f;
+        RowView<DT> rv(P.zt, 0, P.V_t);
+        bool greedy = false, masked = false;
+        float s = 0.f;
+        float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
+        float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
+        bool clean_exit = false;
+        for (unsigned it = 0;; ++it) {
+            const unsigned st = it % kStages, k = it / kStages;
+            if (!mbar_wait(&sm.full[st], k & 1u, &sm.error, P.error)) break;
+            const StageMeta meta = sm.meta[st];
+            if (meta.flags & META_END) { clean_exit = true; break; }
+            if (meta.flags & (META_FIRST | META_NOTICE)) {
+                g = decode_segment(P, meta.id);
+                rv = segment_row<DT>(P, g);
+                greedy = (g.tau == 0.f);
+                masked = g.row > P.K;
+                s = 1.4426950408889634f / g.tau;
+                c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
+            }
+            if (meta.flags & META_NOTICE) {
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&sm.empty[st]);
+                if (tid == 0) {
+                    P.accepted[g.b] = 0; P.next_token[g.b] = 0;
+                    if (P.status) P.status[g.b] = TLI_ROW_BAD_TEMPERATURE;
+                    RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    P.sel[g.b] = sel;
+                }
+                if (tid < P.K) {
+                    if (P.p_out) P.p_out[static_cast<size_t>(g.b) * P.K + tid] = 0.f;
+                    if (P.q_out) P.q_out[static_cast<size_t>(g.b) * P.K + tid] = 0.f;
+                }
+                continue;
+            }
+            const int chunk = meta.chunk;
+            uint4 raw[kSVec];
+            load_chunk<DT>(rv, chunk, stage_base + static_cast<size_t>(st) * kVecPerChunk, tid, raw);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&sm.empty[st]);                        // stage may be refilled now
+            if (greedy) {
+                argmax_chunk<DT>(raw, rv, chunk, tid, best, best_idx);
+            } else if (masked) {
+                uint32_t bits[kSVec];
+                const int nvec = rv.nvec();
+#pragma unroll
+                for (int q = 0; q < kSVec; ++q) {
+                    const int v = chunk * kVecPerChunk + q * kSThreads + tid;
+                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
+                }
+                softmax_chunk<DT, true>(raw, bits, s, c_run, acc);
+            } else {
+                const uint32_t bits[kSVec] = {};
+                softmax_chunk<DT, false>(raw, bits, s, c_run, acc);
+            }
+            if (!(meta.flags & META_LAST)) continue;
+
+            // ---- segment done: one (reference, sum) or (max, index) pair per warp, then per CTA ----
+            float px, py;
+            if (greedy) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+                    int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
+                    if (b2 > best || (b2 == best && i2 < best_idx)) { best = b2; best_idx = i2; }
+                }
+                px = best; py = __int_as_float(best_idx);
+            } else {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    float c2 = __shfl_xor_sync(0xffffffffu, c_run, o);
+                    float a2 = __shfl_xor_sync(0xffffffffu, acc, o);
+                    combine_pair(c_run, acc, c2, a2);
+                }
+                px = c_run; py = acc;
+            }
+            if (lane == 0) sm.pairs[warp] = make_float2(px, py);
+            consumer_sync();
+            if (warp == 0) {
+                float2 pr;
+                if (greedy) {
+                    pr = (lane < kSWarps) ? sm.pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
+                    float bb = pr.x; int ii = __float_as_int(pr.y);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        float b2 = __shfl_xor_sync(0xffffffffu, bb, o);
+                        int i2 = __shfl_xor_sync(0xffffffffu, ii, o);
+                        if (b2 > bb || (b2 == bb && i2 < ii)) { bb = b2; ii = i2; }
+                    }
+                    pr = make_float2(bb, __int_as_float(ii));
+                } else {
+                    pr = (lane < kSWarps) ? sm.pairs[lane] : make_float2(kNegBig, 0.f);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        float c2 = __shfl_xor_sync(0xffffffffu, pr.x, o);
+                        float s2 = __shfl_xor_sync(0xffffffffu, pr.y, o);
+                        combine_pair(pr.x, pr.y, c2, s2);
+                    }
+                }
+                if (lane == 0) {
+                    float2 *dst = (g.row <= P.K)
+                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
+                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
+                    __stcg(dst, pr);
+                    __threadfence();
+                    const unsigned total = greedy ? (P.K + 1) * P.nst : (P.K + 1) * P.nst + P.K * P.nsd;
+                    const unsigned ticket = atomicAdd(P.cnt_stats + g.b, 1u);
+                    sm.last = (ticket == total - 1);
+                }
+            }
+            consumer_sync();
+            if (sm.last) {
+                __threadfence();
+                finalize_sequence<DT>(P, g.b, g.tau, tid);
+            }
+        }
+        // the last CTA to leave puts the segment counter back for the next call
+        if (clean_exit && tid == 0) {
+            __threadfence();
+            const unsigned t = atomicAdd(P.cta_done, 1u);
+            if (t == gridDim.x - 1) { *P.seg_counter = 0u; *P.cta_done = 0u; __threadfence(); }
+        }
     }
 }
 
@@ -730,16 +1010,28 @@ int chunks_per_row(int V, int dtype) {
 
 struct Layout {
     size_t part_t, part_d, sel, tilesum, total;
-    int nct, ncd;
+    int nct, ncd, cps, nst, nsd;
+    unsigned grid;
 };
 
-Layout make_layout(int B, int K, int V_t, int V_d, int dtype) {
+// Segments are sized so that every CTA of the persistent grid (two per SM) gets about eight of
+// them: long enough to amortise the per-segment reduction, short enough to balance the tail.
+Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     Layout L;
     L.nct = chunks_per_row(V_t, dtype);
     L.ncd = chunks_per_row(V_d, dtype);
+    const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
+    const long long ctas = static_cast<long long>(kCtasPerSm) * num_sms;
+    long long cps = chunks / (ctas * 8);
+    L.cps = static_cast<int>(cps < 1 ? 1 : (cps > 16 ? 16 : cps));
+    L.nst = (L.nct + L.cps - 1) / L.cps;
+    L.nsd = (L.ncd + L.cps - 1) / L.cps;
+    const long long nseg = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nst + static_cast<long long>(K) * L.nsd);
+    const long long grid = nseg < ctas ? nseg : ctas;
+    L.grid = static_cast<unsigned>(grid);
     size_t off = 0;
-    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nct, 256);
-    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.ncd, 256);
+    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nst, 256);
+    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.nsd, 256);
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
     L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.nct, 256);
     L.total = off;
@@ -754,7 +1046,8 @@ struct tli_ctx {
     int *d_map;
     int *d_inv;
     uint32_t *d_mask;
-    unsigned *d_counters;       // [2 * (TLI_MAX_B + 1)], zero between calls
+    unsigned *d_counters;       // [2 * (TLI_MAX_B + 1) + 3], zero between calls; last words: sticky error, scheduler
+    int num_sms;
 };
 
 extern "C" {
@@ -787,16 +1080,21 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     if (!c) { cudaSetDevice(prev); return TLI_ERR_ARG; }
     c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
+    c->num_sms = 0;
     int rc = TLI_OK;
     do {
+        if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }
+        // the statistics kernel needs more dynamic shared memory than the default limit
+        if ((e = cudaFuncSetAttribute(tli_stats_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes)) != cudaSuccess ||
+            (e = cudaFuncSetAttribute(tli_stats_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes)) != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
-        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * 2 * (TLI_MAX_B + 1))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (2 * (TLI_MAX_B + 1) + 3))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
         if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
         if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
         if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
-        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * 2 * (TLI_MAX_B + 1))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
+        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (2 * (TLI_MAX_B + 1) + 3))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
     } while (0);
     if (rc != TLI_OK) {
         cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
@@ -823,7 +1121,7 @@ int tli_destroy(tli_ctx *ctx) {
 size_t tli_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype) {
     if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return 0;
     if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
-    return make_layout(B, K, ctx->V_t, ctx->V_d, dtype).total;
+    return make_layout(B, K, ctx->V_t, ctx->V_d, dtype, ctx->num_sms).total;
 }
 
 int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped) {
@@ -846,7 +1144,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
         return TLI_ERR_ARG;
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
-    const Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype);
+    const Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
         return TLI_ERR_WORKSPACE;
 
@@ -865,14 +1163,15 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
     P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
-    P.nct = L.nct; P.ncd = L.ncd;
+    P.error = ctx->d_counters + 2 * (TLI_MAX_B + 1);
+    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
+    P.nct = L.nct; P.ncd = L.ncd; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
-    const dim3 grid1(static_cast<unsigned>((a->K + 1) * L.nct + a->K * L.ncd), static_cast<unsigned>(a->B));
     const dim3 grid2(static_cast<unsigned>(L.nct), static_cast<unsigned>(a->B));
-    if (a->dtype == TLI_F32) tli_stats_kernel<TLI_F32><<<grid1, kThreads, 0, stream>>>(P);
-    else tli_stats_kernel<TLI_BF16><<<grid1, kThreads, 0, stream>>>(P);
+    if (a->dtype == TLI_F32) tli_stats_kernel<TLI_F32><<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(P);
+    else tli_stats_kernel<TLI_BF16><<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(P);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
@@ -949,7 +1248,7 @@ int tli_verify_static(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream)
     if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
     if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
     if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
-    if (make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype).total > TLI_STATIC_SCRATCH_BYTES)
+    if (make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms).total > TLI_STATIC_SCRATCH_BYTES)
         return TLI_ERR_STATIC_SCRATCH;
     int device = -1;
     const cudaError_t e = cudaGetDevice(&device);

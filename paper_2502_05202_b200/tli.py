@@ -30,6 +30,7 @@ TLI_ROW_DRAFT_RANGE = 1
 TLI_ROW_DRAFT_UNMAPPED = 2
 TLI_ROW_NONFINITE = 4
 TLI_ROW_FALLBACK = 8
+TLI_ROW_TIMEOUT = 16
 TLI_ROW_BAD_TEMPERATURE = 32
 TLI_MAX_B = 65535
 TLI_MAX_K = 64

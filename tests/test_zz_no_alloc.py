@@ -68,8 +68,8 @@ def test_static_scratch_refuses_batches_beyond_its_size():
     args = tli.make_args(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"], dev["temperature"],
                          dev["uniforms"], out["accepted"], out["next_token"],
                          torch.empty(0, dtype=torch.uint8, device="cuda"))
-    args.B = 4000                                   # 4000 sequences of this vocabulary need ~7 MiB of scratch
-    assert tli.tli_workspace_bytes(v.ctx, 4000, 1, tli.TLI_F32) > tli.TLI_STATIC_SCRATCH_BYTES
+    args.B = 20000                                  # that many sequences of this vocabulary need ~14 MiB of scratch
+    assert tli.tli_workspace_bytes(v.ctx, 20000, 1, tli.TLI_F32) > tli.TLI_STATIC_SCRATCH_BYTES
     rc = tli.load().tli_verify_static(v.ctx, ctypes.byref(args), None)
     assert rc == tli.TLI_ERR_STATIC_SCRATCH
     assert b"TLI_STATIC_SCRATCH_BYTES" in tli.load().tli_status_string(rc)
