@@ -40,14 +40,14 @@ namespace {
 constexpr int kThreads = 256;
 constexpr int kWarps = kThreads / 32;
 constexpr int kVecPerThread = 4;
-constexpr int kVecPerChunk = kThreads * kVecPerThread;      // 1024 16-byte vectors
-constexpr int kChunkBytes = kVecPerChunk * 16;              // 16 KB
-constexpr int kStages = 6;                                  // 16 KB stages in the shared-memory ring
+constexpr int kVecPerTile = kThreads * kVecPerThread;       // sampling pass: 1024 16-byte vectors per tile
+constexpr int kTileBytes = kVecPerTile * 16;                // 16 KB
+constexpr int kRingBytes = 96 * 1024;                       // shared-memory stage ring of the statistics kernel
+constexpr int kMaxStages = 12;
 constexpr int kCtasPerSm = 2;                               // persistent CTAs of the statistics kernel per SM
 constexpr int kSWarps = 16;                                 // consumer warps of the statistics kernel
 constexpr int kSThreads = kSWarps * 32;
-constexpr int kSVec = kVecPerChunk / kSThreads;             // 16-byte vectors per consumer thread per chunk
-constexpr int kMaxTiles = (TLI_MAX_V * 4 + 15) / kChunkBytes + 2;
+constexpr int kMaxTiles = (TLI_MAX_V * 4 + 15) / kTileBytes + 2;
 constexpr float kNegBig = -FLT_MAX;
 
 enum : int { MODE_SKIP = 0, MODE_RESIDUAL = 1, MODE_TARGET_ONLY = 2 };
@@ -74,7 +74,8 @@ struct Params {
     unsigned *cnt_stats; unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
     unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
-    int nct, ncd;        // 16 KB chunks per target / drafter row
+    int nct, ncd;        // statistics-kernel chunks per target / drafter row
+    int ntile;           // 16 KB tiles per target row (sampling pass)
     int cps;             // chunks per segment
     int nst, nsd;        // segments per target / drafter row
 };
@@ -98,11 +99,6 @@ __device__ __forceinline__ float order_float(int i) {
 }
 __device__ __forceinline__ float warp_max(float m) {
     return order_float(__reduce_max_sync(0xffffffffu, float_order(m)));
-}
-__device__ __forceinline__ float warp_sum(float s) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(0xffffffffu, s, o);
-    return s;
 }
 __device__ __forceinline__ double warp_sum(double s) {
 #pragma unroll
@@ -310,12 +306,12 @@ template <int DT> __device__ __forceinline__ RowView<DT> segment_row(const Param
 
 // Vectors of chunk `chunk` that lie wholly inside the row: [v0, v1).  Only these are bulk-copied;
 // the (at most two) ragged vectors of a row are read element by element by the consumers.
-template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT> &rv, int chunk, int &v0, int &v1) {
+template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT> &rv, int chunk, int cvec, int &v0, int &v1) {
     constexpr int EPV = Elt<DT>::kPerVec;
     const int first_full = rv.head ? 1 : 0;
     const int end_full = (rv.V + rv.head) / EPV;               // vectors [first_full, end_full) are whole
-    v0 = max(chunk * kVecPerChunk, first_full);
-    v1 = min((chunk + 1) * kVecPerChunk, end_full);
+    v0 = max(chunk * cvec, first_full);
+    v1 = min((chunk + 1) * cvec, end_full);
     if (v1 < v0) v1 = v0;
 }
 
@@ -448,35 +444,35 @@ struct StageMeta {
     int chunk;        // chunk of the segment's row held by this stage
     int flags;        // META_*
 };
-enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_NOTICE = 8 };
+enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_NOTICE = 8, META_INTERIOR = 16 };
 
 struct StatsSmem {
-    uint64_t full[kStages];
-    uint64_t empty[kStages];
-    StageMeta meta[kStages];
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    StageMeta meta[kMaxStages];
     float2 pairs[kSWarps];
     int last;
     int error;
 };
 
-constexpr int kStatsSmemBytes = kStages * kChunkBytes + static_cast<int>(sizeof(StatsSmem));
+constexpr int kStatsSmemBytes = kRingBytes + static_cast<int>(sizeof(StatsSmem));
 
-// This thread's vectors of one chunk.  Chunks that lie wholly inside the row (all but the first
+// This thread's CV vectors of one chunk.  Chunks that lie wholly inside the row (all but the first
 // and last of a row) come straight from the stage; the others check every vector.
-template <int DT>
-__device__ __forceinline__ void load_chunk(const RowView<DT> &rv, int chunk, const uint4 *stage, int tid,
-                                           uint4 (&raw)[kSVec]) {
-    int v0, v1;
-    full_vectors<DT>(rv, chunk, v0, v1);
-    if (v0 == chunk * kVecPerChunk && v1 == (chunk + 1) * kVecPerChunk) {
+template <int DT, int CV>
+__device__ __forceinline__ void load_chunk(const RowView<DT> &rv, int chunk, bool interior, const uint4 *stage, int tid,
+                                           uint4 (&raw)[CV]) {
+    if (interior) {
 #pragma unroll
-        for (int q = 0; q < kSVec; ++q) raw[q] = stage[q * kSThreads + tid];
+        for (int q = 0; q < CV; ++q) raw[q] = stage[q * kSThreads + tid];
     } else {
+        int v0, v1;
+        full_vectors<DT>(rv, chunk, kSThreads * CV, v0, v1);
         const int nvec = rv.nvec();
 #pragma unroll
-        for (int q = 0; q < kSVec; ++q) {
+        for (int q = 0; q < CV; ++q) {
             const int g_in = q * kSThreads + tid;
-            const int v = chunk * kVecPerChunk + g_in;
+            const int v = chunk * (kSThreads * CV) + g_in;
             if (v >= v0 && v < v1) raw[q] = stage[g_in];
             else if (v < nvec) raw[q] = rv.load(v);                      // ragged end of the row
             else raw[q] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
@@ -491,55 +487,62 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
 }
 
 // One chunk of a softmax row into this thread's running (reference, sum).
-template <int DT, bool MASKED>
-__device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[kSVec], const uint32_t (&bits)[kSVec], float s,
+template <int DT, int CV, bool MASKED>
+__device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint32_t (&bits)[CV], float s,
                                               float &c_run, float &acc) {
     constexpr int EPV = Elt<DT>::kPerVec;
-    float z[kSVec][EPV];
+    // largest value of the chunk (over ids inside the intersection for a drafter row)
     float m;
     if (DT == TLI_BF16 && !MASKED) {
         uint32_t mm = bf16x2_max(bf16x2_max(raw[0].x, raw[0].y), bf16x2_max(raw[0].z, raw[0].w));
 #pragma unroll
-        for (int q = 1; q < kSVec; ++q)
+        for (int q = 1; q < CV; ++q)
             mm = bf16x2_max(mm, bf16x2_max(bf16x2_max(raw[q].x, raw[q].y), bf16x2_max(raw[q].z, raw[q].w)));
         m = fmaxf(bf16_lo(mm), bf16_hi(mm));
-#pragma unroll
-        for (int q = 0; q < kSVec; ++q) unpack<DT>(raw[q], z[q]);
     } else {
         m = -INFINITY;
 #pragma unroll
-        for (int q = 0; q < kSVec; ++q) {
-            unpack<DT>(raw[q], z[q]);
+        for (int q = 0; q < CV; ++q) {
+            float z[EPV];
+            unpack<DT>(raw[q], z);
 #pragma unroll
             for (int i = 0; i < EPV; ++i) {
-                if (MASKED) z[q][i] = ((bits[q] >> i) & 1u) ? z[q][i] : -INFINITY;
-                m = fmaxf(m, z[q][i]);
+                if (MASKED) z[i] = ((bits[q] >> i) & 1u) ? z[i] : -INFINITY;
+                m = fmaxf(m, z[i]);
             }
         }
     }
     // raise the reference if this chunk tops it; the sum follows by an exact power of two
-    const float c_new = fmaxf(c_run, reference_for(m * s));
-    acc *= pow2_neg(c_run - c_new);
-    c_run = c_new;
+    const float ms = m * s;
+    if (ms > c_run) {
+        const float c_new = reference_for(ms);
+        acc *= pow2_neg(c_run - c_new);
+        c_run = c_new;
+    }
     const float nc = -c_run;
     float a4[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-    for (int q = 0; q < kSVec; ++q) {
+    for (int q = 0; q < CV; ++q) {
+        float z[EPV];
+        unpack<DT>(raw[q], z);
 #pragma unroll
-        for (int i = 0; i < EPV; ++i) a4[i & 3] += ex2(fmaf(z[q][i], s, nc));
+        for (int i = 0; i < EPV; ++i) {
+            if (MASKED) z[i] = ((bits[q] >> i) & 1u) ? z[i] : -INFINITY;
+            a4[i & 3] += ex2(fmaf(z[i], s, nc));
+        }
     }
     acc += (a4[0] + a4[1]) + (a4[2] + a4[3]);
 }
 
-template <int DT>
-__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[kSVec], const RowView<DT> &rv, int chunk, int tid,
+template <int DT, int CV>
+__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], const RowView<DT> &rv, int chunk, int tid,
                                              float &best, int &best_idx) {
     constexpr int EPV = Elt<DT>::kPerVec;
 #pragma unroll
-    for (int q = 0; q < kSVec; ++q) {                     // increasing index order, strict > keeps the lowest
+    for (int q = 0; q < CV; ++q) {                        // increasing index order, strict > keeps the lowest
         float z[EPV];
         unpack<DT>(raw[q], z);
-        const int e0 = rv.first_elem(chunk * kVecPerChunk + q * kSThreads + tid);
+        const int e0 = rv.first_elem(chunk * (kSThreads * CV) + q * kSThreads + tid);
 #pragma unroll
         for (int i = 0; i < EPV; ++i)
             if (z[i] > best) { best = z[i]; best_idx = e0 + i; }
@@ -549,15 +552,20 @@ __device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[kSVec], const Ro
 // Segments are handed out by an atomic counter: a CTA that is busy closing a sequence simply takes
 // fewer of them.  The producer thread fetches the next segment number while it is still loading the
 // current one, streams the chunks through the stage ring and labels every stage for the consumers.
-template <int DT>
+// CV = 16-byte vectors per consumer thread per chunk: the chunk is kSThreads*CV*16 bytes and the
+// ring holds kRingBytes / that many stages.  Large batches use large chunks (less bookkeeping per
+// byte), small ones small chunks (more parallelism across CTAs).
+template <int DT, int CV>
 __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(const Params P) {
+    constexpr int CVEC = kSThreads * CV;                       // vectors per chunk
+    constexpr int NST = kRingBytes / (CVEC * 16);              // stages
+    static_assert(NST >= 2 && NST <= kMaxStages, "stage count");
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw);                       // kStages * 16 KB
-    StatsSmem &sm = *reinterpret_cast<StatsSmem *>(smem_raw + static_cast<size_t>(kStages) * kChunkBytes);
-    asm volatile("griddepcontrol.launch_dependents;");
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw);
+    StatsSmem &sm = *reinterpret_cast<StatsSmem *>(smem_raw + kRingBytes);
     if (threadIdx.x == 0) {
 #pragma unroll
-        for (int i = 0; i < kStages; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
+        for (int i = 0; i < NST; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
         sm.error = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -567,7 +575,8 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
     if (threadIdx.x < 32) {
         // ---------------- producer ----------------
         if (threadIdx.x == 0) {
-            unsigned it = 0;
+            unsigned st = 0, par = 1;                     // stage and the parity of its "empty" phase to wait for
+            unsigned issued = 0;
             bool ok = true;
             long long next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));
             while (ok) {
@@ -578,52 +587,53 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 if (g.skip) {
                     // a bad temperature is answered once per sequence, by the consumers of whoever meets its first segment
                     if (g.row == 0 && g.seg == 0) {
-                        const unsigned st = it % kStages, k = it / kStages;
-                        ok = mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error);
+                        ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
                         if (!ok) break;
                         sm.meta[st].id = id; sm.meta[st].chunk = 0; sm.meta[st].flags = META_NOTICE;
                         mbar_arrive(&sm.full[st]);
-                        ++it;
+                        ++issued;
+                        if (++st == NST) { st = 0; par ^= 1u; }
                     }
                     continue;
                 }
                 const RowView<DT> rv = segment_row<DT>(P, g);
-                for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk, ++it) {
-                    const unsigned st = it % kStages, k = it / kStages;
-                    ok = mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error);
+                for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk) {
+                    ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
                     if (!ok) break;
-                    sm.meta[st].id = id; sm.meta[st].chunk = chunk;
-                    sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0);
                     int v0, v1;
-                    full_vectors<DT>(rv, chunk, v0, v1);
+                    full_vectors<DT>(rv, chunk, CVEC, v0, v1);
+                    const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
+                    sm.meta[st].id = id; sm.meta[st].chunk = chunk;
+                    sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
+                                        (interior ? META_INTERIOR : 0);
                     const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
                     mbar_arrive_expect_tx(&sm.full[st], bytes);
                     if (bytes)
-                        bulk_load(stage_base + static_cast<size_t>(st) * kVecPerChunk + (v0 - chunk * kVecPerChunk),
+                        bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
                                   rv.vec0 + v0, bytes, &sm.full[st]);
+                    ++issued;
+                    if (++st == NST) { st = 0; par ^= 1u; }
                 }
             }
             if (ok) {                                    // tell the consumers there is nothing more
-                const unsigned st = it % kStages, k = it / kStages;
-                if (mbar_wait(&sm.empty[st], (k & 1u) ^ 1u, &sm.error, P.error)) {
+                if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
                     sm.meta[st].id = -1; sm.meta[st].chunk = 0; sm.meta[st].flags = META_END;
                     mbar_arrive(&sm.full[st]);
-                    ++it;
                 }
             }
             // After a timeout nobody may be waiting for the copies still in flight: let them land
             // (bounded) before this CTA's shared memory goes away.
             if (*reinterpret_cast<volatile int *>(&sm.error)) {
-                const unsigned lo = it > kStages ? it - kStages : 0;
-                for (unsigned j = lo; j < it; ++j) {
-                    const unsigned st = j % kStages, k = j / kStages;
-                    for (unsigned i = 0; i < kWaitLimit && !mbar_test(&sm.full[st], k & 1u); ++i) __nanosleep(64);
+                const unsigned n = issued < static_cast<unsigned>(NST) ? issued : static_cast<unsigned>(NST);
+                for (unsigned j = 0; j < n; ++j) {
+                    const unsigned sidx = (st + NST - 1 - j) % NST;           // the last n stages issued
+                    const unsigned use = (issued - 1 - j) / NST;               // how often that stage had been used before
+                    for (unsigned i = 0; i < kWaitLimit && !mbar_test(&sm.full[sidx], use & 1u); ++i) __nanosleep(64);
                 }
             }
         }
     } else {
         // ---------------- consumers ----------------
-        constexpr int EPV = Elt<DT>::kPerVec;
         const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
         Segment g;
         g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f;
@@ -633,10 +643,13 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
         float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
         bool clean_exit = false;
-        for (unsigned it = 0;; ++it) {
-            const unsigned st = it % kStages, k = it / kStages;
-            if (!mbar_wait(&sm.full[st], k & 1u, &sm.error, P.error)) break;
+        unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
+        for (;;) {
+            if (!mbar_wait(&sm.full[st], par, &sm.error, P.error)) break;
             const StageMeta meta = sm.meta[st];
+            const uint4 *stage = stage_base + static_cast<size_t>(st) * CVEC;
+            uint64_t *empty_bar = &sm.empty[st];
+            if (++st == NST) { st = 0; par ^= 1u; }
             if (meta.flags & META_END) { clean_exit = true; break; }
             if (meta.flags & (META_FIRST | META_NOTICE)) {
                 g = decode_segment(P, meta.id);
@@ -648,7 +661,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             }
             if (meta.flags & META_NOTICE) {
                 __syncwarp();
-                if (lane == 0) mbar_arrive(&sm.empty[st]);
+                if (lane == 0) mbar_arrive(empty_bar);
                 if (tid == 0) {
                     P.accepted[g.b] = 0; P.next_token[g.b] = 0;
                     if (P.status) P.status[g.b] = TLI_ROW_BAD_TEMPERATURE;
@@ -662,24 +675,24 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 continue;
             }
             const int chunk = meta.chunk;
-            uint4 raw[kSVec];
-            load_chunk<DT>(rv, chunk, stage_base + static_cast<size_t>(st) * kVecPerChunk, tid, raw);
+            uint4 raw[CV];
+            load_chunk<DT, CV>(rv, chunk, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
             __syncwarp();
-            if (lane == 0) mbar_arrive(&sm.empty[st]);                        // stage may be refilled now
+            if (lane == 0) mbar_arrive(empty_bar);                            // stage may be refilled now
             if (greedy) {
-                argmax_chunk<DT>(raw, rv, chunk, tid, best, best_idx);
+                argmax_chunk<DT, CV>(raw, rv, chunk, tid, best, best_idx);
             } else if (masked) {
-                uint32_t bits[kSVec];
+                uint32_t bits[CV];
                 const int nvec = rv.nvec();
 #pragma unroll
-                for (int q = 0; q < kSVec; ++q) {
-                    const int v = chunk * kVecPerChunk + q * kSThreads + tid;
+                for (int q = 0; q < CV; ++q) {
+                    const int v = chunk * CVEC + q * kSThreads + tid;
                     bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
                 }
-                softmax_chunk<DT, true>(raw, bits, s, c_run, acc);
+                softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
             } else {
-                const uint32_t bits[kSVec] = {};
-                softmax_chunk<DT, false>(raw, bits, s, c_run, acc);
+                const uint32_t bits[CV] = {};
+                softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
             }
             if (!(meta.flags & META_LAST)) continue;
 
@@ -815,7 +828,7 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
     double acc = 0.0;
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = tile * kVecPerChunk + k * kThreads + tid;
+        const int v = tile * kVecPerTile + k * kThreads + tid;
         if (v < nvec) {
             float w[EPV];
             vector_weights<DT>(P, sel, rt, zd_row, v, w);
@@ -839,7 +852,7 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
     constexpr int EPV = Elt<DT>::kPerVec;
     __shared__ double sm_red[kWarps];
     __shared__ double sm_tiles[kMaxTiles];
-    __shared__ float sm_seg[kVecPerChunk];
+    __shared__ float sm_seg[kVecPerTile];
     __shared__ double sm_warp_tot[kWarps];
     __shared__ int sm_last, sm_tile, sm_found, sm_lastpos, sm_retry;
     __shared__ double sm_rem;
@@ -848,7 +861,7 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     RowSel sel = P.sel[b];
     if (sel.mode == MODE_SKIP) return;
-    const int ntile = P.nct;
+    const int ntile = P.ntile;
     RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
     const void *zd_row = reinterpret_cast<const char *>(P.zd) +
         (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
@@ -917,7 +930,7 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int g = k * kThreads + tid;
-        const int v = T * kVecPerChunk + g;
+        const int v = T * kVecPerTile + g;
         float sseg = 0.f;
         if (v < nvec) {
             float w[EPV];
@@ -972,7 +985,7 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
         }
         const double rem2 = (found != INT_MAX) ? (rem - before) : INFINITY;
         float w[EPV];
-        const int v = T * kVecPerChunk + G;
+        const int v = T * kVecPerTile + G;
         vector_weights<DT>(P, sel, rt, zd_row, v, w);
         float runf = 0.f;
         int pick = -1, lastw = 0;
@@ -1003,25 +1016,33 @@ int cuda_fail(cudaError_t e, const char *what) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-int chunks_per_row(int V, int dtype) {
+int chunks_per_row(int V, int dtype, int vec_per_chunk) {
     const long long epv = dtype == TLI_F32 ? 4 : 8;
-    return static_cast<int>((static_cast<long long>(V) + epv - 1 + epv * kVecPerChunk - 1) / (epv * kVecPerChunk));
+    return static_cast<int>((static_cast<long long>(V) + epv - 1 + epv * vec_per_chunk - 1) / (epv * vec_per_chunk));
 }
 
 struct Layout {
     size_t part_t, part_d, sel, tilesum, total;
-    int nct, ncd, cps, nst, nsd;
+    int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
+    int nct, ncd, cps, nst, nsd, ntile;
     unsigned grid;
 };
 
-// Segments are sized so that every CTA of the persistent grid (two per SM) gets about eight of
-// them: long enough to amortise the per-segment reduction, short enough to balance the tail.
+// Chunk size: as large as leaves every CTA of the persistent grid (two per SM) at least ~16 chunks.
+// Segment size: about eight segments per CTA, long enough to amortise the per-segment reduction,
+// short enough to balance the tail.
 Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     Layout L;
-    L.nct = chunks_per_row(V_t, dtype);
-    L.ncd = chunks_per_row(V_d, dtype);
-    const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
+    const long long elt = dtype == TLI_F32 ? 4 : 2;
+    const long long bytes = elt * B * (static_cast<long long>(K + 1) * V_t + static_cast<long long>(K) * V_d);
     const long long ctas = static_cast<long long>(kCtasPerSm) * num_sms;
+    L.cv = 1;
+    if (bytes >= ctas * 16 * (kSThreads * 2 * 16)) L.cv = 2;
+    if (bytes >= ctas * 16 * (kSThreads * 4 * 16)) L.cv = 4;
+    L.nct = chunks_per_row(V_t, dtype, kSThreads * L.cv);
+    L.ncd = chunks_per_row(V_d, dtype, kSThreads * L.cv);
+    L.ntile = chunks_per_row(V_t, dtype, kVecPerTile);
+    const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
     long long cps = chunks / (ctas * 8);
     L.cps = static_cast<int>(cps < 1 ? 1 : (cps > 16 ? 16 : cps));
     L.nst = (L.nct + L.cps - 1) / L.cps;
@@ -1033,7 +1054,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nst, 256);
     L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.nsd, 256);
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
-    L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.nct, 256);
+    L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.ntile, 256);
     L.total = off;
     return L;
 }
@@ -1085,8 +1106,12 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     do {
         if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }
         // the statistics kernel needs more dynamic shared memory than the default limit
-        if ((e = cudaFuncSetAttribute(tli_stats_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes)) != cudaSuccess ||
-            (e = cudaFuncSetAttribute(tli_stats_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes)) != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
+        e = cudaSuccess;
+#define TLI_SET_SMEM(DT, CV) if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_stats_kernel<DT, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes)
+        TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
+        TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
+#undef TLI_SET_SMEM
+        if (e != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
@@ -1165,13 +1190,21 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
     P.error = ctx->d_counters + 2 * (TLI_MAX_B + 1);
     P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
-    P.nct = L.nct; P.ncd = L.ncd; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
+    P.nct = L.nct; P.ncd = L.ncd; P.ntile = L.ntile; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
-    const dim3 grid2(static_cast<unsigned>(L.nct), static_cast<unsigned>(a->B));
-    if (a->dtype == TLI_F32) tli_stats_kernel<TLI_F32><<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(P);
-    else tli_stats_kernel<TLI_BF16><<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(P);
+    const dim3 grid2(static_cast<unsigned>(L.ntile), static_cast<unsigned>(a->B));
+    {
+        const dim3 g1(L.grid), b1(kSThreads + 32);
+#define TLI_LAUNCH_STATS(DT, CV) tli_stats_kernel<DT, CV><<<g1, b1, kStatsSmemBytes, stream>>>(P)
+        if (a->dtype == TLI_F32) {
+            if (L.cv == 4) TLI_LAUNCH_STATS(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_F32, 2); else TLI_LAUNCH_STATS(TLI_F32, 1);
+        } else {
+            if (L.cv == 4) TLI_LAUNCH_STATS(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_BF16, 2); else TLI_LAUNCH_STATS(TLI_BF16, 1);
+        }
+#undef TLI_LAUNCH_STATS
+    }
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
