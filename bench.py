@@ -230,12 +230,14 @@ class GpuCase:
         return h2d, h["out"].numel() * h["out"].element_size()
 
     def profile(self, steps):
-        a = b = 0.0
+        """Average ms of the three kernels: statistics, decision, sampling."""
+        acc = [0.0, 0.0, 0.0]
         for _ in range(steps):
-            ms1, ms2 = self.tli.tli_verify_profile(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
+            ms = self.tli.tli_verify_profile(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
             self.calls += 1
-            a += ms1; b += ms2
-        return a / steps, b / steps
+            for i in range(3):
+                acc[i] += ms[i]
+        return tuple(x / steps for x in acc)
 
     def check(self):
         st = self.status.cpu()
@@ -301,7 +303,7 @@ def gpu_arm(args):
     ms = timed(torch, dist, args.steps, case.step, world)
     # the dominant kernel alone, with events around it, on the same stream and workload
     case.profile(3)
-    ms_stats, ms_sample = case.profile(args.steps)
+    ms_stats, ms_decide, ms_sample = case.profile(args.steps)
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
@@ -324,14 +326,15 @@ def gpu_arm(args):
         "clocks": clocks,
         "e2e": {"value": world * cfg.positions / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": 2 * args.steps,
+        "gpu_launches": 3 * args.steps,
         "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
         "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
                      "traffic": None, "algorithmic_bytes": case.bytes,
-                     "ms_stats_kernel": ms_stats, "ms_sample_kernel": ms_sample},
+                     "ms_stats_kernel": ms_stats, "ms_decide_kernel": ms_decide,
+                     "ms_sample_kernel": ms_sample},
     }
     headline_batch = case.batch
     case.close()
@@ -344,7 +347,7 @@ def gpu_arm(args):
             if c.name == cfg.name:
                 per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
                             "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
-                            "ms_sample_kernel": ms_sample})
+                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample})
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
@@ -352,11 +355,11 @@ def gpu_arm(args):
             steps = max(args.steps, 2 * k.copies)
             m = timed(torch, None, steps, k.step, 1) / steps
             k.profile(3)
-            a, b = k.profile(min(steps, 50))
+            a, d, b = k.profile(min(steps, 50))
             k.check()
             per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
                         "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
-                        "ms_stats_kernel": a, "ms_sample_kernel": b, "l2": k.l2_note})
+                        "ms_stats_kernel": a, "ms_decide_kernel": d, "ms_sample_kernel": b, "l2": k.l2_note})
             k.close()
             del k
             torch.cuda.empty_cache()

@@ -182,14 +182,13 @@ int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stre
 
 /*
  * Measurement hook: the same work as tli_verify(), with CUDA events recorded on
- * `cuda_stream` before, between and after its two kernels (the statistics pass
- * over all logits, then the sampling pass over one row per sequence).  Blocks
- * until the call has finished and returns the two durations in milliseconds
- * through [host] ms_stats and ms_sample.  Creates and destroys three events per
- * call; not meant for the serving path.
+ * `cuda_stream` around each of its three kernels.  Blocks until the call has
+ * finished and writes three durations in milliseconds to [host] ms[3]:
+ * ms[0] the statistics pass over all logits, ms[1] the per-sequence decision,
+ * ms[2] the sampling pass over one row per sequence.  Creates and destroys four
+ * events per call; not meant for the serving path.
  */
-int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream,
-                       float *ms_stats, float *ms_sample);
+int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream, float *ms);
 
 /* Vocabulary sizes and number of mapped drafter ids of a context. */
 int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped);

@@ -1,7 +1,7 @@
 // TLI verification for sm_100a: kernels and the C ABI declared in include/tli.h.
 //
-// Two launches per call, both streaming and HBM-bound (no dense contraction,
-// hence no tensor cores):
+// Three launches per call; the first and the last stream logits and are HBM-bound (no dense
+// contraction, hence no tensor cores):
 //
 //   tli_stats_kernel   persistent grid (two CTAs per SM); each CTA streams 16 KB chunks of
 //                      logit rows through a cp.async.bulk / mbarrier ring.  Target rows:
@@ -71,7 +71,7 @@ struct Params {
     const int *draft; const float *tau; const float *u;
     int *accepted; int *next_token; int *status; float *p_out; float *q_out;
     float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
-    unsigned *cnt_stats; unsigned *cnt_sample;
+    unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
     unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
     int nct, ncd;        // statistics-kernel chunks per target / drafter row
@@ -261,7 +261,7 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned b
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
-__device__ __forceinline__ void consumer_sync() {            // the eight consumer warps only
+__device__ __forceinline__ void consumer_sync() {            // the consumer warps only
     asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory");
 }
 
@@ -315,143 +315,19 @@ template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT>
     if (v1 < v0) v1 = v0;
 }
 
-// Last CTA of a sequence: fp64 combination of the segment partials, Algorithm 5's
-// acceptance tests and count, hand-over to the sampling pass.  Run by the consumer warps.
-template <int DT>
-__device__ void finalize_sequence(const Params &P, int b, float tau, int tid) {
-    __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
-    __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
-    __shared__ int sm_accept[TLI_MAX_K];
-    __shared__ int sm_flags;
-    const int lane = tid & 31, warp = tid >> 5;
-    const int K = P.K;
-    const bool greedy = (tau == 0.f);
-    const int nrows = greedy ? (K + 1) : (2 * K + 1);
-    if (tid == 0) {
-        int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
-        if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
-        sm_flags = fl;
-    }
-
-    for (int r = warp; r < nrows; r += kSWarps) {
-        const bool is_t = r <= K;
-        const int nseg = is_t ? P.nst : P.nsd;
-        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
-                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
-        if (greedy) {
-            float best = -INFINITY; int idx = INT_MAX;
-            for (int i = lane; i < nseg; i += 32) {
-                float2 pr = __ldcg(part + i);
-                int i2 = __float_as_int(pr.y);
-                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
-            }
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
-                float b2 = __shfl_xor_sync(0xffffffffu, best, o);
-                int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
-                if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
-            }
-            if (lane == 0) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
-        } else {
-            float c = kNegBig;
-            for (int i = lane; i < nseg; i += 32) c = fmaxf(c, __ldcg(part + i).x);
-            c = warp_max(c);
-            double s = 0.0;
-            for (int i = lane; i < nseg; i += 32) {
-                float2 pr = __ldcg(part + i);
-                s += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
-            }
-            s = warp_sum(s);
-            if (lane == 0) { sm_c[r] = c; sm_s[r] = s; }
-        }
-    }
-    consumer_sync();
-
-    const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
-    if (tid < K) {
-        const int j = tid;
-        const int x = P.draft[static_cast<size_t>(b) * K + j];
-        int ok = 0, fl = 0;
-        float pv = 0.f, qv = 0.f;
-        int t = -1;
-        if (x < 0 || x >= P.V_d) fl |= TLI_ROW_DRAFT_RANGE;
-        else { t = __ldg(P.map + x); if (t < 0) fl |= TLI_ROW_DRAFT_UNMAPPED; }
-        if (greedy) {
-            ok = (t >= 0 && t == static_cast<int>(sm_s[j]));
-        } else {
-            const double S_t = sm_s[j], S_d = sm_s[K + 1 + j];
-            if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
-            else if (t >= 0) {
-                const double sd = static_cast<double>(s_f);
-                const double zt = static_cast<double>(load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk + t));
-                const double zd = static_cast<double>(load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk + x));
-                const double p = exp2(zt * sd - static_cast<double>(sm_c[j])) / S_t;
-                const double q = (S_d > 0.0) ? exp2(zd * sd - static_cast<double>(sm_c[K + 1 + j])) / S_d : 0.0;
-                double thr;
-                if (q > 0.0) thr = fmin(1.0, p / q);
-                else thr = (p > 0.0) ? 1.0 : 0.0;
-                ok = static_cast<double>(P.u[static_cast<size_t>(b) * (K + 1) + j]) < thr;
-                pv = static_cast<float>(p); qv = static_cast<float>(q);
-            }
-        }
-        sm_accept[j] = ok;
-        if (fl) atomicOr(&sm_flags, fl);
-        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
-        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
-    }
-    // the bonus row's sum must be usable too
-    if (tid == K && !greedy) {
-        const double S_t = sm_s[K];
-        if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
-    }
-    consumer_sync();
-    if (tid == 0) {
-        int n = K;
-        for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
-        int fl = sm_flags;
-        RowSel sel;
-        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
-        sel.v = P.u[static_cast<size_t>(b) * (K + 1) + K];
-        if (greedy) {
-            P.next_token[b] = static_cast<int>(sm_s[n]);
-        } else if (fl & TLI_ROW_NONFINITE) {
-            n = 0;
-            P.next_token[b] = 0;
-        } else {
-            sel.c_t = sm_c[n];
-            sel.rs_t = static_cast<float>(1.0 / sm_s[n]);
-            if (n < K) {
-                const double S_d = sm_s[K + 1 + n];
-                sel.mode = MODE_RESIDUAL;
-                sel.c_d = sm_c[K + 1 + n];
-                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
-            } else {
-                sel.mode = MODE_TARGET_ONLY;
-            }
-        }
-        sel.n = n;
-        P.accepted[b] = n;
-        if (P.status) P.status[b] = fl;
-        P.sel[b] = sel;
-        P.cnt_stats[b] = 0;        // leave the ticket counter ready for the next call
-    }
-    consumer_sync();               // the shared arrays above are reused by the next sequence this CTA finishes
-}
-
 // What the producer tells the consumers about the chunk it put into a stage.
 struct StageMeta {
     long long id;     // segment
     int chunk;        // chunk of the segment's row held by this stage
     int flags;        // META_*
 };
-enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_NOTICE = 8, META_INTERIOR = 16 };
+enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_INTERIOR = 16 };
 
 struct StatsSmem {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
     StageMeta meta[kMaxStages];
-    float2 pairs[kSWarps];
-    int last;
+    float2 pairs[2][kSWarps];     // alternate per segment: one barrier per segment is enough
     int error;
 };
 
@@ -584,18 +460,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 if (id >= nseg_total) break;
                 next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));     // used one segment later
                 const Segment g = decode_segment(P, id);
-                if (g.skip) {
-                    // a bad temperature is answered once per sequence, by the consumers of whoever meets its first segment
-                    if (g.row == 0 && g.seg == 0) {
-                        ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
-                        if (!ok) break;
-                        sm.meta[st].id = id; sm.meta[st].chunk = 0; sm.meta[st].flags = META_NOTICE;
-                        mbar_arrive(&sm.full[st]);
-                        ++issued;
-                        if (++st == NST) { st = 0; par ^= 1u; }
-                    }
-                    continue;
-                }
+                if (g.skip) continue;                    // bad temperature, or drafter row at temperature 0
                 const RowView<DT> rv = segment_row<DT>(P, g);
                 for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk) {
                     ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
@@ -643,6 +508,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
         float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
         bool clean_exit = false;
+        unsigned seg_parity = 0;
         unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
         for (;;) {
             if (!mbar_wait(&sm.full[st], par, &sm.error, P.error)) break;
@@ -651,28 +517,13 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             uint64_t *empty_bar = &sm.empty[st];
             if (++st == NST) { st = 0; par ^= 1u; }
             if (meta.flags & META_END) { clean_exit = true; break; }
-            if (meta.flags & (META_FIRST | META_NOTICE)) {
+            if (meta.flags & META_FIRST) {
                 g = decode_segment(P, meta.id);
                 rv = segment_row<DT>(P, g);
                 greedy = (g.tau == 0.f);
                 masked = g.row > P.K;
                 s = 1.4426950408889634f / g.tau;
                 c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
-            }
-            if (meta.flags & META_NOTICE) {
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
-                if (tid == 0) {
-                    P.accepted[g.b] = 0; P.next_token[g.b] = 0;
-                    if (P.status) P.status[g.b] = TLI_ROW_BAD_TEMPERATURE;
-                    RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                    P.sel[g.b] = sel;
-                }
-                if (tid < P.K) {
-                    if (P.p_out) P.p_out[static_cast<size_t>(g.b) * P.K + tid] = 0.f;
-                    if (P.q_out) P.q_out[static_cast<size_t>(g.b) * P.K + tid] = 0.f;
-                }
-                continue;
             }
             const int chunk = meta.chunk;
             uint4 raw[CV];
@@ -715,12 +566,14 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 }
                 px = c_run; py = acc;
             }
-            if (lane == 0) sm.pairs[warp] = make_float2(px, py);
+            float2 *pairs = sm.pairs[seg_parity];
+            seg_parity ^= 1u;
+            if (lane == 0) pairs[warp] = make_float2(px, py);
             consumer_sync();
             if (warp == 0) {
                 float2 pr;
                 if (greedy) {
-                    pr = (lane < kSWarps) ? sm.pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
+                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
                     float bb = pr.x; int ii = __float_as_int(pr.y);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) {
@@ -730,7 +583,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     }
                     pr = make_float2(bb, __int_as_float(ii));
                 } else {
-                    pr = (lane < kSWarps) ? sm.pairs[lane] : make_float2(kNegBig, 0.f);
+                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(kNegBig, 0.f);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) {
                         float c2 = __shfl_xor_sync(0xffffffffu, pr.x, o);
@@ -743,16 +596,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                         ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
                         : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
                     __stcg(dst, pr);
-                    __threadfence();
-                    const unsigned total = greedy ? (P.K + 1) * P.nst : (P.K + 1) * P.nst + P.K * P.nsd;
-                    const unsigned ticket = atomicAdd(P.cnt_stats + g.b, 1u);
-                    sm.last = (ticket == total - 1);
                 }
-            }
-            consumer_sync();
-            if (sm.last) {
-                __threadfence();
-                finalize_sequence<DT>(P, g.b, g.tau, tid);
             }
         }
         // the last CTA to leave puts the segment counter back for the next call
@@ -763,6 +607,158 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         }
     }
 }
+
+// ---------------------------------------------------------------------------
+// decision: one CTA per sequence
+// ---------------------------------------------------------------------------
+//
+// fp64 combination of the segment partials of every row of the sequence, Algorithm 5's
+// acceptance tests (thresholds in fp64 from two gathered logits each) and count of accepted
+// drafts, hand-over to the sampling pass.  The gathers do not depend on the statistics, so they
+// are issued first and complete while the partials are being combined.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
+    const int b = blockIdx.x;
+    const int tid = threadIdx.x;
+    const float tau = __ldg(P.tau + b);
+    __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
+    __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
+    __shared__ int sm_accept[TLI_MAX_K];
+    __shared__ int sm_flags;
+    const int lane = tid & 31, warp = tid >> 5;
+    const int K = P.K;
+    if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
+        if (tid == 0) {
+            P.accepted[b] = 0; P.next_token[b] = 0;
+            if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
+            RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            P.sel[b] = sel;
+        }
+        if (tid < K) {
+            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
+            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
+        }
+        return;
+    }
+    const bool greedy = (tau == 0.f);
+    // the drafted token's two logits and its target id: loads in flight while the rows are combined
+    int g_x = -1, g_t = -1, g_fl = 0;
+    float g_zt = 0.f, g_zd = 0.f;
+    if (tid < K) {
+        g_x = P.draft[static_cast<size_t>(b) * K + tid];
+        if (g_x < 0 || g_x >= P.V_d) g_fl |= TLI_ROW_DRAFT_RANGE;
+        else { g_t = __ldg(P.map + g_x); if (g_t < 0) g_fl |= TLI_ROW_DRAFT_UNMAPPED; }
+        if (g_t >= 0 && !greedy) {
+            g_zt = load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(tid) * P.t_sk + g_t);
+            g_zd = load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(tid) * P.d_sk + g_x);
+        }
+    }
+    const int nrows = greedy ? (K + 1) : (2 * K + 1);
+    if (tid == 0) {
+        int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+        if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
+        sm_flags = fl;
+    }
+
+    for (int r = warp; r < nrows; r += kWarps) {
+        const bool is_t = r <= K;
+        const int nseg = is_t ? P.nst : P.nsd;
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
+        if (greedy) {
+            float best = -INFINITY; int idx = INT_MAX;
+            for (int i = lane; i < nseg; i += 32) {
+                float2 pr = __ldcg(part + i);
+                int i2 = __float_as_int(pr.y);
+                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+                int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
+            }
+            if (lane == 0) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
+        } else {
+            float c = kNegBig;
+            for (int i = lane; i < nseg; i += 32) c = fmaxf(c, __ldcg(part + i).x);
+            c = warp_max(c);
+            double s = 0.0;
+            for (int i = lane; i < nseg; i += 32) {
+                float2 pr = __ldcg(part + i);
+                s += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
+            }
+            s = warp_sum(s);
+            if (lane == 0) { sm_c[r] = c; sm_s[r] = s; }
+        }
+    }
+    __syncthreads();
+
+    const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
+    if (tid < K) {
+        const int j = tid;
+        int ok = 0, fl = g_fl;
+        float pv = 0.f, qv = 0.f;
+        const int t = g_t;
+        if (greedy) {
+            ok = (t >= 0 && t == static_cast<int>(sm_s[j]));
+        } else {
+            const double S_t = sm_s[j], S_d = sm_s[K + 1 + j];
+            if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
+            else if (t >= 0) {
+                const double sd = static_cast<double>(s_f);
+                const double zt = static_cast<double>(g_zt);
+                const double zd = static_cast<double>(g_zd);
+                const double p = exp2(zt * sd - static_cast<double>(sm_c[j])) / S_t;
+                const double q = (S_d > 0.0) ? exp2(zd * sd - static_cast<double>(sm_c[K + 1 + j])) / S_d : 0.0;
+                double thr;
+                if (q > 0.0) thr = fmin(1.0, p / q);
+                else thr = (p > 0.0) ? 1.0 : 0.0;
+                ok = static_cast<double>(P.u[static_cast<size_t>(b) * (K + 1) + j]) < thr;
+                pv = static_cast<float>(p); qv = static_cast<float>(q);
+            }
+        }
+        sm_accept[j] = ok;
+        if (fl) atomicOr(&sm_flags, fl);
+        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
+        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+    }
+    // the bonus row's sum must be usable too
+    if (tid == K && !greedy) {
+        const double S_t = sm_s[K];
+        if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n = K;
+        for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
+        int fl = sm_flags;
+        RowSel sel;
+        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
+        sel.v = P.u[static_cast<size_t>(b) * (K + 1) + K];
+        if (greedy) {
+            P.next_token[b] = static_cast<int>(sm_s[n]);
+        } else if (fl & TLI_ROW_NONFINITE) {
+            n = 0;
+            P.next_token[b] = 0;
+        } else {
+            sel.c_t = sm_c[n];
+            sel.rs_t = static_cast<float>(1.0 / sm_s[n]);
+            if (n < K) {
+                const double S_d = sm_s[K + 1 + n];
+                sel.mode = MODE_RESIDUAL;
+                sel.c_d = sm_c[K + 1 + n];
+                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
+            } else {
+                sel.mode = MODE_TARGET_ONLY;
+            }
+        }
+        sel.n = n;
+        P.accepted[b] = n;
+        if (P.status) P.status[b] = fl;
+        P.sel[b] = sel;
+    }
+    }
 
 // ---------------------------------------------------------------------------
 // pass 2: the extra token
@@ -856,7 +852,6 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
     __shared__ double sm_warp_tot[kWarps];
     __shared__ int sm_last, sm_tile, sm_found, sm_lastpos, sm_retry;
     __shared__ double sm_rem;
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     const int b = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     RowSel sel = P.sel[b];
@@ -1186,7 +1181,6 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.part_d = reinterpret_cast<float2 *>(ws + L.part_d);
     P.sel = reinterpret_cast<RowSel *>(ws + L.sel);
     P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
-    P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
     P.error = ctx->d_counters + 2 * (TLI_MAX_B + 1);
     P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
@@ -1209,18 +1203,16 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
 
-    // the sampling pass may be scheduled while the statistics pass drains
-    cudaLaunchConfig_t cfg;
-    memset(&cfg, 0, sizeof cfg);
-    cfg.gridDim = grid2; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0; cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1;
-    if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_F32>, P);
-    else e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_BF16>, P);
-    if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
+    if (a->dtype == TLI_F32) tli_decide_kernel<TLI_F32><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
+    else tli_decide_kernel<TLI_BF16><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_decide_kernel");
     if (ev) cudaEventRecord(ev[2], stream);
+    if (a->dtype == TLI_F32) tli_sample_kernel<TLI_F32><<<grid2, kThreads, 0, stream>>>(P);
+    else tli_sample_kernel<TLI_BF16><<<grid2, kThreads, 0, stream>>>(P);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
+    if (ev) cudaEventRecord(ev[3], stream);
     return TLI_OK;
 }
 
@@ -1228,20 +1220,17 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     return verify_impl(ctx, a, cuda_stream, nullptr);
 }
 
-int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, float *ms_stats, float *ms_sample) {
-    if (!ms_stats || !ms_sample) return TLI_ERR_ARG;
-    cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, float *ms) {
+    if (!ms) return TLI_ERR_ARG;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
     cudaError_t e = cudaSuccess;
-    for (int i = 0; i < 3 && e == cudaSuccess; ++i) e = cudaEventCreate(&ev[i]);
+    for (int i = 0; i < 4 && e == cudaSuccess; ++i) e = cudaEventCreate(&ev[i]);
     int rc = (e == cudaSuccess) ? verify_impl(ctx, a, cuda_stream, ev) : cuda_fail(e, "cudaEventCreate");
     if (rc == TLI_OK) {
-        if ((e = cudaEventSynchronize(ev[2])) != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
-        else {
-            cudaEventElapsedTime(ms_stats, ev[0], ev[1]);
-            cudaEventElapsedTime(ms_sample, ev[1], ev[2]);
-        }
+        if ((e = cudaEventSynchronize(ev[3])) != cudaSuccess) rc = cuda_fail(e, "cudaEventSynchronize");
+        else for (int i = 0; i < 3; ++i) cudaEventElapsedTime(&ms[i], ev[i], ev[i + 1]);
     }
-    for (int i = 0; i < 3; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
+    for (int i = 0; i < 4; ++i) if (ev[i]) cudaEventDestroy(ev[i]);
     return rc;
 }
 

@@ -85,7 +85,7 @@ def load() -> ctypes.CDLL:
         lib.tli_verify_static.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p]
         lib.tli_verify_static.restype = ctypes.c_int
         lib.tli_verify_profile.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p,
-                                           ctypes.POINTER(ctypes.c_float), ctypes.POINTER(ctypes.c_float)]
+                                           ctypes.POINTER(ctypes.c_float)]
         lib.tli_verify_profile.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
         lib.tli_ctx_info.restype = ctypes.c_int
@@ -181,14 +181,14 @@ def tli_verify_static(ctx: int, args: tli_verify_args, stream: Optional[int] = N
 
 
 def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
-    """tli_verify_profile(): blocks; returns (ms of the statistics kernel, ms of the sampling kernel)."""
+    """tli_verify_profile(): blocks; returns ms of (statistics kernel, decision kernel, sampling kernel)."""
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
-    a, b = ctypes.c_float(), ctypes.c_float()
-    rc = load().tli_verify_profile(ctx, ctypes.byref(args), ctypes.c_void_p(stream), ctypes.byref(a), ctypes.byref(b))
+    ms = (ctypes.c_float * 3)()
+    rc = load().tli_verify_profile(ctx, ctypes.byref(args), ctypes.c_void_p(stream), ms)
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify_profile")
-    return a.value, b.value
+    return ms[0], ms[1], ms[2]
 
 
 class Verifier:
