@@ -200,13 +200,6 @@ __device__ __forceinline__ double pow2_neg_d(float d) {
 // change of reference is an exact power of two.  Nothing to refer to (-inf) gives kNegBig.
 __device__ __forceinline__ float reference_for(float ms) { return fmaxf(ceilf(ms), kNegBig); }
 
-// (reference, sum) pairs: value = sum * 2^reference, references integer valued.
-__device__ __forceinline__ void combine_pair(float &c, float &s, float c2, float s2) {
-    const float cn = fmaxf(c, c2);
-    s = s * pow2_neg(c - cn) + s2 * pow2_neg(c2 - cn);
-    c = cn;
-}
-
 // ---------------------------------------------------------------------------
 // pass 1: statistics of every row, persistent and pipelined
 // ---------------------------------------------------------------------------
@@ -558,13 +551,12 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 }
                 px = best; py = __int_as_float(best_idx);
             } else {
+                // common reference first, then one exact rescale per lane and a plain sum
+                const float c_w = warp_max(c_run);
+                float a_w = acc * pow2_neg(c_run - c_w);
 #pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    float c2 = __shfl_xor_sync(0xffffffffu, c_run, o);
-                    float a2 = __shfl_xor_sync(0xffffffffu, acc, o);
-                    combine_pair(c_run, acc, c2, a2);
-                }
-                px = c_run; py = acc;
+                for (int o = 16; o > 0; o >>= 1) a_w += __shfl_xor_sync(0xffffffffu, a_w, o);
+                px = c_w; py = a_w;
             }
             float2 *pairs = sm.pairs[seg_parity];
             seg_parity ^= 1u;
@@ -584,12 +576,11 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     pr = make_float2(bb, __int_as_float(ii));
                 } else {
                     pr = (lane < kSWarps) ? pairs[lane] : make_float2(kNegBig, 0.f);
+                    const float c_all = warp_max(pr.x);
+                    float a_all = pr.y * pow2_neg(pr.x - c_all);
 #pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        float c2 = __shfl_xor_sync(0xffffffffu, pr.x, o);
-                        float s2 = __shfl_xor_sync(0xffffffffu, pr.y, o);
-                        combine_pair(pr.x, pr.y, c2, s2);
-                    }
+                    for (int o = 16; o > 0; o >>= 1) a_all += __shfl_xor_sync(0xffffffffu, a_all, o);
+                    pr = make_float2(c_all, a_all);
                 }
                 if (lane == 0) {
                     float2 *dst = (g.row <= P.K)
@@ -1024,8 +1015,8 @@ struct Layout {
 };
 
 // Chunk size: as large as leaves every CTA of the persistent grid (two per SM) at least ~16 chunks.
-// Segment size: about eight segments per CTA, long enough to amortise the per-segment reduction,
-// short enough to balance the tail.
+// Segment size: about four segments per CTA (they are handed out dynamically, so that is enough to
+// balance the tail) and long enough to amortise the per-segment reduction.
 Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     Layout L;
     const long long elt = dtype == TLI_F32 ? 4 : 2;
@@ -1038,7 +1029,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.ncd = chunks_per_row(V_d, dtype, kSThreads * L.cv);
     L.ntile = chunks_per_row(V_t, dtype, kVecPerTile);
     const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
-    long long cps = chunks / (ctas * 8);
+    long long cps = chunks / (ctas * 4);
     L.cps = static_cast<int>(cps < 1 ? 1 : (cps > 16 ? 16 : cps));
     L.nst = (L.nct + L.cps - 1) / L.cps;
     L.nsd = (L.ncd + L.cps - 1) / L.cps;
