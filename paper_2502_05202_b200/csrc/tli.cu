@@ -447,11 +447,13 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             unsigned st = 0, par = 1;                     // stage and the parity of its "empty" phase to wait for
             unsigned issued = 0;
             bool ok = true;
-            long long next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));
+            // every CTA starts on the segment of its own number (so that a small batch spreads over all
+            // CTAs however unevenly they start); the rest come from the counter
+            long long next = blockIdx.x;
             while (ok) {
                 const long long id = next;
                 if (id >= nseg_total) break;
-                next = static_cast<long long>(atomicAdd(P.seg_counter, 1u));     // used one segment later
+                next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);     // used one segment later
                 const Segment g = decode_segment(P, id);
                 if (g.skip) continue;                    // bad temperature, or drafter row at temperature 0
                 const RowView<DT> rv = segment_row<DT>(P, g);
@@ -611,7 +613,10 @@ template <int DT>
 __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
     const int b = blockIdx.x;
     const int tid = threadIdx.x;
+    // loads that depend on nothing go out together: temperature, this thread's uniform, (below) its draft id
     const float tau = __ldg(P.tau + b);
+    const float u_mine = (tid <= P.K) ? __ldg(P.u + static_cast<size_t>(b) * (P.K + 1) + tid) : 0.f;
+    __shared__ float sm_u_last;
     __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
     __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
     __shared__ int sm_accept[TLI_MAX_K];
@@ -645,6 +650,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         }
     }
     const int nrows = greedy ? (K + 1) : (2 * K + 1);
+    if (tid == K) sm_u_last = u_mine;
     if (tid == 0) {
         int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
         if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
@@ -705,7 +711,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
                 double thr;
                 if (q > 0.0) thr = fmin(1.0, p / q);
                 else thr = (p > 0.0) ? 1.0 : 0.0;
-                ok = static_cast<double>(P.u[static_cast<size_t>(b) * (K + 1) + j]) < thr;
+                ok = static_cast<double>(u_mine) < thr;
                 pv = static_cast<float>(p); qv = static_cast<float>(q);
             }
         }
@@ -726,7 +732,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         int fl = sm_flags;
         RowSel sel;
         sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
-        sel.v = P.u[static_cast<size_t>(b) * (K + 1) + K];
+        sel.v = sm_u_last;
         if (greedy) {
             P.next_token[b] = static_cast<int>(sm_s[n]);
         } else if (fl & TLI_ROW_NONFINITE) {
