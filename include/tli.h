@@ -181,14 +181,24 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 
 /*
- * Measurement hook: the same work as tli_verify(), with CUDA events recorded on
- * `cuda_stream` around each of its three kernels.  Blocks until the call has
- * finished and writes three durations in milliseconds to [host] ms[3]:
- * ms[0] the statistics pass over all logits, ms[1] the per-sequence decision,
- * ms[2] the sampling pass over one row per sequence.  Creates and destroys four
- * events per call; not meant for the serving path.
+ * Measurement hook: the three-kernel form of tli_verify() (see tli_set_fused)
+ * with CUDA events recorded on `cuda_stream` around each kernel.  Blocks until
+ * the call has finished and writes three durations in milliseconds to [host]
+ * ms[3]: ms[0] the statistics pass over all logits, ms[1] the per-sequence
+ * decision, ms[2] the sampling pass over one row per sequence.  Creates and
+ * destroys four events per call; not meant for the serving path.
  */
 int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream, float *ms);
+
+/*
+ * How tli_verify() and tli_verify_static() run on this context.  enabled = 1
+ * (default): one persistent kernel that streams the statistics, decides each
+ * sequence as soon as its last statistic has arrived and draws its extra token
+ * while later sequences are still streaming.  enabled = 0: the same steps as
+ * three kernels one after the other (statistics, decision, sampling).  Results
+ * are identical; the second form exists for per-kernel measurements.
+ */
+int tli_set_fused(tli_ctx *ctx, int enabled);
 
 /* Vocabulary sizes and number of mapped drafter ids of a context. */
 int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped);

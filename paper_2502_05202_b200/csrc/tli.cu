@@ -52,7 +52,7 @@ constexpr float kNegBig = -FLT_MAX;
 
 enum : int { MODE_SKIP = 0, MODE_RESIDUAL = 1, MODE_TARGET_ONLY = 2 };
 
-struct RowSel {          // what the sampling pass needs for one sequence
+struct __align__(16) RowSel {   // what the sampling pass needs for one sequence
     int n;               // accepted drafts = row to sample from
     int mode;            // MODE_*
     float s;             // log2(e) / tau
@@ -71,9 +71,12 @@ struct Params {
     const int *draft; const float *tau; const float *u;
     int *accepted; int *next_token; int *status; float *p_out; float *q_out;
     float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
-    unsigned *cnt_sample;
+    unsigned *cnt_stats; unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
     unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
+    unsigned *samp_counter;             // fused kernel: next sampling item; zero between calls
+    int *seq_state;                     // fused kernel: SEQ_* per sequence; zero between calls
+    double *stripsum;                   // fused kernel: [B][nct][kSWarps] weight sums in target-id order
     int nct, ncd;        // statistics-kernel chunks per target / drafter row
     int ntile;           // 16 KB tiles per target row (sampling pass)
     int cps;             // chunks per segment
@@ -765,11 +768,9 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
 // p(t), or max(0, p(t) - q'(inv[t])) for the residual.  The same code feeds the
 // tile sums and every rescan, so the levels of the CDF walk agree bit for bit.
 template <int DT>
-__device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
-                                               const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
+__device__ __forceinline__ void vector_weights_from(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
+                                                    const void *zd_row, float (&w)[Elt<DT>::kPerVec]) {
     constexpr int EPV = Elt<DT>::kPerVec;
-    const uint4 raw = rt.load(v);
-    const int e0 = rt.first_elem(v);
     float z[EPV];
     unpack<DT>(raw, z);
     int x[EPV];
@@ -802,6 +803,13 @@ __device__ __forceinline__ void vector_weights(const Params &P, const RowSel &se
         // p and q' are each rounded before the subtraction, so that equal distributions leave exactly 0
         w[i] = fmaxf(0.f, __fsub_rn(__fmul_rn(et, sel.rs_t), q));
     }
+}
+
+template <int DT>
+__device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
+                                               const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
+    const uint4 raw = rt.load(v);
+    vector_weights_from<DT>(P, sel, raw, rt.first_elem(v), zd_row, w);
 }
 
 template <int N> __device__ __forceinline__ float ordered_sum(const float (&w)[N]) {
@@ -996,6 +1004,664 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
 }
 
 // ---------------------------------------------------------------------------
+// the fused kernel: statistics, decisions and sampling in one persistent grid
+// ---------------------------------------------------------------------------
+//
+// The statistics kernel's machinery with two additions.  (1) Once a sequence is decided, the
+// segments of the one target row its extra token is drawn from become work items of the same
+// ring: a producer takes them (in sequence order, by compare-and-swap on one counter, as soon as
+// the sequence is marked decided) ahead of further statistics segments, so the row is still in L2.
+// Consumers turn such a chunk into weights and store one sum per warp-sized strip, in target-id
+// order.  (2) The two short serial jobs per sequence -- the decision when its last statistic
+// arrives, the CDF inversion when its last strip sum arrives -- go to a seventeenth "epilogue"
+// warp through a mailbox in shared memory, so the streaming warps never stop for them.
+// Nothing waits without bound: producers that run out of work poll for the last decisions with a
+// limit, consumers and the epilogue warp wait only on their own CTA.
+
+enum : int { META_SAMPLE = 32 };
+enum : int { SEQ_PENDING = 0, SEQ_SAMPLE = 1, SEQ_NO_SAMPLE = 2 };
+constexpr int kMailbox = 32;
+constexpr unsigned kIdleLimit = 1u << 20;
+
+struct FusedSmem {
+    uint64_t full[kMaxStages];
+    uint64_t empty[kMaxStages];
+    StageMeta meta[kMaxStages];
+    RowSel sel[kMaxStages];            // with META_SAMPLE | META_FIRST: the sequence's RowSel
+    float2 pairs[2][kSWarps];
+    int error;
+    // consumers -> epilogue warp: entry = (sequence << 1) | job, job 0 = decide, 1 = invert the CDF
+    int mail[kMailbox];
+    unsigned mail_tail, mail_head;
+    int consumers_done;
+    float ep_c[2 * TLI_MAX_K + 1];     // epilogue warp: reference (or max value) per row
+    double ep_s[2 * TLI_MAX_K + 1];    //                sum (or arg-max index) per row
+};
+
+constexpr int kFusedSmemBytes = kRingBytes + static_cast<int>(sizeof(FusedSmem));
+constexpr int kFThreads = kSThreads + 64;          // producer warp + consumers + epilogue warp
+
+__device__ __forceinline__ int ld_volatile(const int *p) { return *reinterpret_cast<const volatile int *>(p); }
+__device__ __forceinline__ unsigned ld_volatile(const unsigned *p) { return *reinterpret_cast<const volatile unsigned *>(p); }
+__device__ __forceinline__ void st_volatile(int *p, int v) { *reinterpret_cast<volatile int *>(p) = v; }
+
+// Hand a job to the epilogue warp (called by one consumer thread only).
+__device__ __forceinline__ void mail_push(FusedSmem &sm, int entry, unsigned *g_error) {
+    volatile unsigned *head = &sm.mail_head;
+    volatile unsigned *tail = &sm.mail_tail;
+    unsigned t = *tail;
+    for (unsigned i = 0; t - *head >= kMailbox; ++i) {          // full: the epilogue warp is behind
+        if (i > kIdleLimit) { atomicOr(g_error, 4u); return; }
+        __nanosleep(128);
+    }
+    reinterpret_cast<volatile int *>(sm.mail)[t % kMailbox] = entry;
+    __threadfence_block();
+    *tail = t + 1;
+}
+
+// A RowSel written by another CTA, read past L1.
+__device__ __forceinline__ RowSel load_sel(const RowSel *p) {
+    const uint4 a = __ldcg(reinterpret_cast<const uint4 *>(p));
+    const uint4 b = __ldcg(reinterpret_cast<const uint4 *>(p) + 1);
+    RowSel r;
+    r.n = static_cast<int>(a.x); r.mode = static_cast<int>(a.y);
+    r.s = __uint_as_float(a.z); r.c_t = __uint_as_float(a.w);
+    r.rs_t = __uint_as_float(b.x); r.c_d = __uint_as_float(b.y);
+    r.rs_d = __uint_as_float(b.z); r.v = __uint_as_float(b.w);
+    return r;
+}
+
+// The decision for one sequence by one warp: lanes over rows, then lanes over drafts.
+template <int DT>
+__device__ void warp_decide(const Params &P, FusedSmem &sm, int b, int lane) {
+    const int K = P.K;
+    const float tau = __ldg(P.tau + b);
+    const bool greedy = (tau == 0.f);
+    const float s_f = 1.4426950408889634f / tau;
+    // loads that depend on nothing first: uniforms, draft ids -> map -> the two logits
+    float u_j[2]; int g_t[2]; int g_fl[2]; float g_zt[2], g_zd[2];
+    const float u_last = __ldg(P.u + static_cast<size_t>(b) * (K + 1) + K);
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int j = lane + 32 * r;
+        u_j[r] = 0.f; g_t[r] = -1; g_fl[r] = 0; g_zt[r] = 0.f; g_zd[r] = 0.f;
+        if (j < K) {
+            u_j[r] = __ldg(P.u + static_cast<size_t>(b) * (K + 1) + j);
+            const int x = P.draft[static_cast<size_t>(b) * K + j];
+            if (x < 0 || x >= P.V_d) g_fl[r] = TLI_ROW_DRAFT_RANGE;
+            else { g_t[r] = __ldg(P.map + x); if (g_t[r] < 0) g_fl[r] = TLI_ROW_DRAFT_UNMAPPED; }
+            if (g_t[r] >= 0 && !greedy) {
+                g_zt[r] = load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk + g_t[r]);
+                g_zd[r] = load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk + x);
+            }
+        }
+    }
+    // every row's partials into one (reference, sum) or (max, index), a row per lane
+    const int nrows = greedy ? (K + 1) : (2 * K + 1);
+    for (int r = lane; r < nrows; r += 32) {
+        const bool is_t = r <= K;
+        const int nseg = is_t ? P.nst : P.nsd;
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
+        if (greedy) {
+            float best = -INFINITY; int idx = INT_MAX;
+            for (int i = 0; i < nseg; ++i) {
+                const float2 pr = __ldcg(part + i);
+                const int i2 = __float_as_int(pr.y);
+                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
+            }
+            sm.ep_c[r] = best; sm.ep_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx);
+        } else {
+            float c = kNegBig;
+            for (int i = 0; i < nseg; ++i) c = fmaxf(c, __ldcg(part + i).x);
+            double sum = 0.0;
+            for (int i = 0; i < nseg; ++i) {
+                const float2 pr = __ldcg(part + i);
+                sum += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
+            }
+            sm.ep_c[r] = c; sm.ep_s[r] = sum;
+        }
+    }
+    __syncwarp();
+    int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+    if (ld_volatile(P.error)) fl |= TLI_ROW_TIMEOUT;
+    int n = K;
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const int j = lane + 32 * r;
+        int ok = 1;                       // lanes beyond K do not reject
+        float pv = 0.f, qv = 0.f;
+        if (j < K) {
+            ok = 0;
+            fl |= g_fl[r];
+            const int t = g_t[r];
+            if (greedy) {
+                ok = (t >= 0 && t == static_cast<int>(sm.ep_s[j]));
+            } else {
+                const double S_t = sm.ep_s[j], S_d = sm.ep_s[K + 1 + j];
+                if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
+                else if (t >= 0) {
+                    const double sd = static_cast<double>(s_f);
+                    const double p = exp2(static_cast<double>(g_zt[r]) * sd - static_cast<double>(sm.ep_c[j])) / S_t;
+                    const double q = (S_d > 0.0) ? exp2(static_cast<double>(g_zd[r]) * sd - static_cast<double>(sm.ep_c[K + 1 + j])) / S_d : 0.0;
+                    double thr;
+                    if (q > 0.0) thr = fmin(1.0, p / q);
+                    else thr = (p > 0.0) ? 1.0 : 0.0;
+                    ok = static_cast<double>(u_j[r]) < thr;
+                    pv = static_cast<float>(p); qv = static_cast<float>(q);
+                }
+            }
+            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
+            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+        }
+        const unsigned rejected = __ballot_sync(0xffffffffu, !ok);
+        if (rejected && n == K) n = 32 * r + (__ffs(rejected) - 1);
+    }
+    if (!greedy) {                        // the bonus row's sum must be usable too
+        const double S_k = sm.ep_s[K];
+        if (!(S_k > 0.0) || !isfinite(S_k)) fl |= TLI_ROW_NONFINITE;
+    }
+    fl = __reduce_or_sync(0xffffffffu, fl);
+    if (lane == 0) {
+        RowSel sel;
+        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
+        sel.v = u_last;
+        if (greedy) {
+            P.next_token[b] = static_cast<int>(sm.ep_s[n]);
+        } else if (fl & TLI_ROW_NONFINITE) {
+            n = 0;
+            P.next_token[b] = 0;
+        } else {
+            sel.c_t = sm.ep_c[n];
+            sel.rs_t = static_cast<float>(1.0 / sm.ep_s[n]);
+            if (n < K) {
+                const double S_d = sm.ep_s[K + 1 + n];
+                sel.mode = MODE_RESIDUAL;
+                sel.c_d = sm.ep_c[K + 1 + n];
+                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
+            } else {
+                sel.mode = MODE_TARGET_ONLY;
+            }
+        }
+        sel.n = n;
+        P.accepted[b] = n;
+        if (P.status) P.status[b] = fl;
+        P.sel[b] = sel;
+        __threadfence();                  // the RowSel before the mark that lets producers take the sequence
+        st_volatile(P.seq_state + b, sel.mode == MODE_SKIP ? SEQ_NO_SAMPLE : SEQ_SAMPLE);
+    }
+    __syncwarp();
+}
+
+// Strip (chunk, warp) of the sampled row: vectors chunk*CVEC + warp*32*CV + q*32 + lane, q < CV.
+// Sum of one lane's CV vectors of the strip, the vectors' own sums in vs[].
+template <int DT, int CV>
+__device__ __forceinline__ double strip_lane_sum(const Params &P, const RowSel &sel, const RowView<DT> &rt,
+                                                 const void *zd_row, int chunk, int w, int lane, float (&vs)[CV]) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int nvec = rt.nvec();
+    double acc = 0.0;
+#pragma unroll
+    for (int q = 0; q < CV; ++q) {
+        const int v = chunk * (kSThreads * CV) + w * (32 * CV) + q * 32 + lane;
+        vs[q] = 0.f;
+        if (v < nvec) {
+            float wt[EPV];
+            vector_weights<DT>(P, sel, rt, zd_row, v, wt);
+            vs[q] = ordered_sum(wt);
+        }
+        acc += static_cast<double>(vs[q]);
+    }
+    return acc;
+}
+
+// CDF inversion for one sequence by one warp: strip sums -> strip -> vector -> element.
+template <int DT, int CV>
+__device__ void warp_select(const Params &P, int b, int lane) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    RowSel sel = load_sel(P.sel + b);
+    const int ntot = P.nct * kSWarps;
+    double *base = P.stripsum + static_cast<size_t>(b) * ntot;
+    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
+        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
+    const int per = (ntot + 31) / 32;
+    const int i0 = min(lane * per, ntot), i1 = min(i0 + per, ntot);
+    int token = 0;
+    bool done = false;
+    for (int attempt = 0; attempt < 2 && !done; ++attempt) {
+        double mine = 0.0;
+        for (int i = i0; i < i1; ++i) mine += __ldcg(base + i);
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        const double R = __shfl_sync(0xffffffffu, incl, 31);
+        if (!(R > 0.0) || !isfinite(R)) {
+            if (attempt == 1) {                    // no usable mass even from p: give up on the row
+                if (lane == 0 && P.status) P.status[b] |= TLI_ROW_NONFINITE;
+                token = 0; done = true;
+                break;
+            }
+            // zero residual mass: sample from p of the same position instead
+            sel.mode = MODE_TARGET_ONLY;
+            if (lane == 0 && P.status) P.status[b] |= TLI_ROW_FALLBACK;
+            for (int e = 0; e < ntot; ++e) {
+                float vs[CV];
+                const double t2 = warp_sum(strip_lane_sum<DT, CV>(P, sel, rt, zd_row, e / kSWarps, e % kSWarps, lane, vs));
+                if (lane == 0) base[e] = t2;
+            }
+            __threadfence();
+            __syncwarp();
+            continue;
+        }
+        const double target = static_cast<double>(sel.v) * R;
+        // the lane whose block holds the target, else the last lane with any mass
+        const unsigned over = __ballot_sync(0xffffffffu, incl > target);
+        const unsigned some = __ballot_sync(0xffffffffu, mine > 0.0);
+        const bool clamped = (over == 0u);
+        const int L = clamped ? (31 - __clz(some)) : (__ffs(over) - 1);
+        const double before_L = __shfl_sync(0xffffffffu, incl - mine, L);
+        int found = -1;
+        double rem = 0.0;
+        if (lane == L) {
+            const double want = clamped ? INFINITY : (target - before_L);
+            double run = 0.0;
+            int lastpos = i0;
+            for (int i = i0; i < i1; ++i) {
+                const double x = __ldcg(base + i);
+                if (x > 0.0) lastpos = i;
+                if (found < 0 && run + x > want) { found = i; rem = want - run; }
+                run += x;
+            }
+            if (found < 0) { found = lastpos; rem = INFINITY; }
+        }
+        found = __shfl_sync(0xffffffffu, found, L);
+        rem = __shfl_sync(0xffffffffu, rem, L);
+        // the strip's vectors again, in order: q-major, then lane
+        const int chunk = found / kSWarps, w = found % kSWarps;
+        float vs[CV];
+        strip_lane_sum<DT, CV>(P, sel, rt, zd_row, chunk, w, lane, vs);
+        double run = 0.0;
+        int pick_q = -1, pick_lane = -1;
+        double pick_before = 0.0;
+        int last_q = -1, last_lane = -1;
+#pragma unroll
+        for (int q = 0; q < CV; ++q) {
+            const double x = static_cast<double>(vs[q]);
+            double inc = x;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const double up = __shfl_up_sync(0xffffffffu, inc, o);
+                if (lane >= o) inc += up;
+            }
+            const unsigned ov = __ballot_sync(0xffffffffu, run + inc > rem);
+            const unsigned pos = __ballot_sync(0xffffffffu, x > 0.0);
+            if (pos) { last_q = q; last_lane = 31 - __clz(pos); }
+            if (pick_q < 0 && ov) {
+                pick_q = q; pick_lane = __ffs(ov) - 1;
+                pick_before = run + __shfl_sync(0xffffffffu, inc - x, pick_lane);
+            }
+            run += __shfl_sync(0xffffffffu, inc, 31);
+        }
+        double rem2 = rem - pick_before;
+        if (pick_q < 0) { pick_q = last_q; pick_lane = last_lane; rem2 = INFINITY; }
+        if (pick_q < 0) { token = 0; done = true; break; }       // cannot happen when the strip has mass
+        if (lane == pick_lane) {
+            // walk the elements of that vector with the same running fp32 sum that formed its total
+            const int v = chunk * (kSThreads * CV) + w * (32 * CV) + pick_q * 32 + lane;
+            float wt[EPV];
+            vector_weights<DT>(P, sel, rt, zd_row, v, wt);
+            float runf = 0.f;
+            int pick = -1, lastw = 0;
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                runf = (i == 0) ? wt[0] : __fadd_rn(runf, wt[i]);
+                if (wt[i] > 0.f) lastw = i;
+                if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
+            }
+            if (pick < 0) pick = lastw;
+            token = min(max(rt.first_elem(v) + pick, 0), P.V_t - 1);
+        }
+        token = __shfl_sync(0xffffffffu, token, pick_lane);
+        done = true;
+    }
+    if (lane == 0) {
+        P.next_token[b] = token;
+        st_volatile(P.seq_state + b, SEQ_PENDING);       // ready for the next call
+    }
+    __syncwarp();
+}
+
+template <int DT, int CV>
+__global__ void __launch_bounds__(kFThreads, kCtasPerSm) tli_fused_kernel(const Params P) {
+    constexpr int CVEC = kSThreads * CV;                       // vectors per chunk
+    constexpr int NST = kRingBytes / (CVEC * 16);              // stages
+    constexpr int EPV = Elt<DT>::kPerVec;
+    static_assert(NST >= 2 && NST <= kMaxStages, "stage count");
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw);
+    FusedSmem &sm = *reinterpret_cast<FusedSmem *>(smem_raw + kRingBytes);
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int i = 0; i < NST; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
+        sm.error = 0; sm.mail_tail = 0; sm.mail_head = 0; sm.consumers_done = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const long long nseg_total = static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
+    const long long nsamp_total = static_cast<long long>(P.B) * P.nst;
+
+    if (threadIdx.x < 32) {
+        // ---------------- producer ----------------
+        if (threadIdx.x == 0) {
+            unsigned st = 0, par = 1;                     // stage and the parity of its "empty" phase to wait for
+            unsigned issued = 0, idle = 0;
+            bool ok = true;
+            long long next = blockIdx.x;                  // own number first, then from the counter
+            while (ok) {
+                // sampling items first: their rows are still in L2
+                const long long k = ld_volatile(P.samp_counter);
+                if (k < nsamp_total) {
+                    const int b = static_cast<int>(k / P.nst);
+                    const int state = ld_volatile(P.seq_state + b);
+                    if (state != SEQ_PENDING) {
+                        if (atomicCAS(P.samp_counter, static_cast<unsigned>(k), static_cast<unsigned>(k) + 1u) == static_cast<unsigned>(k)) {
+                            idle = 0;
+                            const int seg = static_cast<int>(k - static_cast<long long>(b) * P.nst);
+                            if (state == SEQ_NO_SAMPLE) {
+                                if (seg == P.nst - 1) st_volatile(P.seq_state + b, SEQ_PENDING);   // last item: ready for the next call
+                            } else {
+                                __threadfence();
+                                const RowSel sel = load_sel(P.sel + b);
+                                const RowView<DT> rv(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+                                const int c0 = seg * P.cps, c1 = min(c0 + P.cps, P.nct);
+                                for (int chunk = c0; chunk < c1; ++chunk) {
+                                    ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
+                                    if (!ok) break;
+                                    int v0, v1;
+                                    full_vectors<DT>(rv, chunk, CVEC, v0, v1);
+                                    const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
+                                    sm.meta[st].id = k; sm.meta[st].chunk = chunk;
+                                    sm.meta[st].flags = META_SAMPLE | (chunk == c0 ? META_FIRST : 0) | (chunk == c1 - 1 ? META_LAST : 0) |
+                                                        (interior ? META_INTERIOR : 0);
+                                    if (chunk == c0) sm.sel[st] = sel;
+                                    const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
+                                    mbar_arrive_expect_tx(&sm.full[st], bytes);
+                                    if (bytes)
+                                        bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
+                                                  rv.vec0 + v0, bytes, &sm.full[st]);
+                                    ++issued;
+                                    if (++st == NST) { st = 0; par ^= 1u; }
+                                }
+                            }
+                        }
+                        continue;
+                    }
+                }
+                if (next < nseg_total) {
+                    idle = 0;
+                    const long long id = next;
+                    next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);     // used one segment later
+                    const Segment g = decode_segment(P, id);
+                    if (g.skip) {                            // bad temperature, or drafter row at temperature 0
+                        // a sequence with a bad temperature has no statistics: it is answered here, once
+                        if (g.row == 0 && g.seg == 0) {
+                            P.accepted[g.b] = 0; P.next_token[g.b] = 0;
+                            if (P.status) P.status[g.b] = TLI_ROW_BAD_TEMPERATURE;
+                            for (int j = 0; j < P.K; ++j) {
+                                if (P.p_out) P.p_out[static_cast<size_t>(g.b) * P.K + j] = 0.f;
+                                if (P.q_out) P.q_out[static_cast<size_t>(g.b) * P.K + j] = 0.f;
+                            }
+                            __threadfence();
+                            st_volatile(P.seq_state + g.b, SEQ_NO_SAMPLE);
+                        }
+                        continue;
+                    }
+                    const RowView<DT> rv = segment_row<DT>(P, g);
+                    for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk) {
+                        ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
+                        if (!ok) break;
+                        int v0, v1;
+                        full_vectors<DT>(rv, chunk, CVEC, v0, v1);
+                        const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
+                        sm.meta[st].id = id; sm.meta[st].chunk = chunk;
+                        sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
+                                            (interior ? META_INTERIOR : 0);
+                        const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
+                        mbar_arrive_expect_tx(&sm.full[st], bytes);
+                        if (bytes)
+                            bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
+                                      rv.vec0 + v0, bytes, &sm.full[st]);
+                        ++issued;
+                        if (++st == NST) { st = 0; par ^= 1u; }
+                    }
+                    continue;
+                }
+                if (k >= nsamp_total) break;                 // all work handed out
+                // every statistic is handed out; the last sequences are still being decided
+                if (++idle > kIdleLimit) { sm.error = 1; atomicOr(P.error, 8u); ok = false; break; }
+                __nanosleep(256);
+            }
+            if (ok) {                                    // tell the consumers there is nothing more
+                if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
+                    sm.meta[st].id = -1; sm.meta[st].chunk = 0; sm.meta[st].flags = META_END;
+                    mbar_arrive(&sm.full[st]);
+                }
+            }
+            // After a timeout nobody may be waiting for the copies still in flight: let them land
+            // (bounded) before this CTA's shared memory goes away.
+            if (*reinterpret_cast<volatile int *>(&sm.error)) {
+                const unsigned n = issued < static_cast<unsigned>(NST) ? issued : static_cast<unsigned>(NST);
+                for (unsigned j = 0; j < n; ++j) {
+                    const unsigned sidx = (st + NST - 1 - j) % NST;           // the last n stages issued
+                    const unsigned use = (issued - 1 - j) / NST;               // how often that stage had been used before
+                    for (unsigned i = 0; i < kWaitLimit && !mbar_test(&sm.full[sidx], use & 1u); ++i) __nanosleep(64);
+                }
+            }
+        }
+    } else if (threadIdx.x >= 32 + kSThreads) {
+        // ---------------- epilogue warp ----------------
+        const int lane = threadIdx.x & 31;
+        unsigned head = 0;
+        for (unsigned spins = 0;;) {
+            const unsigned tail = *reinterpret_cast<volatile unsigned *>(&sm.mail_tail);
+            if (head == tail) {
+                if (*reinterpret_cast<volatile int *>(&sm.consumers_done) &&
+                    head == *reinterpret_cast<volatile unsigned *>(&sm.mail_tail)) break;
+                if (++spins > (1u << 24)) { if (lane == 0) atomicOr(P.error, 16u); break; }
+                __nanosleep(200);
+                continue;
+            }
+            spins = 0;
+            const int entry = reinterpret_cast<volatile int *>(sm.mail)[head % kMailbox];
+            ++head;
+            __syncwarp();
+            if (lane == 0) *reinterpret_cast<volatile unsigned *>(&sm.mail_head) = head;
+            __threadfence();
+            if (entry & 1) warp_select<DT, CV>(P, entry >> 1, lane);
+            else warp_decide<DT>(P, sm, entry >> 1, lane);
+        }
+    } else {
+        // ---------------- consumers ----------------
+        const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
+        Segment g;
+        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f;
+        RowView<DT> rv(P.zt, 0, P.V_t);
+        bool greedy = false, masked = false;
+        float s = 0.f;
+        float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
+        float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
+        RowSel ssel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // sampling items
+        const void *zd_row = P.zd;
+        int sb = 0;
+        bool clean_exit = false;
+        unsigned seg_parity = 0;
+        unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
+        for (;;) {
+            if (!mbar_wait(&sm.full[st], par, &sm.error, P.error)) break;
+            const StageMeta meta = sm.meta[st];
+            const uint4 *stage = stage_base + static_cast<size_t>(st) * CVEC;
+            uint64_t *empty_bar = &sm.empty[st];
+            const unsigned st_now = st;
+            if (++st == NST) { st = 0; par ^= 1u; }
+            if (meta.flags & META_END) { clean_exit = true; break; }
+            const int chunk = meta.chunk;
+
+            if (meta.flags & META_SAMPLE) {
+                // ---- a chunk of the row the extra token is drawn from: weights, one sum per warp strip ----
+                if (meta.flags & META_FIRST) {
+                    sb = static_cast<int>(meta.id / P.nst);
+                    ssel = sm.sel[st_now];
+                    rv = RowView<DT>(P.zt, static_cast<long long>(sb) * P.t_sb + static_cast<long long>(ssel.n) * P.t_sk, P.V_t);
+                    zd_row = reinterpret_cast<const char *>(P.zd) +
+                        (static_cast<long long>(sb) * P.d_sb + static_cast<long long>(ssel.n < P.K ? ssel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
+                }
+                uint4 raw[CV];
+                int vidx[CV];
+                {
+                    int v0 = 0, v1 = 0;
+                    const bool interior = (meta.flags & META_INTERIOR) != 0;
+                    if (!interior) full_vectors<DT>(rv, chunk, CVEC, v0, v1);
+                    const int nvec = rv.nvec();
+#pragma unroll
+                    for (int q = 0; q < CV; ++q) {
+                        const int g_in = warp * (32 * CV) + q * 32 + lane;        // strips are contiguous in target-id order
+                        const int v = chunk * CVEC + g_in;
+                        vidx[q] = v;
+                        if (interior || (v >= v0 && v < v1)) raw[q] = stage[g_in];
+                        else if (v < nvec) raw[q] = rv.load(v);
+                        else { raw[q] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord); vidx[q] = -1; }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(empty_bar);
+                double wsum = 0.0;
+#pragma unroll
+                for (int q = 0; q < CV; ++q) {
+                    float vsum = 0.f;
+                    if (vidx[q] >= 0) {
+                        float wt[EPV];
+                        vector_weights_from<DT>(P, ssel, raw[q], rv.first_elem(vidx[q]), zd_row, wt);
+                        vsum = ordered_sum(wt);
+                    }
+                    wsum += static_cast<double>(vsum);
+                }
+                wsum = warp_sum(wsum);
+                if (lane == 0) __stcg(P.stripsum + (static_cast<size_t>(sb) * P.nct + chunk) * kSWarps + warp, wsum);
+                if (!(meta.flags & META_LAST)) continue;
+                if (lane == 0) __threadfence();
+                consumer_sync();
+                if (tid == 0) {
+                    if (atomicAdd(P.cnt_sample + sb, 1u) == static_cast<unsigned>(P.nst) - 1u) {
+                        P.cnt_sample[sb] = 0;
+                        mail_push(sm, (sb << 1) | 1, P.error);
+                    }
+                }
+                continue;
+            }
+
+            if (meta.flags & META_FIRST) {
+                g = decode_segment(P, meta.id);
+                rv = segment_row<DT>(P, g);
+                greedy = (g.tau == 0.f);
+                masked = g.row > P.K;
+                s = 1.4426950408889634f / g.tau;
+                c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
+            }
+            uint4 raw[CV];
+            load_chunk<DT, CV>(rv, chunk, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_bar);                            // stage may be refilled now
+            if (greedy) {
+                argmax_chunk<DT, CV>(raw, rv, chunk, tid, best, best_idx);
+            } else if (masked) {
+                uint32_t bits[CV];
+                const int nvec = rv.nvec();
+#pragma unroll
+                for (int q = 0; q < CV; ++q) {
+                    const int v = chunk * CVEC + q * kSThreads + tid;
+                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
+                }
+                softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
+            } else {
+                const uint32_t bits[CV] = {};
+                softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
+            }
+            if (!(meta.flags & META_LAST)) continue;
+
+            // ---- segment done: one (reference, sum) or (max, index) pair per warp, then per CTA ----
+            float px, py;
+            if (greedy) {
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                    float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+                    int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
+                    if (b2 > best || (b2 == best && i2 < best_idx)) { best = b2; best_idx = i2; }
+                }
+                px = best; py = __int_as_float(best_idx);
+            } else {
+                const float c_w = warp_max(c_run);
+                float a_w = acc * pow2_neg(c_run - c_w);
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) a_w += __shfl_xor_sync(0xffffffffu, a_w, o);
+                px = c_w; py = a_w;
+            }
+            float2 *pairs = sm.pairs[seg_parity];
+            seg_parity ^= 1u;
+            if (lane == 0) pairs[warp] = make_float2(px, py);
+            consumer_sync();
+            if (warp == 0) {
+                float2 pr;
+                if (greedy) {
+                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
+                    float bb = pr.x; int ii = __float_as_int(pr.y);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) {
+                        float b2 = __shfl_xor_sync(0xffffffffu, bb, o);
+                        int i2 = __shfl_xor_sync(0xffffffffu, ii, o);
+                        if (b2 > bb || (b2 == bb && i2 < ii)) { bb = b2; ii = i2; }
+                    }
+                    pr = make_float2(bb, __int_as_float(ii));
+                } else {
+                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(kNegBig, 0.f);
+                    const float c_all = warp_max(pr.x);
+                    float a_all = pr.y * pow2_neg(pr.x - c_all);
+#pragma unroll
+                    for (int o = 16; o > 0; o >>= 1) a_all += __shfl_xor_sync(0xffffffffu, a_all, o);
+                    pr = make_float2(c_all, a_all);
+                }
+                if (lane == 0) {
+                    float2 *dst = (g.row <= P.K)
+                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
+                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
+                    __stcg(dst, pr);
+                    // the last partial of a sequence: its decision goes to the epilogue warp
+                    __threadfence();
+                    const unsigned total = greedy ? (P.K + 1) * P.nst : (P.K + 1) * P.nst + P.K * P.nsd;
+                    if (atomicAdd(P.cnt_stats + g.b, 1u) == total - 1u) {
+                        P.cnt_stats[g.b] = 0;
+                        mail_push(sm, g.b << 1, P.error);
+                    }
+                }
+            }
+        }
+        if (tid == 0) {
+            __threadfence_block();
+            *reinterpret_cast<volatile int *>(&sm.consumers_done) = 1;
+            // the last CTA to leave puts the schedulers' counters back for the next call
+            if (clean_exit) {
+                __threadfence();
+                const unsigned t = atomicAdd(P.cta_done, 1u);
+                if (t == gridDim.x - 1) { *P.seg_counter = 0u; *P.samp_counter = 0u; *P.cta_done = 0u; __threadfence(); }
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
 
@@ -1014,7 +1680,7 @@ int chunks_per_row(int V, int dtype, int vec_per_chunk) {
 }
 
 struct Layout {
-    size_t part_t, part_d, sel, tilesum, total;
+    size_t part_t, part_d, sel, tilesum, stripsum, total;
     int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
     int nct, ncd, cps, nst, nsd, ntile;
     unsigned grid;
@@ -1047,6 +1713,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.nsd, 256);
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
     L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.ntile, 256);
+    L.stripsum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.nct * kSWarps, 256);
     L.total = off;
     return L;
 }
@@ -1059,7 +1726,9 @@ struct tli_ctx {
     int *d_map;
     int *d_inv;
     uint32_t *d_mask;
-    unsigned *d_counters;       // [2 * (TLI_MAX_B + 1) + 3], zero between calls; last words: sticky error, scheduler
+    int fused;                  // option: one fused kernel (default) or three kernels
+    unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 4], zero between calls: tickets, tickets, sequence states,
+                                // sticky error, schedulers
     int num_sms;
 };
 
@@ -1094,6 +1763,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
+    c->fused = 1;
     int rc = TLI_OK;
     do {
         if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }
@@ -1103,15 +1773,19 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
         TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
 #undef TLI_SET_SMEM
+#define TLI_SET_SMEM(DT, CV) if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_fused_kernel<DT, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBytes)
+        TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
+        TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
+#undef TLI_SET_SMEM
         if (e != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
-        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (2 * (TLI_MAX_B + 1) + 3))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 4))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
         if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
         if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
         if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
-        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (2 * (TLI_MAX_B + 1) + 3))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
+        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 4))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
     } while (0);
     if (rc != TLI_OK) {
         cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
@@ -1178,13 +1852,29 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.part_d = reinterpret_cast<float2 *>(ws + L.part_d);
     P.sel = reinterpret_cast<RowSel *>(ws + L.sel);
     P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
+    P.stripsum = reinterpret_cast<double *>(ws + L.stripsum);
+    P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
-    P.error = ctx->d_counters + 2 * (TLI_MAX_B + 1);
-    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
+    P.seq_state = reinterpret_cast<int *>(ctx->d_counters + 2 * (TLI_MAX_B + 1));
+    P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
+    P.seg_counter = P.error + 1; P.cta_done = P.error + 2; P.samp_counter = P.error + 3;
     P.nct = L.nct; P.ncd = L.ncd; P.ntile = L.ntile; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
+    if (ctx->fused && !ev) {
+        const dim3 g1(L.grid), b1(kFThreads);
+#define TLI_LAUNCH_FUSED(DT, CV) tli_fused_kernel<DT, CV><<<g1, b1, kFusedSmemBytes, stream>>>(P)
+        if (a->dtype == TLI_F32) {
+            if (L.cv == 4) TLI_LAUNCH_FUSED(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_FUSED(TLI_F32, 2); else TLI_LAUNCH_FUSED(TLI_F32, 1);
+        } else {
+            if (L.cv == 4) TLI_LAUNCH_FUSED(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_FUSED(TLI_BF16, 2); else TLI_LAUNCH_FUSED(TLI_BF16, 1);
+        }
+#undef TLI_LAUNCH_FUSED
+        const cudaError_t ef = cudaGetLastError();
+        if (ef != cudaSuccess) return cuda_fail(ef, "launch tli_fused_kernel");
+        return TLI_OK;
+    }
     const dim3 grid2(static_cast<unsigned>(L.ntile), static_cast<unsigned>(a->B));
     {
         const dim3 g1(L.grid), b1(kSThreads + 32);
@@ -1215,6 +1905,12 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
 
 int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     return verify_impl(ctx, a, cuda_stream, nullptr);
+}
+
+int tli_set_fused(tli_ctx *ctx, int enabled) {
+    if (!ctx) return TLI_ERR_ARG;
+    ctx->fused = enabled ? 1 : 0;
+    return TLI_OK;
 }
 
 int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, float *ms) {

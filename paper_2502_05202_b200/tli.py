@@ -37,7 +37,7 @@ TLI_MAX_K = 64
 TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -87,6 +87,8 @@ def load() -> ctypes.CDLL:
         lib.tli_verify_profile.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p,
                                            ctypes.POINTER(ctypes.c_float)]
         lib.tli_verify_profile.restype = ctypes.c_int
+        lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        lib.tli_set_fused.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
         lib.tli_ctx_info.restype = ctypes.c_int
         lib.tli_status_string.argtypes = [ctypes.c_int]
@@ -191,13 +193,22 @@ def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = 
     return ms[0], ms[1], ms[2]
 
 
+def tli_set_fused(ctx: int, enabled: bool) -> None:
+    """tli_set_fused(): one fused kernel per call (default) or three kernels."""
+    rc = load().tli_set_fused(ctx, 1 if enabled else 0)
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_set_fused")
+
+
 class Verifier:
     """Convenience owner of one context plus its scratch and output tensors."""
 
-    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0):
+    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0, fused: bool = True):
         self.device = torch.device("cuda", device)
         self.V_t, self.V_d = int(V_t), int(V_d)
         self.ctx = tli_create(device, V_t, V_d, id_map)
+        if not fused:
+            tli_set_fused(self.ctx, False)
         self._ws: Optional[torch.Tensor] = None
 
     def close(self) -> None:

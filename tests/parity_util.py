@@ -43,19 +43,33 @@ def to_device(batch: Dict[str, np.ndarray], device="cuda") -> Dict[str, torch.Te
 
 def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = None,
             dev: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, np.ndarray]:
-    own = verifier is None
-    if own:
-        V_t = batch["target_logits"].shape[2]
-        V_d = batch["drafter_logits"].shape[2]
-        verifier = tli.Verifier(V_t, V_d, batch["id_map"])
+    """One tli_verify() call.  Without a verifier of the caller's, both forms of the call are run
+    (the fused kernel and the three-kernel sequence) and must agree bit for bit."""
     if dev is None:
         dev = to_device(batch)
-    out = verifier.verify(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"],
-                          dev["temperature"], dev["uniforms"])
-    torch.cuda.synchronize()
-    res = {k: v.cpu().numpy() for k, v in out.items()}
-    if own:
-        verifier.close()
+
+    def once(v):
+        out = v.verify(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"],
+                       dev["temperature"], dev["uniforms"])
+        torch.cuda.synchronize()
+        return {k: x.cpu().numpy() for k, x in out.items()}
+
+    if verifier is not None:
+        return once(verifier)
+    V_t = batch["target_logits"].shape[2]
+    V_d = batch["drafter_logits"].shape[2]
+    res = None
+    for fused in (False, True):
+        v = tli.Verifier(V_t, V_d, batch["id_map"], fused=fused)
+        r = once(v)
+        r2 = once(v)                                  # a second call on the same context: counters came back to zero
+        v.close()
+        for k in r:
+            np.testing.assert_array_equal(r[k], r2[k], err_msg="repeat call differs (%s, fused=%s)" % (k, fused))
+        if res is not None:
+            for k in r:
+                np.testing.assert_array_equal(res[k], r[k], err_msg="fused and three-kernel results differ: " + k)
+        res = r
     return res
 
 
