@@ -191,12 +191,14 @@ int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stre
 int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream, float *ms);
 
 /*
- * How tli_verify() and tli_verify_static() run on this context.  enabled = 1
- * (default): one persistent kernel that streams the statistics, decides each
- * sequence as soon as its last statistic has arrived and draws its extra token
- * while later sequences are still streaming.  enabled = 0: the same steps as
- * three kernels one after the other (statistics, decision, sampling).  Results
- * are identical; the second form exists for per-kernel measurements.
+ * How tli_verify() and tli_verify_static() run on this context.  enabled = 0
+ * (default): three kernels one after the other (statistics, decision,
+ * sampling).  enabled = 1: one persistent kernel that streams the statistics,
+ * decides each sequence as soon as its last statistic has arrived and draws its
+ * extra token while later sequences are still streaming.  Results are identical
+ * bit for bit.  The fused form is the slower one today (its sampling chunks
+ * stall the streaming warps on their gathers) and is kept as the basis for
+ * further work; see the design doc.
  */
 int tli_set_fused(tli_ctx *ctx, int enabled);
 

@@ -1763,7 +1763,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
-    c->fused = 1;
+    c->fused = 0;
     int rc = TLI_OK;
     do {
         if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }

@@ -194,7 +194,7 @@ def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = 
 
 
 def tli_set_fused(ctx: int, enabled: bool) -> None:
-    """tli_set_fused(): one fused kernel per call (default) or three kernels."""
+    """tli_set_fused(): three kernels per call (default) or one fused kernel."""
     rc = load().tli_set_fused(ctx, 1 if enabled else 0)
     if rc != TLI_OK:
         raise TLIError(rc, "tli_set_fused")
@@ -203,12 +203,12 @@ def tli_set_fused(ctx: int, enabled: bool) -> None:
 class Verifier:
     """Convenience owner of one context plus its scratch and output tensors."""
 
-    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0, fused: bool = True):
+    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0, fused: bool = False):
         self.device = torch.device("cuda", device)
         self.V_t, self.V_d = int(V_t), int(V_d)
         self.ctx = tli_create(device, V_t, V_d, id_map)
-        if not fused:
-            tli_set_fused(self.ctx, False)
+        if fused:
+            tli_set_fused(self.ctx, True)
         self._ws: Optional[torch.Tensor] = None
 
     def close(self) -> None:
