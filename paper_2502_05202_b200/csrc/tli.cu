@@ -624,7 +624,6 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
     __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
     __shared__ int sm_accept[TLI_MAX_K];
     __shared__ int sm_flags;
-    const int lane = tid & 31, warp = tid >> 5;
     const int K = P.K;
     if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
         if (tid == 0) {
@@ -660,36 +659,49 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         sm_flags = fl;
     }
 
-    for (int r = warp; r < nrows; r += kWarps) {
+    // Eight lanes per row, one pass: every lane folds its share of the row's partials into a running
+    // pair (changes of reference are exact powers of two), then the eight lanes are folded together.
+    // (the loop bound is the same for all lanes of a warp: lanes beyond the last row run along with
+    // zero partials, because the shuffles below need the whole warp)
+    for (int r0 = 0; r0 < nrows; r0 += kThreads / 8) {
+        const int r = r0 + (tid >> 3);
+        const int sub = tid & 7;
         const bool is_t = r <= K;
-        const int nseg = is_t ? P.nst : P.nsd;
+        const int nseg = (r >= nrows) ? 0 : (is_t ? P.nst : P.nsd);
         const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
                                   : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
         if (greedy) {
             float best = -INFINITY; int idx = INT_MAX;
-            for (int i = lane; i < nseg; i += 32) {
+            for (int i = sub; i < nseg; i += 8) {
                 float2 pr = __ldcg(part + i);
                 int i2 = __float_as_int(pr.y);
                 if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
             }
 #pragma unroll
-            for (int o = 16; o > 0; o >>= 1) {
+            for (int o = 4; o > 0; o >>= 1) {
                 float b2 = __shfl_xor_sync(0xffffffffu, best, o);
                 int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
                 if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
             }
-            if (lane == 0) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
+            if (sub == 0 && r < nrows) { sm_c[r] = best; sm_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx); }
         } else {
             float c = kNegBig;
-            for (int i = lane; i < nseg; i += 32) c = fmaxf(c, __ldcg(part + i).x);
-            c = warp_max(c);
-            double s = 0.0;
-            for (int i = lane; i < nseg; i += 32) {
-                float2 pr = __ldcg(part + i);
-                s += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
+            double sum = 0.0;
+            for (int i = sub; i < nseg; i += 8) {
+                const float2 pr = __ldcg(part + i);
+                const float cn = fmaxf(c, pr.x);
+                sum = sum * pow2_neg_d(c - cn) + static_cast<double>(pr.y) * pow2_neg_d(pr.x - cn);
+                c = cn;
             }
-            s = warp_sum(s);
-            if (lane == 0) { sm_c[r] = c; sm_s[r] = s; }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                const float c2 = __shfl_xor_sync(0xffffffffu, c, o);
+                const double s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+                const float cn = fmaxf(c, c2);
+                sum = sum * pow2_neg_d(c - cn) + s2 * pow2_neg_d(c2 - cn);
+                c = cn;
+            }
+            if (sub == 0 && r < nrows) { sm_c[r] = c; sm_s[r] = sum; }
         }
     }
     __syncthreads();
