@@ -79,6 +79,7 @@ struct Params {
     double *stripsum;                   // fused kernel: [B][nct][kSWarps] weight sums in target-id order
     int nct, ncd;        // statistics-kernel chunks per target / drafter row
     int ntile;           // 16 KB tiles per target row (sampling pass)
+    int split_select;    // 1: the CDF inversions run as a kernel of their own
     int cps;             // chunks per segment
     int nst, nsd;        // segments per target / drafter row
 };
@@ -860,35 +861,20 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
     return tot;
 }
 
+// The CDF inversion for one sequence by one CTA, tile -> vector -> element, from the tile sums in
+// the workspace.  Either the last CTA of the sampling kernel to finish a tile of the sequence runs
+// it, or (large batches) the selection kernel does, one CTA per sequence.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
+__device__ void select_sequence(const Params &P, int b, RowSel sel, const RowView<DT> &rt, const void *zd_row) {
     constexpr int EPV = Elt<DT>::kPerVec;
     __shared__ double sm_red[kWarps];
     __shared__ double sm_tiles[kMaxTiles];
     __shared__ float sm_seg[kVecPerTile];
     __shared__ double sm_warp_tot[kWarps];
-    __shared__ int sm_last, sm_tile, sm_found, sm_lastpos, sm_retry;
+    __shared__ int sm_tile, sm_found, sm_lastpos, sm_retry;
     __shared__ double sm_rem;
-    const int b = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    RowSel sel = P.sel[b];
-    if (sel.mode == MODE_SKIP) return;
     const int ntile = P.ntile;
-    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
-    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
-        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
-
-    const double tot = tile_weight_sum<DT>(P, sel, rt, zd_row, tile, sm_red);
-    if (tid == 0) {
-        __stcg(P.tilesum + static_cast<size_t>(b) * ntile + tile, tot);
-        __threadfence();
-        const unsigned ticket = atomicAdd(P.cnt_sample + b, 1u);
-        sm_last = (ticket == static_cast<unsigned>(ntile) - 1);
-    }
-    __syncthreads();
-    if (!sm_last) return;
-    __threadfence();
-
     // ---- last CTA of the sequence: invert the CDF, tile -> vector -> element ----
     for (int i = tid; i < ntile; i += kThreads) sm_tiles[i] = __ldcg(P.tilesum + static_cast<size_t>(b) * ntile + i);
     __syncthreads();
@@ -921,7 +907,6 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
             if (tid == 0) {
                 P.next_token[b] = 0;
                 if (P.status) P.status[b] |= TLI_ROW_NONFINITE;
-                P.cnt_sample[b] = 0;
             }
             return;
         }
@@ -984,7 +969,7 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
     const int found = sm_found;
     const int G = (found != INT_MAX) ? found : sm_lastpos;
     if (G < 0) {                                   // cannot happen when the tile has positive mass
-        if (tid == 0) { P.next_token[b] = 0; P.cnt_sample[b] = 0; }
+        if (tid == 0) P.next_token[b] = 0;
         return;
     }
     if (tid == G / kVecPerThread) {
@@ -1011,8 +996,53 @@ __global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
         int token = rt.first_elem(v) + pick;
         token = min(max(token, 0), P.V_t - 1);
         P.next_token[b] = token;
-        P.cnt_sample[b] = 0;
     }
+}
+
+// The sampling pass: one CTA per 16 KB tile of the target row the extra token is drawn from
+// (blockIdx.y = sequence).  With P.split_select the kernel only leaves the tile sums; otherwise
+// the last CTA of a sequence (atomic ticket, nobody waits) goes on to invert the CDF.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
+    __shared__ double sm_red[kWarps];
+    __shared__ int sm_last;
+    const int b = blockIdx.y, tile = blockIdx.x;
+    const int tid = threadIdx.x;
+    const RowSel sel = P.sel[b];
+    if (sel.mode == MODE_SKIP) return;
+    const int ntile = P.ntile;
+    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
+        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
+
+    const double tot = tile_weight_sum<DT>(P, sel, rt, zd_row, tile, sm_red);
+    if (tid == 0) {
+        __stcg(P.tilesum + static_cast<size_t>(b) * ntile + tile, tot);
+        sm_last = 0;
+        if (!P.split_select) {
+            __threadfence();
+            const unsigned ticket = atomicAdd(P.cnt_sample + b, 1u);
+            sm_last = (ticket == static_cast<unsigned>(ntile) - 1);
+            if (sm_last) P.cnt_sample[b] = 0;
+        }
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+    select_sequence<DT>(P, b, sel, rt, zd_row);
+}
+
+// Large batches: the CDF inversions as a kernel of their own, one CTA per sequence, so that the
+// tile CTAs of the sampling kernel carry neither a fence nor a ticket.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
+    const int b = blockIdx.x;
+    const RowSel sel = P.sel[b];
+    if (sel.mode == MODE_SKIP) return;
+    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
+        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
+    select_sequence<DT>(P, b, sel, rt, zd_row);
 }
 
 // ---------------------------------------------------------------------------
@@ -1870,6 +1900,8 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.seq_state = reinterpret_cast<int *>(ctx->d_counters + 2 * (TLI_MAX_B + 1));
     P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
     P.seg_counter = P.error + 1; P.cta_done = P.error + 2; P.samp_counter = P.error + 3;
+    // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
+    P.split_select = (static_cast<long long>(a->B) * L.ntile >= 4096) ? 1 : 0;
     P.nct = L.nct; P.ncd = L.ncd; P.ntile = L.ntile; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
@@ -1911,6 +1943,12 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     else tli_sample_kernel<TLI_BF16><<<grid2, kThreads, 0, stream>>>(P);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
+    if (P.split_select) {
+        if (a->dtype == TLI_F32) tli_select_kernel<TLI_F32><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
+        else tli_select_kernel<TLI_BF16><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return cuda_fail(e, "launch tli_select_kernel");
+    }
     if (ev) cudaEventRecord(ev[3], stream);
     return TLI_OK;
 }
