@@ -1003,7 +1003,7 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
 // (blockIdx.y = sequence).  With P.split_select the kernel only leaves the tile sums; otherwise
 // the last CTA of a sequence (atomic ticket, nobody waits) goes on to invert the CDF.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) tli_sample_kernel(const Params P) {
+__global__ void __launch_bounds__(kThreads, 8) tli_sample_kernel(const Params P) {
     __shared__ double sm_red[kWarps];
     __shared__ int sm_last;
     const int b = blockIdx.y, tile = blockIdx.x;
