@@ -660,6 +660,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         sm_flags = fl;
     }
 
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     // Eight lanes per row, one pass: every lane folds its share of the row's partials into a running
     // pair (changes of reference are exact powers of two), then the eight lanes are folded together.
     // (the loop bound is the same for all lanes of a warp: lanes beyond the last row run along with
@@ -1008,6 +1009,7 @@ __global__ void __launch_bounds__(kThreads, 8) tli_sample_kernel(const Params P)
     __shared__ int sm_last;
     const int b = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const RowSel sel = P.sel[b];
     if (sel.mode == MODE_SKIP) return;
     const int ntile = P.ntile;
@@ -1037,6 +1039,7 @@ __global__ void __launch_bounds__(kThreads, 8) tli_sample_kernel(const Params P)
 template <int DT>
 __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
     const int b = blockIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const RowSel sel = P.sel[b];
     if (sel.mode == MODE_SKIP) return;
     RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
@@ -1934,19 +1937,28 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
 
-    if (a->dtype == TLI_F32) tli_decide_kernel<TLI_F32><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
-    else tli_decide_kernel<TLI_BF16><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
-    e = cudaGetLastError();
+    // The three small kernels are launched as programmatic dependents: none of their predecessors
+    // triggers early, so they still start only when the predecessor is done, but their launch is
+    // set up while it runs (4-6 us per call).  Each begins with griddepcontrol.wait.
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1; cfg.stream = stream; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0;
+    cfg.gridDim = dim3(static_cast<unsigned>(a->B));
+    if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_decide_kernel<TLI_F32>, P);
+    else e = cudaLaunchKernelEx(&cfg, tli_decide_kernel<TLI_BF16>, P);
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_decide_kernel");
     if (ev) cudaEventRecord(ev[2], stream);
-    if (a->dtype == TLI_F32) tli_sample_kernel<TLI_F32><<<grid2, kThreads, 0, stream>>>(P);
-    else tli_sample_kernel<TLI_BF16><<<grid2, kThreads, 0, stream>>>(P);
-    e = cudaGetLastError();
+    cfg.gridDim = grid2;
+    if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_F32>, P);
+    else e = cudaLaunchKernelEx(&cfg, tli_sample_kernel<TLI_BF16>, P);
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_sample_kernel");
     if (P.split_select) {
-        if (a->dtype == TLI_F32) tli_select_kernel<TLI_F32><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
-        else tli_select_kernel<TLI_BF16><<<static_cast<unsigned>(a->B), kThreads, 0, stream>>>(P);
-        e = cudaGetLastError();
+        cfg.gridDim = dim3(static_cast<unsigned>(a->B));
+        if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_select_kernel<TLI_F32>, P);
+        else e = cudaLaunchKernelEx(&cfg, tli_select_kernel<TLI_BF16>, P);
         if (e != cudaSuccess) return cuda_fail(e, "launch tli_select_kernel");
     }
     if (ev) cudaEventRecord(ev[3], stream);
