@@ -48,7 +48,7 @@ def algorithmic_bytes(cfg, batch) -> int:
 
 
 class ClockSampler:
-    """nvidia-smi clocks and throttle reasons of one GPU, sampled every 200 ms in the background."""
+    """nvidia-smi clocks and throttle reasons of one GPU, sampled every 50 ms in the background."""
 
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
@@ -63,7 +63,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
-                 "--format=csv,noheader,nounits", "-lms", "200"],
+                 "--format=csv,noheader,nounits", "-lms", "50"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             threading.Thread(target=self._read, daemon=True).start()
         except OSError:
@@ -152,6 +152,13 @@ def reference_arm(args):
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": used, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def kernels_per_call(cfg) -> int:
+    """statistics + decision + sampling, plus the separate selection kernel for large batches."""
+    epv = 4 if cfg.elt == 4 else 8
+    ntile = -(-(cfg.V_t + epv - 1) // (epv * 1024))
+    return 4 if cfg.B * ntile >= 4096 else 3
 
 
 def workload_config(cfg, l2_note):
@@ -326,7 +333,7 @@ def gpu_arm(args):
         "clocks": clocks,
         "e2e": {"value": world * cfg.positions / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": 3 * args.steps,
+        "gpu_launches": kernels_per_call(cfg) * args.steps,
         "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
         "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
