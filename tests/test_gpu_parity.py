@@ -278,3 +278,28 @@ def test_argument_errors_are_reported_not_launched():
     assert call(good()) == tli.TLI_OK
     torch.cuda.synchronize()
     v.close()
+
+
+def test_many_tiles_use_the_separate_selection_kernel():
+    """B x tiles >= 4096: the CDF inversions run as their own kernel; same results required."""
+    cfg = wl.tiny_config(B=300, K=1, V_t=60001, V_d=3000, dtype=wl.F32, f_mapped=0.5, sigma_d=0.7,
+                         temperatures=(0.8, 1.0), seed=81)
+    rep = check(wl.make_batch(cfg))
+    assert rep.rows == 300
+
+
+def test_profile_hook_reports_three_positive_durations_and_the_same_results():
+    cfg = wl.tiny_config(B=6, K=3, V_t=20000, V_d=15000, dtype=wl.BF16, f_mapped=0.5, seed=82)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    dev = to_device(batch)
+    ref = run_gpu(batch, v, dev)
+    acc = torch.full((6,), -1, dtype=torch.int32, device="cuda")
+    nxt = torch.full((6,), -1, dtype=torch.int32, device="cuda")
+    args = tli.make_args(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"], dev["temperature"],
+                         dev["uniforms"], acc, nxt, v.workspace(6, 3, tli.TLI_BF16))
+    ms = tli.tli_verify_profile(v.ctx, args)
+    assert len(ms) == 3 and all(m > 0 for m in ms)
+    np.testing.assert_array_equal(acc.cpu().numpy(), ref["accepted"])
+    np.testing.assert_array_equal(nxt.cpu().numpy(), ref["next_token"])
+    v.close()
