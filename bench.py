@@ -154,6 +154,18 @@ def reference_arm(args):
     }))
 
 
+def stats_kernel_traffic(cfg):
+    """DRAM bytes (read + write) of one tli_stats_kernel launch from the committed ncu capture
+    (profiles/stats_kernel_cfg3_b64_cfg2.md): cfg3 with B=64 moved 459 076 352 + 3 920 128 bytes;
+    traffic is proportional to B, so the full batch is 4 x that.  None for the other workloads and
+    to be set back to None whenever the kernel changes."""
+    if cfg.name == "cfg3" and cfg.B % 64 == 0:
+        return (459076352 + 3920128) * (cfg.B // 64)
+    if cfg.name == "cfg2" and cfg.B == 64:
+        return 208605696 + 4318464
+    return None
+
+
 def kernels_per_call(cfg) -> int:
     """statistics + decision + sampling, plus the separate selection kernel for large batches."""
     epv = 4 if cfg.elt == 4 else 8
@@ -339,7 +351,7 @@ def gpu_arm(args):
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
-                     "traffic": None, "algorithmic_bytes": case.bytes,
+                     "traffic": stats_kernel_traffic(cfg), "algorithmic_bytes": case.bytes,
                      "ms_stats_kernel": ms_stats, "ms_decide_kernel": ms_decide,
                      "ms_sample_kernel": ms_sample},
     }
