@@ -202,6 +202,18 @@ int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_str
  */
 int tli_set_fused(tli_ctx *ctx, int enabled);
 
+/*
+ * Self-test of the kernels' bounded waits.  Every wait inside the kernels (on a
+ * shared-memory barrier that a bulk copy or another warp completes) gives up
+ * after a fixed number of polls, records the fact and lets the kernel finish;
+ * rows decided afterwards carry TLI_ROW_TIMEOUT.  This call runs a one-thread
+ * kernel that waits, with the same code and a limit of `polls` (1 .. 2^22), on
+ * a barrier nothing will ever complete, synchronises the stream and reports
+ * through [host] gave_up whether the wait ended the way it must (1).  It does
+ * not touch the context's sticky error word; the context stays usable.
+ */
+int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up);
+
 /* Vocabulary sizes and number of mapped drafter ids of a context. */
 int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped);
 

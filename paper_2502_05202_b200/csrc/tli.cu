@@ -240,9 +240,10 @@ __device__ __forceinline__ bool mbar_test(uint64_t *bar, unsigned parity) {
 // Bounded wait: gives up after kWaitLimit polls, records the fact and lets the caller go on
 // (results of that call are then flagged, never trusted).  Returns false on timeout.
 constexpr unsigned kWaitLimit = 1u << 22;
-__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, unsigned parity, int *sm_error, unsigned *g_error) {
+__device__ __noinline__ bool mbar_wait_slow(uint64_t *bar, unsigned parity, int *sm_error, unsigned *g_error,
+                                            unsigned limit = kWaitLimit) {
     if (*reinterpret_cast<volatile int *>(sm_error)) return false;
-    for (unsigned i = 0; i < kWaitLimit; ++i) {
+    for (unsigned i = 0; i < limit; ++i) {
         if (mbar_test(bar, parity)) return true;
         if (i > 64) __nanosleep(64);
     }
@@ -1706,6 +1707,21 @@ __global__ void __launch_bounds__(kFThreads, kCtasPerSm) tli_fused_kernel(const 
     }
 }
 
+// Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete,
+// with a caller-chosen poll limit, and reports how the wait ended.  The kernel returns normally.
+__global__ void tli_bounded_wait_kernel(unsigned limit, int *result, unsigned *scratch_error) {
+    __shared__ uint64_t bar;
+    __shared__ int sm_error;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1);
+        sm_error = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const bool completed = mbar_wait_slow(&bar, 0u, &sm_error, scratch_error, limit);
+        result[0] = completed ? 0 : 1;              // 1: gave up, as it must
+        result[1] = sm_error;                       // 1: the CTA-wide error flag was raised
+    }
+}
+
 // ---------------------------------------------------------------------------
 // host side
 // ---------------------------------------------------------------------------
@@ -1772,7 +1788,7 @@ struct tli_ctx {
     int *d_inv;
     uint32_t *d_mask;
     int fused;                  // option: one fused kernel (default) or three kernels
-    unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 4], zero between calls: tickets, tickets, sequence states,
+    unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
 };
@@ -1826,11 +1842,11 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
-        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 4))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
         if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
         if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
         if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
-        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 4))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
+        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
     } while (0);
     if (rc != TLI_OK) {
         cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
@@ -1967,6 +1983,23 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
 
 int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     return verify_impl(ctx, a, cuda_stream, nullptr);
+}
+
+int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up) {
+    if (!ctx || !gave_up || polls == 0 || polls > kWaitLimit) return TLI_ERR_ARG;
+    // scratch: the two unused words after the schedulers' counters, so the sticky error word stays clean
+    int *d_result = reinterpret_cast<int *>(ctx->d_counters + 3 * (TLI_MAX_B + 1) + 4);
+    unsigned *d_err = ctx->d_counters + 3 * (TLI_MAX_B + 1) + 6;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = cudaMemsetAsync(d_result, 0, 3 * sizeof(int), stream);
+    if (e != cudaSuccess) return cuda_fail(e, "cudaMemsetAsync");
+    tli_bounded_wait_kernel<<<1, 32, 0, stream>>>(polls, d_result, d_err);
+    if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail(e, "launch tli_bounded_wait_kernel");
+    int h[3] = {0, 0, 0};
+    if ((e = cudaMemcpyAsync(h, d_result, sizeof h, cudaMemcpyDeviceToHost, stream)) != cudaSuccess) return cuda_fail(e, "cudaMemcpyAsync");
+    if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
+    *gave_up = (h[0] == 1 && h[1] == 1) ? 1 : 0;
+    return TLI_OK;
 }
 
 int tli_set_fused(tli_ctx *ctx, int enabled) {

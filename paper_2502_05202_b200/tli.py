@@ -37,7 +37,7 @@ TLI_MAX_K = 64
 TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -89,6 +89,8 @@ def load() -> ctypes.CDLL:
         lib.tli_verify_profile.restype = ctypes.c_int
         lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_fused.restype = ctypes.c_int
+        lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
+        lib.tli_selftest_bounded_wait.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
         lib.tli_ctx_info.restype = ctypes.c_int
         lib.tli_status_string.argtypes = [ctypes.c_int]
@@ -198,6 +200,17 @@ def tli_set_fused(ctx: int, enabled: bool) -> None:
     rc = load().tli_set_fused(ctx, 1 if enabled else 0)
     if rc != TLI_OK:
         raise TLIError(rc, "tli_set_fused")
+
+
+def tli_selftest_bounded_wait(ctx: int, polls: int = 2000, stream: Optional[int] = None) -> bool:
+    """tli_selftest_bounded_wait(): True if a wait on a barrier nothing completes gave up after `polls` polls."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    out = ctypes.c_int(0)
+    rc = load().tli_selftest_bounded_wait(ctx, ctypes.c_void_p(stream), polls, ctypes.byref(out))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_selftest_bounded_wait")
+    return out.value == 1
 
 
 class Verifier:

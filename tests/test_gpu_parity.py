@@ -303,3 +303,19 @@ def test_profile_hook_reports_three_positive_durations_and_the_same_results():
     np.testing.assert_array_equal(acc.cpu().numpy(), ref["accepted"])
     np.testing.assert_array_equal(nxt.cpu().numpy(), ref["next_token"])
     v.close()
+
+
+def test_a_wait_that_nothing_completes_gives_up_and_leaves_the_context_usable():
+    """The kernels' waits are bounded: run the same wait code on a barrier nobody will complete."""
+    cfg = wl.tiny_config(B=3, K=2, V_t=9000, V_d=7000, dtype=wl.F32, f_mapped=0.5, seed=83)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    before = run_gpu(batch, v)
+    assert tli.tli_selftest_bounded_wait(v.ctx, polls=2000)
+    after = run_gpu(batch, v)
+    for k in before:
+        np.testing.assert_array_equal(before[k], after[k])
+    assert (after["row_status"] & tli.TLI_ROW_TIMEOUT == 0).all()     # the self-test keeps its own error word
+    with pytest.raises(tli.TLIError):
+        tli.tli_selftest_bounded_wait(v.ctx, polls=0)
+    v.close()
