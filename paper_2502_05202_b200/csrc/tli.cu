@@ -1,26 +1,28 @@
 // TLI verification for sm_100a: kernels and the C ABI declared in include/tli.h.
 //
-// Three launches per call; the first and the last stream logits and are HBM-bound (no dense
-// contraction, hence no tensor cores):
+// A call is three launches (four for large batches).  The first and the third stream logits and
+// are HBM-bound; there is no dense contraction on this path, hence no tensor cores.
 //
-//   tli_stats_kernel   persistent grid (two CTAs per SM); each CTA streams 16 KB chunks of
-//                      logit rows through a cp.async.bulk / mbarrier ring.  Target rows:
-//                      (reference, sum of 2^(z*s - reference)) with s = log2(e)/tau;
-//                      drafter rows: the same over ids inside the intersection
-//                      only (Algorithm 4's renormalisation: the full-softmax
-//                      denominator cancels in q' = q / sum_{T cap D} q);
-//                      temperature-0 rows: (max, lowest index).  The last CTA to
-//                      finish a sequence (atomic ticket, nobody waits) combines
-//                      the partials in fp64, runs Algorithm 5's acceptance tests
-//                      and first-rejection count, and records which row the
-//                      extra token is drawn from.
-//   tli_sample_kernel  one CTA per 16 KB tile of that one target row: tile sums
-//                      of max(0, p - q'_T) (or of p for the bonus row); the last
-//                      CTA of a sequence walks tile -> 16-byte vector -> element
-//                      to invert the CDF.
+//   tli_stats_kernel   persistent grid, two CTAs per SM, each one producer warp and sixteen
+//                      consumer warps around a 96 KB ring of shared-memory stages filled by
+//                      cp.async.bulk with mbarrier completion.  Target rows: (reference, sum of
+//                      2^(z*s - reference)) with s = log2(e)/tau; drafter rows: the same over ids
+//                      inside the intersection only (Algorithm 4's renormalisation: the
+//                      full-softmax denominator cancels in q' = q / sum_{T cap D} q);
+//                      temperature-0 rows: (max, lowest index).  One pair per segment of a row
+//                      goes to the workspace.
+//   tli_decide_kernel  one CTA per sequence: fp64 combination of the pairs, Algorithm 5's
+//                      acceptance tests and count of accepted drafts, which row the extra token
+//                      is drawn from.
+//   tli_sample_kernel  one CTA per 16 KB tile of that one target row: tile sums of
+//                      max(0, p - q'_T) (or of p for the bonus row); the last CTA of a sequence
+//                      walks tile -> 16-byte vector -> element to invert the CDF.
+//   tli_select_kernel  large batches only: those inversions as a kernel of their own.
+//   tli_fused_kernel   all of the above in one persistent grid (tli_set_fused; not the default).
 //
-// Softmax terms are formed as ex2(fma(z, s, -c)) with a per-warp reference c in
-// log2 units, so the only per-term rounding is the one in the fma.
+// Softmax terms are formed as ex2(fma(z, s, -c)) with an integer-valued reference c in log2
+// units: the only per-term rounding is the one in the fma, and every change or combination of
+// references is an exact power of two.
 
 #include <cuda_runtime.h>
 #include <float.h>
