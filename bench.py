@@ -385,7 +385,7 @@ def gpu_arm(args):
         out["per_config"] = per
 
     if rank == 0 and world == 1 and not args.kernels_only:
-        v, cores, reps, secs = time_oracle(headline_batch, cfg.positions)
+        v, cores, reps, secs = time_oracle(headline_batch, cfg.positions, min_seconds=args.cpu_seconds)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
                                "sample": "all %d sequences of %s, %d repetitions in %.1f s" % (cfg.B, cfg.name, reps, secs)}
     if rank == 0:
@@ -403,6 +403,7 @@ def main():
     ap.add_argument("--config", default="cfg3")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-config", action="store_true", help="skip the four other workloads")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time given to the oracle baseline leg")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's B (profiling on a smaller case)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the device-timed loop: no per-config, end-to-end or CPU legs (for profiler runs)")
