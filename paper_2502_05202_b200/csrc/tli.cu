@@ -1765,6 +1765,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.ntile = chunks_per_row(V_t, dtype, kVecPerTile);
     const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
     long long cps = chunks / (ctas * 4);
+    if (chunks <= ctas * 16) cps = (chunks + ctas - 1) / ctas;      // small batch: about one segment per CTA
     L.cps = static_cast<int>(cps < 1 ? 1 : (cps > 16 ? 16 : cps));
     L.nst = (L.nct + L.cps - 1) / L.cps;
     L.nsd = (L.ncd + L.cps - 1) / L.cps;
