@@ -121,6 +121,25 @@ def time_oracle(batch, positions, min_seconds=10.0, max_reps=50):
     return positions * reps / dt, min(cores, len(batch["temperature"])), reps, dt
 
 
+def time_oracle_single_thread(batch, K, rows=8, min_seconds=2.0, max_reps=20):
+    """The oracle on one thread, on the first few sequences; returns (positions/s, sequences used)."""
+    import oracle
+    rows = min(rows, len(batch["temperature"]))
+    sub = {k: (v if k == "id_map" else v[:rows]) for k, v in batch.items()
+           if k in ("target_logits", "drafter_logits", "id_map", "draft_ids", "temperature", "uniforms")}
+    run = lambda: oracle.verify(sub["target_logits"], sub["drafter_logits"], sub["id_map"], sub["draft_ids"],
+                                sub["temperature"], sub["uniforms"], threads=1)
+    t0 = time.perf_counter()
+    reps = 0
+    while True:
+        run()
+        reps += 1
+        dt = time.perf_counter() - t0
+        if dt >= min_seconds or reps >= max_reps:
+            break
+    return rows * K * reps / dt, rows
+
+
 def reference_arm(args):
     """`--impl reference`: the CPU oracle on the same workload, rank 0 only."""
     if int(os.environ.get("RANK", "0")) != 0:
@@ -243,6 +262,31 @@ class GpuCase:
         self.tli.tli_verify(self.ver.ctx, self.args[0], self.stream)
         h["out"].copy_(self.out, non_blocking=True)
 
+    def make_graph(self):
+        """One CUDA graph holding a tli_verify() call on every input copy; returns (graph, calls in it)."""
+        torch = self.torch
+        side = torch.cuda.Stream()
+        side.wait_stream(torch.cuda.current_stream())
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            h = torch.cuda.current_stream().cuda_stream
+            for i in range(self.copies):
+                self.tli.tli_verify(self.ver.ctx, self.args[i], h)
+        torch.cuda.current_stream().wait_stream(side)
+        return g, self.copies
+
+    def per_call_ms(self, calls):
+        """Events around single calls: (median, min) ms."""
+        torch = self.torch
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(calls)]
+        for a, b in ev:
+            a.record()
+            self.step()
+            b.record()
+        torch.cuda.synchronize()
+        t = [a.elapsed_time(b) for a, b in ev]
+        return statistics.median(t), min(t)
+
     def e2e_bytes(self):
         h = self.host
         h2d = sum(h[k].numel() * h[k].element_size() for k in ("zt", "zd", "draft", "tau", "u"))
@@ -289,6 +333,18 @@ def timed(torch, dist, steps, fn, world):
     return ms
 
 
+def call_timings(case, torch, steps):
+    """Per-call figures beside the K-step loop: events around single calls, and a CUDA-graph replay."""
+    med, mn = case.per_call_ms(min(max(steps, 20), 200))
+    g, n = case.make_graph()
+    reps = max(3, -(-steps // n))
+    for _ in range(2):
+        g.replay()
+    ms = timed(torch, None, reps, g.replay, 1) / (reps * n)
+    del g
+    return {"ms_call_median": med, "ms_call_min": mn, "ms_call_graph_replay": ms}
+
+
 def gpu_arm(args):
     import torch
     from paper_2502_05202_b200 import tli, workload as wl
@@ -323,6 +379,7 @@ def gpu_arm(args):
     # the dominant kernel alone, with events around it, on the same stream and workload
     case.profile(3)
     ms_stats, ms_decide, ms_sample = case.profile(args.steps)
+    calls = call_timings(case, torch, args.steps)
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
@@ -348,6 +405,7 @@ def gpu_arm(args):
         "gpu_launches": kernels_per_call(cfg) * args.steps,
         "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
         "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
+        "per_call": calls,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
@@ -366,7 +424,7 @@ def gpu_arm(args):
             if c.name == cfg.name:
                 per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
                             "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
-                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample})
+                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls})
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
@@ -375,10 +433,11 @@ def gpu_arm(args):
             m = timed(torch, None, steps, k.step, 1) / steps
             k.profile(3)
             a, d, b = k.profile(min(steps, 50))
+            kc = call_timings(k, torch, steps)
             k.check()
             per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
                         "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
-                        "ms_stats_kernel": a, "ms_decide_kernel": d, "ms_sample_kernel": b, "l2": k.l2_note})
+                        "ms_stats_kernel": a, "ms_decide_kernel": d, "ms_sample_kernel": b, "l2": k.l2_note, **kc})
             k.close()
             del k
             torch.cuda.empty_cache()
@@ -386,8 +445,11 @@ def gpu_arm(args):
 
     if rank == 0 and world == 1 and not args.kernels_only:
         v, cores, reps, secs = time_oracle(headline_batch, cfg.positions, min_seconds=args.cpu_seconds)
+        v1, rows1 = time_oracle_single_thread(headline_batch, cfg.K)
         out["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
-                               "sample": "all %d sequences of %s, %d repetitions in %.1f s" % (cfg.B, cfg.name, reps, secs)}
+                               "sample": "all %d sequences of %s, %d repetitions in %.1f s" % (cfg.B, cfg.name, reps, secs),
+                               "single_thread_value": v1,
+                               "single_thread_sample": "first %d sequences of %s on one thread" % (rows1, cfg.name)}
     if rank == 0:
         print(json.dumps(out))
     if world > 1:

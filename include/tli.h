@@ -13,7 +13,10 @@
  *     library never frees or reallocates them.  Pointers marked [host] are
  *     read during the call only.
  *   - tli_verify() is asynchronous on the stream it is given, allocates
- *     nothing and does not synchronise.
+ *     nothing and does not synchronise.  It only launches kernels, so it may
+ *     be recorded into a CUDA graph by stream capture and replayed; calls on
+ *     one context must not overlap in time (they share the context's
+ *     counters), so replays of such a graph are serialised by the caller.
  *   - Functions return TLI_OK or a negative tli error code.  Errors in the
  *     data (a draft id outside the vocabulary, a NaN logit, a negative
  *     temperature) never fault: they set bits in row_status.

@@ -305,6 +305,38 @@ def test_profile_hook_reports_three_positive_durations_and_the_same_results():
     v.close()
 
 
+def test_calls_recorded_in_a_cuda_graph_replay_to_the_same_results():
+    """tli_verify() only launches kernels: captured into a graph (two calls, two dtypes of batch) and replayed."""
+    cfg = wl.tiny_config(B=9, K=4, V_t=70001, V_d=33000, dtype=wl.F32, f_mapped=0.6, temperatures=(0.0, 0.7, 1.0), seed=84)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    dev = to_device(batch)
+    ref = run_gpu(batch, v, dev)
+    outs = [{k: torch.full((9,), -7, dtype=torch.int32, device="cuda") for k in ("acc", "nxt", "st")} for _ in range(2)]
+    ws = v.workspace(9, 4, tli.TLI_F32)
+    args = [tli.make_args(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"], dev["temperature"],
+                          dev["uniforms"], o["acc"], o["nxt"], ws, o["st"]) for o in outs]
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        for a in args:
+            tli.tli_verify(v.ctx, a, torch.cuda.current_stream().cuda_stream)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        for o in outs:
+            for t in o.values():
+                t.fill_(-7)
+        g.replay()
+        torch.cuda.synchronize()
+        for o in outs:
+            np.testing.assert_array_equal(o["acc"].cpu().numpy(), ref["accepted"])
+            np.testing.assert_array_equal(o["nxt"].cpu().numpy(), ref["next_token"])
+            np.testing.assert_array_equal(o["st"].cpu().numpy(), ref["row_status"])
+    del g
+    v.close()
+
+
 def test_a_wait_that_nothing_completes_gives_up_and_leaves_the_context_usable():
     """The kernels' waits are bounded: run the same wait code on a barrier nobody will complete."""
     cfg = wl.tiny_config(B=3, K=2, V_t=9000, V_d=7000, dtype=wl.F32, f_mapped=0.5, seed=83)
