@@ -362,6 +362,26 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
     return d;
 }
 
+// bf16 vectors of a drafter row: the elements whose mask bit is 0 become -inf, two at a time.
+// The low eight bits of `bits` go to the top bits of eight bytes (a multiplication by four
+// shifted ones, four bits per word), prmt's sign replication widens each to a 16-bit lane mask.
+__device__ __forceinline__ uint32_t prmt_sign(uint32_t a, uint32_t sel) {
+    uint32_t d;
+    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(0u), "r"(sel));
+    return d;
+}
+__device__ __forceinline__ uint32_t keep_or_neg_inf(uint32_t w, uint32_t lanes) {
+    return (w & lanes) | (~lanes & Elt<TLI_BF16>::kNegInfWord);
+}
+__device__ __forceinline__ void mask_bf16_vector(uint4 &r, uint32_t bits) {
+    const uint32_t lo = (bits & 0xfu) * 0x10204080u;           // bit i -> top bit of byte i
+    const uint32_t hi = ((bits >> 4) & 0xfu) * 0x10204080u;
+    r.x = keep_or_neg_inf(r.x, prmt_sign(lo, 0x9988u));        // bytes 0,0,1,1 of lo, sign-replicated
+    r.y = keep_or_neg_inf(r.y, prmt_sign(lo, 0xbbaau));        // bytes 2,2,3,3
+    r.z = keep_or_neg_inf(r.z, prmt_sign(hi, 0x9988u));
+    r.w = keep_or_neg_inf(r.w, prmt_sign(hi, 0xbbaau));
+}
+
 // One chunk of a softmax row into this thread's running (reference, sum).
 template <int DT, int CV, bool MASKED>
 __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint32_t (&bits)[CV], float s,
@@ -528,6 +548,15 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
             }
             const int chunk = meta.chunk;
+            uint32_t bits[CV] = {};
+            if (masked) {                                  // the mask words travel while the stage is read
+                const int nvec = rv.nvec();
+#pragma unroll
+                for (int q = 0; q < CV; ++q) {
+                    const int v = chunk * CVEC + q * kSThreads + tid;
+                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
+                }
+            }
             uint4 raw[CV];
             load_chunk<DT, CV>(rv, chunk, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
             __syncwarp();
@@ -535,16 +564,14 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             if (greedy) {
                 argmax_chunk<DT, CV>(raw, rv, chunk, tid, best, best_idx);
             } else if (masked) {
-                uint32_t bits[CV];
-                const int nvec = rv.nvec();
+                if constexpr (DT == TLI_BF16) {               // mask the packed words, then as a target row
 #pragma unroll
-                for (int q = 0; q < CV; ++q) {
-                    const int v = chunk * CVEC + q * kSThreads + tid;
-                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
+                    for (int q = 0; q < CV; ++q) mask_bf16_vector(raw[q], bits[q]);
+                    softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
+                } else {
+                    softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
                 }
-                softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
             } else {
-                const uint32_t bits[CV] = {};
                 softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
             }
             if (!(meta.flags & META_LAST)) continue;
@@ -1633,7 +1660,13 @@ __global__ void __launch_bounds__(kFThreads, kCtasPerSm) tli_fused_kernel(const 
                     const int v = chunk * CVEC + q * kSThreads + tid;
                     bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
                 }
-                softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
+                if constexpr (DT == TLI_BF16) {               // mask the packed words, then as a target row
+#pragma unroll
+                    for (int q = 0; q < CV; ++q) mask_bf16_vector(raw[q], bits[q]);
+                    softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
+                } else {
+                    softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
+                }
             } else {
                 const uint32_t bits[CV] = {};
                 softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
