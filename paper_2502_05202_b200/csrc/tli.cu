@@ -261,6 +261,11 @@ __device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned b
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
 }
+__device__ __forceinline__ float2 ld_shared_pair(const float2 *p) {     // a pair another warp wrote: not from a register copy
+    float2 v;
+    asm volatile("ld.volatile.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(smem_addr(p)) : "memory");
+    return v;
+}
 __device__ __forceinline__ void consumer_sync() {            // the consumer warps only
     asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory");
 }
@@ -323,11 +328,26 @@ struct StageMeta {
 };
 enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_INTERIOR = 16 };
 
+// The statistics kernel's label also carries the decoded segment, so that only the producer
+// thread divides segment numbers and reads temperatures.
+struct __align__(16) StatsMeta {
+    int chunk, flags;
+    int b, row;       // as in Segment
+    int seg;
+    float tau;
+    int pad[2];
+};
+
+// Per-warp results of a segment wait in one of kMaxStages + 1 slots (slot = the CTA's segment
+// count modulo that): a warp can be at most a ring of chunks, hence at most kMaxStages segment
+// ends, ahead of the warp that is still combining a slot, so no slot is rewritten while in use.
+constexpr int kPairSlots = kMaxStages + 1;
 struct StatsSmem {
     uint64_t full[kMaxStages];
     uint64_t empty[kMaxStages];
-    StageMeta meta[kMaxStages];
-    float2 pairs[2][kSWarps];     // alternate per segment: one barrier per segment is enough
+    StatsMeta meta[kMaxStages];
+    float2 pairs[kPairSlots][kSWarps];
+    unsigned arrived[kPairSlots];
     int error;
 };
 
@@ -462,6 +482,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
     if (threadIdx.x == 0) {
 #pragma unroll
         for (int i = 0; i < NST; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
+        for (int i = 0; i < kPairSlots; ++i) sm.arrived[i] = 0u;
         sm.error = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -490,9 +511,12 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     int v0, v1;
                     full_vectors<DT>(rv, chunk, CVEC, v0, v1);
                     const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
-                    sm.meta[st].id = id; sm.meta[st].chunk = chunk;
-                    sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
-                                        (interior ? META_INTERIOR : 0);
+                    StatsMeta mt;
+                    mt.chunk = chunk;
+                    mt.flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
+                               (interior ? META_INTERIOR : 0);
+                    mt.b = g.b; mt.row = g.row; mt.seg = g.seg; mt.tau = g.tau; mt.pad[0] = mt.pad[1] = 0;
+                    sm.meta[st] = mt;
                     const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
                     mbar_arrive_expect_tx(&sm.full[st], bytes);
                     if (bytes)
@@ -504,7 +528,9 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             }
             if (ok) {                                    // tell the consumers there is nothing more
                 if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
-                    sm.meta[st].id = -1; sm.meta[st].chunk = 0; sm.meta[st].flags = META_END;
+                    StatsMeta mt;
+                    mt.chunk = 0; mt.flags = META_END; mt.b = 0; mt.row = 0; mt.seg = 0; mt.tau = 1.f; mt.pad[0] = mt.pad[1] = 0;
+                    sm.meta[st] = mt;
                     mbar_arrive(&sm.full[st]);
                 }
             }
@@ -530,17 +556,17 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
         float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
         bool clean_exit = false;
-        unsigned seg_parity = 0;
+        unsigned slot = 0;                                 // where this segment's per-warp results meet
         unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
         for (;;) {
             if (!mbar_wait(&sm.full[st], par, &sm.error, P.error)) break;
-            const StageMeta meta = sm.meta[st];
+            const StatsMeta meta = sm.meta[st];
             const uint4 *stage = stage_base + static_cast<size_t>(st) * CVEC;
             uint64_t *empty_bar = &sm.empty[st];
             if (++st == NST) { st = 0; par ^= 1u; }
             if (meta.flags & META_END) { clean_exit = true; break; }
             if (meta.flags & META_FIRST) {
-                g = decode_segment(P, meta.id);
+                g.b = meta.b; g.row = meta.row; g.seg = meta.seg; g.tau = meta.tau;
                 rv = segment_row<DT>(P, g);
                 greedy = (g.tau == 0.f);
                 masked = g.row > P.K;
@@ -594,14 +620,23 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 for (int o = 16; o > 0; o >>= 1) a_w += __shfl_xor_sync(0xffffffffu, a_w, o);
                 px = c_w; py = a_w;
             }
-            float2 *pairs = sm.pairs[seg_parity];
-            seg_parity ^= 1u;
-            if (lane == 0) pairs[warp] = make_float2(px, py);
-            consumer_sync();
-            if (warp == 0) {
+            // the last warp to arrive combines the sixteen results, always in warp order
+            float2 *pairs = sm.pairs[slot];
+            unsigned *arrived = &sm.arrived[slot];
+            if (++slot == kPairSlots) slot = 0;
+            unsigned ticket = 0;
+            if (lane == 0) {
+                pairs[warp] = make_float2(px, py);
+                __threadfence_block();
+                ticket = atomicAdd(arrived, 1u);
+            }
+            ticket = __shfl_sync(0xffffffffu, ticket, 0);
+            if (ticket == kSWarps - 1) {
+                if (lane == 0) *arrived = 0u;
+                __threadfence_block();
                 float2 pr;
                 if (greedy) {
-                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
+                    pr = (lane < kSWarps) ? ld_shared_pair(pairs + lane) : make_float2(-INFINITY, __int_as_float(INT_MAX));
                     float bb = pr.x; int ii = __float_as_int(pr.y);
 #pragma unroll
                     for (int o = 16; o > 0; o >>= 1) {
@@ -611,7 +646,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     }
                     pr = make_float2(bb, __int_as_float(ii));
                 } else {
-                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(kNegBig, 0.f);
+                    pr = (lane < kSWarps) ? ld_shared_pair(pairs + lane) : make_float2(kNegBig, 0.f);
                     const float c_all = warp_max(pr.x);
                     float a_all = pr.y * pow2_neg(pr.x - c_all);
 #pragma unroll
