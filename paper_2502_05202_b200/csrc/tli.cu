@@ -1819,7 +1819,7 @@ struct Layout {
 
 // Chunk size: as large as leaves every CTA of the persistent grid (two per SM) at least ~16 chunks.
 // Segment size: about four segments per CTA (they are handed out dynamically, so that is enough to
-// balance the tail) and long enough to amortise the per-segment reduction.
+// balance the tail), long enough to amortise the per-segment reduction, at most 128 KB.
 Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     Layout L;
     const long long elt = dtype == TLI_F32 ? 4 : 2;
@@ -1834,7 +1834,8 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
     long long cps = chunks / (ctas * 4);
     if (chunks <= ctas * 16) cps = (chunks + ctas - 1) / ctas;      // small batch: about one segment per CTA
-    L.cps = static_cast<int>(cps < 1 ? 1 : (cps > 16 ? 16 : cps));
+    const long long cap = 16 / L.cv;                                 // 128 KB: longer segments interleave rows worse
+    L.cps = static_cast<int>(cps < 1 ? 1 : (cps > cap ? cap : cps));
     L.nst = (L.nct + L.cps - 1) / L.cps;
     L.nsd = (L.ncd + L.cps - 1) / L.cps;
     const long long nseg = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nst + static_cast<long long>(K) * L.nsd);
