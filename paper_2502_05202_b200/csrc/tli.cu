@@ -1817,7 +1817,8 @@ struct Layout {
     unsigned grid;
 };
 
-// Chunk size: as large as leaves every CTA of the persistent grid (two per SM) at least ~16 chunks.
+// Chunk size: as large as leaves every CTA of the persistent grid (two per SM) about one chunk
+// (measured: the per-chunk bookkeeping costs more than a few idle CTAs do).
 // Segment size: about four segments per CTA (they are handed out dynamically, so that is enough to
 // balance the tail), long enough to amortise the per-segment reduction, at most 128 KB.
 Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
@@ -1826,8 +1827,8 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     const long long bytes = elt * B * (static_cast<long long>(K + 1) * V_t + static_cast<long long>(K) * V_d);
     const long long ctas = static_cast<long long>(kCtasPerSm) * num_sms;
     L.cv = 1;
-    if (bytes >= ctas * 16 * (kSThreads * 2 * 16)) L.cv = 2;
-    if (bytes >= ctas * 16 * (kSThreads * 4 * 16)) L.cv = 4;
+    if (bytes >= ctas * (kSThreads * 2 * 16)) L.cv = 2;
+    if (bytes >= ctas * (kSThreads * 4 * 16)) L.cv = 4;
     L.nct = chunks_per_row(V_t, dtype, kSThreads * L.cv);
     L.ncd = chunks_per_row(V_d, dtype, kSThreads * L.cv);
     L.ntile = chunks_per_row(V_t, dtype, kVecPerTile);
