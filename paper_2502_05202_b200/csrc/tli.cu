@@ -376,6 +376,27 @@ __device__ __forceinline__ void load_chunk(const RowView<DT> &rv, int chunk, boo
     }
 }
 
+// Two fp32 lanes in one 64-bit register: the packed fma / add of sm_100, each lane rounded as the
+// scalar instruction would.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float &lo, float &hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+    uint64_t d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
 __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
     uint32_t d;
     asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
@@ -435,19 +456,28 @@ __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint
         acc *= pow2_neg(c_run - c_new);
         c_run = c_new;
     }
-    const float nc = -c_run;
-    float a4[4] = {0.f, 0.f, 0.f, 0.f};
+    // four running sums (elements i, i+4, i+8, ... each), two to a packed register
+    const uint64_t s2 = pack2(s, s), nc2 = pack2(-c_run, -c_run);
+    uint64_t a2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
     for (int q = 0; q < CV; ++q) {
         float z[EPV];
         unpack<DT>(raw[q], z);
 #pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-            if (MASKED) z[i] = ((bits[q] >> i) & 1u) ? z[i] : -INFINITY;
-            a4[i & 3] += ex2(fmaf(z[i], s, nc));
+        for (int i = 0; i < EPV; i += 2) {
+            if (MASKED) {
+                z[i] = ((bits[q] >> i) & 1u) ? z[i] : -INFINITY;
+                z[i + 1] = ((bits[q] >> (i + 1)) & 1u) ? z[i + 1] : -INFINITY;
+            }
+            float x0, x1;
+            unpack2(fma2(pack2(z[i], z[i + 1]), s2, nc2), x0, x1);
+            a2[(i >> 1) & 1] = add2(a2[(i >> 1) & 1], pack2(ex2(x0), ex2(x1)));
         }
     }
-    acc += (a4[0] + a4[1]) + (a4[2] + a4[3]);
+    float a0, a1, a3, a4;
+    unpack2(a2[0], a0, a1);
+    unpack2(a2[1], a3, a4);
+    acc += (a0 + a1) + (a3 + a4);
 }
 
 template <int DT, int CV>
