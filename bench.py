@@ -175,13 +175,13 @@ def reference_arm(args):
 
 def stats_kernel_traffic(cfg):
     """DRAM bytes (read + write) of one tli_stats_kernel launch from the committed ncu capture
-    (profiles/stats_kernel_cfg3_b64_cfg2.md): cfg3 with B=64 moved 459 076 352 + 3 920 128 bytes;
+    (profiles/stats_kernel_cfg3_b64_cfg2.md): cfg3 with B=64 moved 459 066 112 + 4 182 016 bytes;
     traffic is proportional to B, so the full batch is 4 x that.  None for the other workloads and
     to be set back to None whenever the kernel changes."""
     if cfg.name == "cfg3" and cfg.B % 64 == 0:
-        return (459076352 + 3920128) * (cfg.B // 64)
+        return (459066112 + 4182016) * (cfg.B // 64)
     if cfg.name == "cfg2" and cfg.B == 64:
-        return 208605696 + 4318464
+        return 207997952 + 3759872
     return None
 
 
