@@ -1,7 +1,8 @@
 """TEST INFRASTRUCTURE -- not part of the product path.
 
 ctypes front end of the fp64 CPU oracle in ``tli_oracle.c`` (Algorithms 4 and 5
-of the paper).  Only tests, the smoke check and the benchmark's CPU-baseline
+of the paper: ``verify`` for the verification half, ``draft`` for drawing the
+draft ids from q').  Only tests, the smoke check and the benchmark's CPU-baseline
 legs may import this package; the CUDA library never does, and this package
 imports nothing from it.
 """
@@ -46,6 +47,18 @@ class _Args(ctypes.Structure):
     ]
 
 
+class _DraftArgs(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("R", ctypes.c_int32), ("V_d", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_r", ctypes.c_int64),
+        ("id_map", ctypes.c_void_p), ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("probe_id", ctypes.c_void_p),
+        ("draft_ids", ctypes.c_void_p), ("flags", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
+        ("cdf_lo", ctypes.c_void_p), ("cdf_hi", ctypes.c_void_p),
+        ("probe_lo", ctypes.c_void_p), ("probe_hi", ctypes.c_void_p), ("probe_w", ctypes.c_void_p),
+    ]
+
+
 def build(force: bool = False) -> str:
     """Compile ``tli_oracle.c`` with gcc -O2 into ``liboracle.so`` beside it."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
@@ -67,6 +80,8 @@ def _load():
         lib.oracle_tli_distributions.argtypes = [ctypes.POINTER(_Args), ctypes.c_int32, ctypes.c_int32,
                                                  ctypes.c_void_p, ctypes.c_void_p]
         lib.oracle_tli_distributions.restype = ctypes.c_int
+        lib.oracle_tli_draft.argtypes = [ctypes.POINTER(_DraftArgs), ctypes.c_int32, ctypes.c_int32]
+        lib.oracle_tli_draft.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -178,3 +193,56 @@ def distributions(target_logits, drafter_logits, id_map, temperature, b: int, j:
     if rc != 0:
         raise RuntimeError("oracle_tli_distributions failed with code %d" % rc)
     return p, qT
+
+
+def draft(drafter_logits, id_map, temperature, uniforms, probe_id=None, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Draw one drafter id per row of ``drafter_logits`` [B,R,V_d] from Algorithm 4's q'.
+
+    ``uniforms`` is [B,R].  Returns ``draft_ids`` (int32 [B,R], -1 where none can be drawn),
+    ``flags`` (int32 [B]), ``q_draft``, ``cdf_lo``, ``cdf_hi`` (float64 [B,R]) and, with
+    ``probe_id`` (int32 [B,R]), ``probe_lo/hi/w``: the normalised CDF interval and weight of that id.
+    """
+    lib = _load()
+    zd = np.asarray(drafter_logits)
+    if zd.dtype == np.float32:
+        dtype = F32
+    elif zd.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must be float32 or uint16 bfloat16 bit patterns")
+    if zd.ndim != 3 or zd.strides[2] != zd.itemsize:
+        raise ValueError("drafter logits must be [B,R,V_d] with a contiguous vocabulary axis")
+    B, R, V_d = zd.shape
+    idm = np.ascontiguousarray(id_map, dtype=np.int32)
+    if idm.shape != (V_d,):
+        raise ValueError("id_map must be [V_d]")
+    tau = np.ascontiguousarray(temperature, dtype=np.float32).reshape(B)
+    u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, R)
+    probe = None if probe_id is None else np.ascontiguousarray(probe_id, dtype=np.int32).reshape(B, R)
+    out: Dict[str, np.ndarray] = {
+        "draft_ids": np.zeros((B, R), np.int32), "flags": np.zeros(B, np.int32),
+        "q_draft": np.zeros((B, R), np.float64), "cdf_lo": np.zeros((B, R), np.float64),
+        "cdf_hi": np.zeros((B, R), np.float64),
+    }
+    if probe is not None:
+        out.update(probe_lo=np.zeros((B, R), np.float64), probe_hi=np.zeros((B, R), np.float64),
+                   probe_w=np.zeros((B, R), np.float64))
+    args = _DraftArgs(B, R, V_d, dtype, zd.ctypes.data, zd.strides[0] // zd.itemsize, zd.strides[1] // zd.itemsize,
+                      _ptr(idm), _ptr(tau), _ptr(u), _ptr(probe),
+                      _ptr(out["draft_ids"]), _ptr(out["flags"]), _ptr(out["q_draft"]),
+                      _ptr(out["cdf_lo"]), _ptr(out["cdf_hi"]),
+                      _ptr(out.get("probe_lo")), _ptr(out.get("probe_hi")), _ptr(out.get("probe_w")))
+    threads = max(1, min(int(threads), B))
+
+    def run(lo_hi):
+        rc = lib.oracle_tli_draft(ctypes.byref(args), lo_hi[0], lo_hi[1])
+        if rc != 0:
+            raise RuntimeError("oracle_tli_draft failed with code %d" % rc)
+
+    if threads == 1:
+        run((0, B))
+    else:
+        cuts = [(B * i) // threads for i in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(run, [(cuts[i], cuts[i + 1]) for i in range(threads)]))
+    return out

@@ -39,6 +39,9 @@
  * Every sum runs in index order in double precision; there is no blocking,
  * fusion or reordering.
  *
+ * The file also holds the drafting side of the same algorithms
+ * (oracle_tli_draft, at the end): drawing the draft ids from q'.
+ *
  * Parity status: every function here is pinned by tests that do not use this
  * file's own formulas (worked example, brute-force losslessness on tiny
  * vocabularies, chi-square losslessness, closed-form acceptance rate,
@@ -370,4 +373,119 @@ int oracle_tli_distributions(const oracle_args *a, int32_t b, int32_t j, double 
             if (a->id_map[x] >= 0 && a->id_map[x] < a->V_t) qT_out[a->id_map[x]] = qp[x];
     free(q); free(qp);
     return ok ? 0 : -4;
+}
+
+/*
+ * Drafting with Algorithm 4's q' (the sampling step of Algorithm 5 run with
+ * q'): for every sequence b and row r of drafter logits, draw a drafter id
+ * from q'(x) = q(x) / sum_{T cap D} q on the intersection.  One uniform per
+ * row; inverse CDF in increasing drafter-id order: the smallest x whose
+ * cumulative q' exceeds v * (sum of q'), so ids outside the intersection
+ * (weight 0) are never drawn.  tau == 0: the lowest id among those attaining
+ * the largest logit inside the intersection.  No id can be drawn (-1) when the
+ * intersection is empty, when a logit is not finite or the temperature is
+ * invalid; the row is flagged.  Parity status: pinned by the worked example of
+ * q', by a chi-square test of the drawn ids against q' formed independently,
+ * by the boundaries of the CDF on tiny vocabularies, and by the reduction to
+ * a plain softmax sampler when every id is in the intersection.
+ */
+typedef struct {
+    int32_t B, R, V_d, dtype;
+    const void *drafter_logits; /* [B, R, V_d], strides in elements */
+    int64_t d_stride_b, d_stride_r;
+    const int32_t *id_map;      /* [V_d] */
+    const float *temperature;   /* [B] */
+    const float *uniforms;      /* [B, R] */
+    const int32_t *probe_id;    /* [B, R] or NULL: report this id's CDF interval */
+    /* outputs */
+    int32_t *draft_ids;         /* [B, R] drafter ids, -1 if none can be drawn */
+    int32_t *flags;             /* [B] */
+    double *q_draft;            /* [B, R] q'(drawn id) */
+    double *cdf_lo, *cdf_hi;    /* [B, R] normalised CDF around the drawn id */
+    double *probe_lo, *probe_hi, *probe_w; /* [B, R] (only if probe_id) */
+} oracle_draft_args;
+
+int oracle_tli_draft(const oracle_draft_args *a, int32_t row_begin, int32_t row_end)
+{
+    if (!a || a->B < 1 || a->R < 1 || a->V_d < 1) return -1;
+    if (a->dtype != ORACLE_F32 && a->dtype != ORACLE_BF16) return -1;
+    if (row_begin < 0 || row_end > a->B || row_begin > row_end) return -1;
+    const int V_d = a->V_d, R = a->R;
+    double *q = (double *)malloc(sizeof(double) * (size_t)V_d);
+    double *qp = (double *)malloc(sizeof(double) * (size_t)V_d);
+    if (!q || !qp) { free(q); free(qp); return -3; }
+    /* qprime_row() reads the drafter side of the verification arguments */
+    oracle_args va;
+    memset(&va, 0, sizeof va);
+    va.V_d = V_d; va.dtype = a->dtype; va.drafter_logits = a->drafter_logits; va.id_map = a->id_map;
+
+    for (int b = row_begin; b < row_end; ++b) {
+        const double tau = (double)a->temperature[b];
+        int flags = 0;
+        for (int r = 0; r < R; ++r) {
+            const int64_t o = (int64_t)b * R + r;
+            const int64_t off = (int64_t)b * a->d_stride_b + (int64_t)r * a->d_stride_r;
+            int d = -1;
+            double qd = 0.0, lo = 0.0, hi = 0.0;
+            if (!(tau >= 0.0) || isinf(tau)) {
+                flags |= FLAG_BAD_TEMPERATURE;
+            } else if (tau == 0.0) {
+                /* lowest id attaining the maximum inside the intersection */
+                double m = 0.0;
+                int finite = 1;
+                for (int x = 0; x < V_d; ++x) {
+                    double z = load_logit(a->drafter_logits, a->dtype, off + x);
+                    if (!isfinite(z)) finite = 0;
+                    if (a->id_map[x] >= 0 && (d < 0 || z > m)) { m = z; d = x; }
+                }
+                if (!finite) { flags |= FLAG_NONFINITE; d = -1; }
+                else if (d < 0) flags |= FLAG_FALLBACK;
+                else { qd = 1.0; lo = 0.0; hi = 1.0; }
+            } else {
+                int ok_sc, empty;
+                if (!qprime_row(&va, off, tau, q, qp, &ok_sc, &empty)) {
+                    flags |= FLAG_NONFINITE;
+                } else {
+                    if (!ok_sc) flags |= FLAG_SELFCHECK;
+                    double total = 0.0;
+                    for (int x = 0; x < V_d; ++x) total += qp[x];
+                    if (!(total > 0.0)) {
+                        flags |= FLAG_FALLBACK;           /* empty intersection */
+                    } else {
+                        const double target = (double)a->uniforms[o] * total;
+                        double C = 0.0, C_before = 0.0;
+                        int last_pos = 0;
+                        for (int x = 0; x < V_d; ++x) {
+                            double Cn = C + qp[x];
+                            if (qp[x] > 0.0) last_pos = x;
+                            if (d < 0 && Cn > target) { d = x; C_before = C; hi = Cn / total; }
+                            C = Cn;
+                        }
+                        if (d < 0) { d = last_pos; C_before = C - qp[last_pos]; hi = 1.0; }
+                        lo = C_before / total;
+                        qd = qp[d];
+                        if (a->probe_id) {
+                            int g = a->probe_id[o];
+                            double plo = 0.0, phi = 0.0, pw = 0.0;
+                            if (g >= 0 && g < V_d) {
+                                double Cc = 0.0;
+                                for (int x = 0; x < g; ++x) Cc += qp[x];
+                                plo = Cc / total; phi = (Cc + qp[g]) / total; pw = qp[g] / total;
+                            }
+                            if (a->probe_lo) a->probe_lo[o] = plo;
+                            if (a->probe_hi) a->probe_hi[o] = phi;
+                            if (a->probe_w) a->probe_w[o] = pw;
+                        }
+                    }
+                }
+            }
+            a->draft_ids[o] = d;
+            if (a->q_draft) a->q_draft[o] = qd;
+            if (a->cdf_lo) a->cdf_lo[o] = lo;
+            if (a->cdf_hi) a->cdf_hi[o] = hi;
+        }
+        if (a->flags) a->flags[b] = flags;
+    }
+    free(q); free(qp);
+    return 0;
 }
