@@ -183,6 +183,56 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
  */
 int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 
+typedef struct {
+    int32_t B;      /* sequences, >= 1 */
+    int32_t R;      /* rows of drafter logits per sequence, >= 1; B * R <= TLI_MAX_B */
+    int32_t dtype;  /* TLI_F32 or TLI_BF16 */
+
+    /* [device] drafter logits [B, R, V_d]; strides in elements, vocabulary axis
+     * contiguous, base pointer aligned to the element size. */
+    const void *drafter_logits;
+    int64_t d_stride_b, d_stride_r;
+
+    const float *temperature;   /* [device] float[B]; 0 = arg-max over the intersection */
+    const float *uniforms;      /* [device] float[B, R] in [0, 1), one per row */
+
+    int32_t *draft_ids;         /* [device] out int32[B, R]: the drawn drafter-vocabulary id,
+                                 * always inside the intersection; -1 when none can be drawn */
+    float *q_draft;             /* [device] out float[B, R]: q'(drawn id) (1 at temperature 0,
+                                 * 0 when no id was drawn); may be NULL */
+    int32_t *draft_status;      /* [device] out int32[B, R] of TLI_ROW_* bits (NONFINITE,
+                                 * FALLBACK = empty intersection or no mass in it,
+                                 * BAD_TEMPERATURE); may be NULL */
+
+    void *workspace;            /* [device] scratch, 256-byte aligned, >= tli_draft_workspace_bytes() */
+    size_t workspace_bytes;
+} tli_draft_args;
+
+/* Bytes of device scratch tli_draft_sample() needs for (B, R, dtype); 0 on bad arguments. */
+size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32_t dtype);
+
+/*
+ * Draw the draft tokens: the drafter's side of Algorithm 4.  TLI has the
+ * drafter sample from q' instead of q (Algorithm 5's drafting step run with
+ * q'), so that every draft lies in the intersection of the vocabularies.  For
+ * every sequence b and row r, with tau = temperature[b] and v = uniforms[b,r]:
+ *
+ *   tau > 0:  w(x) = exp((z[x] - m) / tau) if map[x] >= 0, else 0 (m = largest
+ *             logit inside the intersection); q'(x) = w(x) / sum w, which equals
+ *             Algorithm 4's q(x) / sum_{T cap D} q because the softmax
+ *             denominator cancels; the id is found by inverse CDF in increasing
+ *             drafter-id order: the smallest x whose cumulative weight exceeds
+ *             v * total.
+ *   tau == 0: the lowest id attaining the largest logit inside the intersection.
+ *
+ * The ids are what tli_verify() takes as draft_ids, and q_draft is the q'(d_j)
+ * it recomputes.  One pass over the logits; arithmetic as in tli_verify().
+ * Asynchronous on the stream, allocates nothing, only launches a kernel; it
+ * uses the context's counters, so it must not overlap another call on the same
+ * context.  Errors as for tli_verify().
+ */
+int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *args, void *cuda_stream);
+
 /*
  * Measurement hook: the three-kernel form of tli_verify() (see tli_set_fused)
  * with CUDA events recorded on `cuda_stream` around each kernel.  Blocks until
@@ -201,7 +251,7 @@ int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_str
  * extra token while later sequences are still streaming.  Results are identical
  * bit for bit.  The fused form is the slower one today (its sampling chunks
  * stall the streaming warps on their gathers) and is kept as the basis for
- * further work; see the design doc.
+ * further work.
  */
 int tli_set_fused(tli_ctx *ctx, int enabled);
 

@@ -1144,6 +1144,300 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
 }
 
 // ---------------------------------------------------------------------------
+// drafting: one id per drafter row from q' (Algorithm 4 as a sampling distribution)
+// ---------------------------------------------------------------------------
+//
+// One CTA per 16 KB tile of a drafter row.  A tile leaves (c, S): its own integer-valued
+// reference c = ceil(max * s) over the ids inside the intersection and S = sum 2^(z*s - c) over
+// them, fp32 per vector and fp64 across vectors.  The last CTA of the row (atomic ticket, nobody
+// waits) brings the tiles to the row's reference by exact powers of two, finds the tile the
+// target v * total falls into, and walks that tile vector by vector and element by element with
+// the sums formed by the very code that formed S -- one pass over the logits.
+
+struct DraftParams {
+    int B, R, V_d, ntile;
+    const void *zd; long long d_sb, d_sr;
+    const uint32_t *maskbits;
+    const float *tau; const float *u;
+    int *draft_ids; float *q_out; int *status;
+    struct DraftPart *part;        // [B*R][ntile]
+    unsigned *cnt;                 // [B*R] tickets, zero between calls
+};
+struct __align__(16) DraftPart {
+    double S;      // weight of the tile at its own reference (temperature 0: the tile's best id)
+    float c;       // the tile's reference (temperature 0: the tile's largest logit)
+    int flags;     // TLI_ROW_NONFINITE if the tile holds a NaN or +inf
+};
+
+// Elements of vector v of a drafter row: the logit inside the intersection, -inf outside it and
+// outside the row.  `bad` collects NaN / +inf anywhere in the row.
+template <int DT>
+__device__ __forceinline__ void draft_vector(const DraftParams &P, const RowView<DT> &rv, int v, int nvec,
+                                             float (&z)[Elt<DT>::kPerVec], uint32_t &bits, bool &bad) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    bits = 0u;
+    if (v >= nvec) {
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) z[i] = -INFINITY;
+        return;
+    }
+    const uint4 raw = rv.load(v);
+    unpack<DT>(raw, z);
+    bits = mask_bits(P.maskbits, rv.first_elem(v));
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) {
+        bad = bad || !(z[i] < INFINITY);                    // NaN or +inf
+        z[i] = ((bits >> i) & 1u) ? z[i] : -INFINITY;
+    }
+}
+
+template <int N> __device__ __forceinline__ void draft_weights(const float (&z)[N], float s, float nc, float (&w)[N]) {
+#pragma unroll
+    for (int i = 0; i < N; ++i) w[i] = ex2(__fmaf_rn(z[i], s, nc));
+}
+
+// 2^k * x for an integer-valued k >= 0
+__device__ __forceinline__ double scale_up(double x, float k) { return scalbn(x, static_cast<int>(k)); }
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_draft_kernel(const DraftParams P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    __shared__ double sm_red[kWarps];
+    __shared__ float sm_max[kWarps];
+    __shared__ int sm_idx[kWarps];
+    __shared__ int sm_flag, sm_last;
+    __shared__ double sm_tiles[kMaxTiles];
+    __shared__ float sm_ref[kMaxTiles];
+    __shared__ float sm_seg[kVecPerTile];
+    __shared__ double sm_warp_tot[kWarps];
+    __shared__ int sm_tile, sm_found, sm_lastpos, sm_none;
+    __shared__ double sm_rem, sm_total;
+    __shared__ float sm_cmax;
+    const int row = blockIdx.y, tile = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int b = row / P.R, r = row - b * P.R;
+    const float tau = __ldg(P.tau + b);
+    if (!(tau >= 0.f) || isinf(tau)) {
+        if (tile == 0 && tid == 0) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = TLI_ROW_BAD_TEMPERATURE;
+        }
+        return;
+    }
+    const bool greedy = (tau == 0.f);
+    const float s = 1.4426950408889634f / tau;
+    const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
+    const int nvec = rv.nvec();
+    if (tid == 0) sm_flag = 0;
+
+    // ---- this tile ----
+    float z[kVecPerThread][EPV];
+    bool bad = false;
+    float best = -INFINITY; int best_idx = INT_MAX;        // largest logit inside the intersection, lowest id
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = tile * kVecPerTile + k * kThreads + tid;
+        uint32_t bits;
+        draft_vector<DT>(P, rv, v, nvec, z[k], bits, bad);
+        const int e0 = rv.first_elem(v);
+#pragma unroll
+        for (int i = 0; i < EPV; ++i)
+            if (((bits >> i) & 1u) && (best_idx == INT_MAX || z[k][i] > best)) { best = z[k][i]; best_idx = e0 + i; }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+        const int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
+        if (i2 != INT_MAX && (best_idx == INT_MAX || b2 > best || (b2 == best && i2 < best_idx))) { best = b2; best_idx = i2; }
+    }
+    if (lane == 0) { sm_max[warp] = best; sm_idx[warp] = best_idx; }
+    __syncthreads();
+    if (bad) atomicOr(&sm_flag, static_cast<int>(TLI_ROW_NONFINITE));
+    best = sm_max[0]; best_idx = sm_idx[0];
+#pragma unroll
+    for (int i = 1; i < kWarps; ++i) {
+        const float b2 = sm_max[i]; const int i2 = sm_idx[i];
+        if (i2 != INT_MAX && (best_idx == INT_MAX || b2 > best || (b2 == best && i2 < best_idx))) { best = b2; best_idx = i2; }
+    }
+    const float c_tile = (best_idx == INT_MAX) ? kNegBig : reference_for(best * s);
+    double acc = 0.0;
+    if (!greedy) {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            float w[EPV];
+            draft_weights(z[k], s, -c_tile, w);
+            acc += static_cast<double>(ordered_sum(w));
+        }
+    }
+    acc = warp_sum(acc);
+    if (lane == 0) sm_red[warp] = acc;
+    __syncthreads();
+    if (tid == 0) {
+        double tot = 0.0;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) tot += sm_red[i];
+        DraftPart pt;
+        pt.S = greedy ? static_cast<double>(best_idx) : tot;
+        pt.c = greedy ? best : c_tile;
+        pt.flags = sm_flag;
+        DraftPart *dst = P.part + static_cast<size_t>(row) * P.ntile + tile;
+        __stcg(reinterpret_cast<double2 *>(dst), *reinterpret_cast<const double2 *>(&pt));
+        __threadfence();
+        const unsigned ticket = atomicAdd(P.cnt + row, 1u);
+        sm_last = (ticket == static_cast<unsigned>(P.ntile) - 1);
+        if (sm_last) P.cnt[row] = 0;
+    }
+    __syncthreads();
+    if (!sm_last) return;
+    __threadfence();
+
+    // ---- last CTA of the row: pick the id ----
+    const int ntile = P.ntile;
+    if (tid == 0) { sm_flag = 0; sm_none = 0; }
+    __syncthreads();
+    for (int i = tid; i < ntile; i += kThreads) {
+        const double2 raw = __ldcg(reinterpret_cast<const double2 *>(P.part + static_cast<size_t>(row) * ntile + i));
+        const DraftPart pt = *reinterpret_cast<const DraftPart *>(&raw);
+        sm_tiles[i] = pt.S; sm_ref[i] = pt.c;
+        if (pt.flags) atomicOr(&sm_flag, pt.flags);
+    }
+    __syncthreads();
+    int status = sm_flag;
+    if (greedy) {
+        if (tid == 0) {
+            float bb = -INFINITY; int ii = INT_MAX;
+            for (int i = 0; i < ntile; ++i) {               // tiles in increasing id order: strict > keeps the lowest id
+                const int i2 = static_cast<int>(sm_tiles[i]);
+                if (i2 != INT_MAX && (ii == INT_MAX || sm_ref[i] > bb)) { bb = sm_ref[i]; ii = i2; }
+            }
+            int d = ii;
+            if (status & TLI_ROW_NONFINITE) d = -1;
+            else if (ii == INT_MAX) { d = -1; status |= TLI_ROW_FALLBACK; }
+            P.draft_ids[row] = d;
+            if (P.q_out) P.q_out[row] = d >= 0 ? 1.f : 0.f;
+            if (P.status) P.status[row] = status;
+        }
+        return;
+    }
+    if (tid == 0) {
+        float cmax = kNegBig;
+        for (int i = 0; i < ntile; ++i) cmax = fmaxf(cmax, sm_ref[i]);
+        double R = 0.0;
+        for (int i = 0; i < ntile; ++i) { sm_tiles[i] *= pow2_neg_d(sm_ref[i] - cmax); R += sm_tiles[i]; }
+        if ((status & TLI_ROW_NONFINITE) || !isfinite(R)) { status |= TLI_ROW_NONFINITE; sm_none = 1; }
+        else if (!(R > 0.0)) { status |= TLI_ROW_FALLBACK; sm_none = 1; }
+        else {
+            const double target = static_cast<double>(__ldg(P.u + row)) * R;
+            double run = 0.0, before = 0.0;
+            int T = -1, lastpos = 0;
+            for (int i = 0; i < ntile; ++i) {
+                const double nx = run + sm_tiles[i];
+                if (sm_tiles[i] > 0.0) lastpos = i;
+                if (T < 0 && nx > target) { T = i; before = run; }
+                run = nx;
+            }
+            if (T < 0) { T = lastpos; before = R - sm_tiles[lastpos]; }
+            sm_tile = T;
+            sm_rem = scale_up(target - before, cmax - sm_ref[T]);     // in the tile's own scale
+            sm_total = R; sm_cmax = cmax;
+        }
+        if (sm_none) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = status;
+        }
+        sm_found = INT_MAX; sm_lastpos = -1;
+    }
+    __syncthreads();
+    if (sm_none) return;
+    const int T = sm_tile;
+    const double rem = sm_rem;
+    const float nc = -sm_ref[T];
+    // vector sums of tile T in address order, by the code that formed the tile's sum
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int g = k * kThreads + tid;
+        const int v = T * kVecPerTile + g;
+        float zz[EPV], w[EPV];
+        uint32_t bits; bool ignore = false;
+        draft_vector<DT>(P, rv, v, nvec, zz, bits, ignore);
+        draft_weights(zz, s, nc, w);
+        sm_seg[g] = ordered_sum(w);
+    }
+    __syncthreads();
+    // thread i owns vectors 4i .. 4i+3: block-wide exclusive prefix in fp64
+    double loc[kVecPerThread];
+    double mine = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) { loc[k] = static_cast<double>(sm_seg[tid * kVecPerThread + k]); mine += loc[k]; }
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) sm_warp_tot[warp] = incl;
+    __syncthreads();
+    double base = 0.0;
+    for (int i = 0; i < warp; ++i) base += sm_warp_tot[i];
+    double run = base + incl - mine;                       // mass before this thread's first vector
+    int cand = INT_MAX, lastpos = -1;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const double nx = run + loc[k];
+        if (loc[k] > 0.0) lastpos = tid * kVecPerThread + k;
+        if (cand == INT_MAX && nx > rem) cand = tid * kVecPerThread + k;
+        run = nx;
+    }
+    if (cand != INT_MAX) atomicMin(&sm_found, cand);
+    if (lastpos >= 0) atomicMax(&sm_lastpos, lastpos);
+    __syncthreads();
+    const int found = sm_found;
+    const int G = (found != INT_MAX) ? found : sm_lastpos;
+    if (G < 0) {                                           // cannot happen when the tile has positive mass
+        if (tid == 0) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = status | TLI_ROW_FALLBACK;
+        }
+        return;
+    }
+    if (tid == G / kVecPerThread) {
+        // walk the elements of vector G with the running fp32 sum that formed its total; when
+        // rounding left no vector above the target, take the last positive element instead
+        double before = 0.0;
+        if (found != INT_MAX) {
+            before = base + incl - mine;
+            for (int k = 0; k < G - tid * kVecPerThread; ++k) before += loc[k];
+        }
+        const double rem2 = (found != INT_MAX) ? (rem - before) : INFINITY;
+        const int v = T * kVecPerTile + G;
+        float zz[EPV], w[EPV];
+        uint32_t bits; bool ignore = false;
+        draft_vector<DT>(P, rv, v, nvec, zz, bits, ignore);
+        draft_weights(zz, s, nc, w);
+        float runf = 0.f;
+        int pick = -1, lastw = 0;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+            runf = (i == 0) ? w[0] : __fadd_rn(runf, w[i]);
+            if (w[i] > 0.f) lastw = i;
+            if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
+        }
+        if (pick < 0) pick = lastw;
+        float wp = w[0];
+#pragma unroll
+        for (int i = 1; i < EPV; ++i) wp = (i == pick) ? w[i] : wp;
+        int id = rv.first_elem(v) + pick;
+        id = min(max(id, 0), P.V_d - 1);
+        P.draft_ids[row] = id;
+        if (P.q_out) P.q_out[row] = static_cast<float>(static_cast<double>(wp) * pow2_neg_d(sm_ref[T] - sm_cmax) / sm_total);
+        if (P.status) P.status[row] = status;
+    }
+}
+
+// ---------------------------------------------------------------------------
 // the fused kernel: statistics, decisions and sampling in one persistent grid
 // ---------------------------------------------------------------------------
 //
@@ -2086,6 +2380,42 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
 
 int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
     return verify_impl(ctx, a, cuda_stream, nullptr);
+}
+
+size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32_t dtype) {
+    if (!ctx || B < 1 || R < 1 || static_cast<long long>(B) * R > TLI_MAX_B) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    const size_t ntile = static_cast<size_t>(chunks_per_row(ctx->V_d, dtype, kVecPerTile));
+    return align_up(sizeof(DraftPart) * static_cast<size_t>(B) * R * ntile, 256);
+}
+
+int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->R < 1) return TLI_ERR_ARG;
+    if (static_cast<long long>(a->B) * a->R > TLI_MAX_B) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->drafter_logits || !a->temperature || !a->uniforms || !a->draft_ids) return TLI_ERR_ARG;
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(a->drafter_logits) % elt) return TLI_ERR_ARG;
+    if (a->d_stride_b < 0 || a->d_stride_r < 0) return TLI_ERR_ARG;
+    const size_t need = tli_draft_workspace_bytes(ctx, a->B, a->R, a->dtype);
+    if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < need)
+        return TLI_ERR_WORKSPACE;
+    DraftParams P;
+    P.B = a->B; P.R = a->R; P.V_d = ctx->V_d;
+    P.ntile = chunks_per_row(ctx->V_d, a->dtype, kVecPerTile);
+    P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sr = a->d_stride_r;
+    P.maskbits = ctx->d_mask; P.tau = a->temperature; P.u = a->uniforms;
+    P.draft_ids = a->draft_ids; P.q_out = a->q_draft; P.status = a->draft_status;
+    P.part = reinterpret_cast<DraftPart *>(a->workspace);
+    P.cnt = ctx->d_counters + (TLI_MAX_B + 1);           // the sampling pass's tickets: zero between calls
+    const dim3 grid(static_cast<unsigned>(P.ntile), static_cast<unsigned>(a->B * a->R));
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (a->dtype == TLI_F32) tli_draft_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(P);
+    else tli_draft_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(P);
+    const cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_kernel");
+    return TLI_OK;
 }
 
 int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up) {

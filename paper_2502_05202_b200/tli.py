@@ -38,6 +38,7 @@ TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
 EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
+           "tli_draft_workspace_bytes", "tli_draft_sample",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -50,6 +51,16 @@ class tli_verify_args(ctypes.Structure):
         ("draft_ids", ctypes.c_void_p), ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
         ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
         ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+class tli_draft_args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("R", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_r", ctypes.c_int64),
+        ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("draft_ids", ctypes.c_void_p), ("q_draft", ctypes.c_void_p), ("draft_status", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
 
@@ -87,6 +98,10 @@ def load() -> ctypes.CDLL:
         lib.tli_verify_profile.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p,
                                            ctypes.POINTER(ctypes.c_float)]
         lib.tli_verify_profile.restype = ctypes.c_int
+        lib.tli_draft_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_draft_workspace_bytes.restype = ctypes.c_size_t
+        lib.tli_draft_sample.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_draft_args), ctypes.c_void_p]
+        lib.tli_draft_sample.restype = ctypes.c_int
         lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_fused.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
@@ -184,6 +199,38 @@ def tli_verify_static(ctx: int, args: tli_verify_args, stream: Optional[int] = N
         raise TLIError(rc, "tli_verify_static")
 
 
+def tli_draft_workspace_bytes(ctx: int, B: int, R: int, dtype: int) -> int:
+    return int(load().tli_draft_workspace_bytes(ctx, B, R, dtype))
+
+
+def make_draft_args(drafter_logits: torch.Tensor, temperature: torch.Tensor, uniforms: torch.Tensor,
+                    draft_ids: torch.Tensor, workspace: torch.Tensor, q_draft: Optional[torch.Tensor] = None,
+                    draft_status: Optional[torch.Tensor] = None) -> tli_draft_args:
+    """Fill a tli_draft_args from device tensors (no copies; the tensors must outlive the call)."""
+    B, R, _ = drafter_logits.shape
+    dt = _logit_dtype(drafter_logits)
+    if drafter_logits.stride(2) != 1:
+        raise ValueError("the vocabulary axis must be contiguous")
+    for name, t, dtype, shape in (("temperature", temperature, torch.float32, (B,)),
+                                  ("uniforms", uniforms, torch.float32, (B, R)),
+                                  ("draft_ids", draft_ids, torch.int32, (B, R))):
+        if t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous %s tensor of shape %s" % (name, dtype, shape))
+    opt = lambda t: None if t is None else t.data_ptr()
+    return tli_draft_args(B, R, dt, drafter_logits.data_ptr(), drafter_logits.stride(0), drafter_logits.stride(1),
+                          temperature.data_ptr(), uniforms.data_ptr(), draft_ids.data_ptr(), opt(q_draft),
+                          opt(draft_status), workspace.data_ptr(), workspace.numel() * workspace.element_size())
+
+
+def tli_draft_sample(ctx: int, args: tli_draft_args, stream: Optional[int] = None) -> None:
+    """tli_draft_sample() on ``stream`` (a cudaStream_t as int; default: torch's current stream)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_draft_sample(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_draft_sample")
+
+
 def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
     """tli_verify_profile(): blocks; returns ms of (statistics kernel, decision kernel, sampling kernel)."""
     if stream is None:
@@ -242,6 +289,23 @@ class Verifier:
         if self._ws is None or self._ws.numel() < need:
             self._ws = torch.empty(need, dtype=torch.uint8, device=self.device)
         return self._ws
+
+    def draft(self, drafter_logits, temperature, uniforms) -> Dict[str, torch.Tensor]:
+        """Draw one drafter id per row of ``drafter_logits`` [B,R,V_d] from q'; returns device tensors."""
+        B, R, _ = drafter_logits.shape
+        dev = self.device
+        out = {"draft_ids": torch.empty(B, R, dtype=torch.int32, device=dev),
+               "q_draft": torch.empty(B, R, dtype=torch.float32, device=dev),
+               "draft_status": torch.empty(B, R, dtype=torch.int32, device=dev)}
+        need = tli_draft_workspace_bytes(self.ctx, B, R, _logit_dtype(drafter_logits))
+        if need == 0:
+            raise TLIError(TLI_ERR_UNSUPPORTED, "tli_draft_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        args = make_draft_args(drafter_logits, temperature, uniforms, out["draft_ids"], self._ws,
+                               out["q_draft"], out["draft_status"])
+        tli_draft_sample(self.ctx, args)
+        return out
 
     def verify(self, target_logits, drafter_logits, draft_ids, temperature, uniforms,
                diagnostics: bool = True) -> Dict[str, torch.Tensor]:
