@@ -287,6 +287,28 @@ class GpuCase:
         t = [a.elapsed_time(b) for a, b in ev]
         return statistics.median(t), min(t)
 
+    def draft_timing(self, steps):
+        """tli_draft_sample() on this workload's drafter logits, all K rows per sequence: ms per call."""
+        torch, tli, cfg = self.torch, self.tli, self.cfg
+        ids = torch.empty(cfg.B, cfg.K, dtype=torch.int32, device=self.zd[0].device)
+        need = tli.tli_draft_workspace_bytes(self.ver.ctx, cfg.B, cfg.K, tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16)
+        ws = torch.empty(need, dtype=torch.uint8, device=self.zd[0].device)
+        u = self.u[:, :cfg.K].contiguous()
+        args = [tli.make_draft_args(z, self.tau, u, ids, ws) for z in self.zd]
+        n = [0]
+
+        def step():
+            tli.tli_draft_sample(self.ver.ctx, args[n[0] % len(args)], self.stream)
+            n[0] += 1
+        for _ in range(3 + len(args)):
+            step()
+        ms = timed(torch, None, steps, step, 1) / steps
+        assert int((ids < 0).sum()) == 0, "a draft id could not be drawn on benchmark inputs"
+        greedy = int((self.tau == 0).sum())
+        nbytes = cfg.elt * cfg.B * cfg.K * cfg.V_d
+        return {"ms_per_call": ms, "rows_per_s": cfg.B * cfg.K / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
+                "rows_per_call": cfg.B * cfg.K, "bytes_per_call": nbytes, "greedy_sequences": greedy}
+
     def e2e_bytes(self):
         h = self.host
         h2d = sum(h[k].numel() * h[k].element_size() for k in ("zt", "zd", "draft", "tau", "u"))
@@ -380,6 +402,7 @@ def gpu_arm(args):
     case.profile(3)
     ms_stats, ms_decide, ms_sample = case.profile(args.steps)
     calls = call_timings(case, torch, args.steps)
+    draft = case.draft_timing(max(args.steps, 20)) if world == 1 else None
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
@@ -406,6 +429,7 @@ def gpu_arm(args):
         "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
         "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
         "per_call": calls,
+        "draft_sample": draft,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
@@ -424,7 +448,8 @@ def gpu_arm(args):
             if c.name == cfg.name:
                 per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
                             "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
-                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls})
+                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls,
+                            "draft_sample": draft})
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
@@ -434,6 +459,7 @@ def gpu_arm(args):
             k.profile(3)
             a, d, b = k.profile(min(steps, 50))
             kc = call_timings(k, torch, steps)
+            kc["draft_sample"] = k.draft_timing(steps)
             k.check()
             per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
                         "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,

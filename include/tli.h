@@ -227,6 +227,9 @@ size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32
  *
  * The ids are what tli_verify() takes as draft_ids, and q_draft is the q'(d_j)
  * it recomputes.  One pass over the logits; arithmetic as in tli_verify().
+ * A logit of -inf is an id of probability zero; NaN or +inf at an id inside
+ * the intersection flags the row (-1, TLI_ROW_NONFINITE).  Logits outside the
+ * intersection do not enter q' and are not examined.
  * Asynchronous on the stream, allocates nothing, only launches a kernel; it
  * uses the context's counters, so it must not overlap another call on the same
  * context.  Errors as for tli_verify().

@@ -1147,72 +1147,255 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
 // drafting: one id per drafter row from q' (Algorithm 4 as a sampling distribution)
 // ---------------------------------------------------------------------------
 //
-// One CTA per 16 KB tile of a drafter row.  A tile leaves (c, S): its own integer-valued
-// reference c = ceil(max * s) over the ids inside the intersection and S = sum 2^(z*s - c) over
-// them, fp32 per vector and fp64 across vectors.  The last CTA of the row (atomic ticket, nobody
-// waits) brings the tiles to the row's reference by exact powers of two, finds the tile the
-// target v * total falls into, and walks that tile vector by vector and element by element with
-// the sums formed by the very code that formed S -- one pass over the logits.
+// One pass over the logits.  A CTA takes a 16 KB tile of a drafter row, each of its warps a 2 KB
+// strip of it (128 vectors, vector k*32 + lane to lane `lane`), and nothing in a strip needs
+// another warp: the strip leaves (c, S), its own integer-valued reference c = ceil(max * s) over
+// the ids inside the intersection and S = sum 2^(z*s - c) over them, fp32 per vector and fp64
+// across vectors.  Then one CTA per row -- the last tile CTA to finish (atomic ticket, nobody
+// waits) or, for large batches, a second kernel -- brings the strips to the row's reference by
+// exact powers of two, finds the strip the target v * total falls into, and one warp walks that
+// strip vector by vector and element by element with sums formed by the code that formed S.
 
+constexpr int kStripsPerTile = kWarps;
+constexpr int kMaxStrips = kMaxTiles * kStripsPerTile;
+
+struct __align__(16) DraftPart {
+    double S;      // weight of the strip at its own reference (temperature 0: the strip's best id)
+    float c;       // the strip's reference (temperature 0: the strip's largest logit)
+    int flags;     // temperature 0: TLI_ROW_NONFINITE if an id inside the intersection holds NaN or +inf
+};
 struct DraftParams {
-    int B, R, V_d, ntile;
+    int B, R, V_d, ntile, nstrip, split;
     const void *zd; long long d_sb, d_sr;
     const uint32_t *maskbits;
     const float *tau; const float *u;
     int *draft_ids; float *q_out; int *status;
-    struct DraftPart *part;        // [B*R][ntile]
+    DraftPart *part;               // [B*R][nstrip]
     unsigned *cnt;                 // [B*R] tickets, zero between calls
 };
-struct __align__(16) DraftPart {
-    double S;      // weight of the tile at its own reference (temperature 0: the tile's best id)
-    float c;       // the tile's reference (temperature 0: the tile's largest logit)
-    int flags;     // TLI_ROW_NONFINITE if the tile holds a NaN or +inf
-};
 
-// Elements of vector v of a drafter row: the logit inside the intersection, -inf outside it and
-// outside the row.  `bad` collects NaN / +inf anywhere in the row.
+// Vector v of a drafter row with the ids outside the intersection (and outside the row) set to -inf.
 template <int DT>
-__device__ __forceinline__ void draft_vector(const DraftParams &P, const RowView<DT> &rv, int v, int nvec,
-                                             float (&z)[Elt<DT>::kPerVec], uint32_t &bits, bool &bad) {
-    constexpr int EPV = Elt<DT>::kPerVec;
+__device__ __forceinline__ uint4 draft_masked_vector(const DraftParams &P, const RowView<DT> &rv, int v, int nvec,
+                                                     uint32_t &bits) {
+    constexpr uint32_t NI = Elt<DT>::kNegInfWord;
     bits = 0u;
-    if (v >= nvec) {
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) z[i] = -INFINITY;
-        return;
-    }
-    const uint4 raw = rv.load(v);
-    unpack<DT>(raw, z);
+    if (v >= nvec) return make_uint4(NI, NI, NI, NI);
+    uint4 raw = rv.load(v);
     bits = mask_bits(P.maskbits, rv.first_elem(v));
-#pragma unroll
-    for (int i = 0; i < EPV; ++i) {
-        bad = bad || !(z[i] < INFINITY);                    // NaN or +inf
-        z[i] = ((bits >> i) & 1u) ? z[i] : -INFINITY;
+    if constexpr (DT == TLI_BF16) {
+        mask_bf16_vector(raw, bits);
+    } else {
+        raw.x = (bits & 1u) ? raw.x : NI; raw.y = (bits & 2u) ? raw.y : NI;
+        raw.z = (bits & 4u) ? raw.z : NI; raw.w = (bits & 8u) ? raw.w : NI;
     }
+    return raw;
 }
 
-template <int N> __device__ __forceinline__ void draft_weights(const float (&z)[N], float s, float nc, float (&w)[N]) {
+// fp32 sum, in element order, of the weights 2^(z*s + nc) of one masked vector; the weights in w[]
+template <int DT>
+__device__ __forceinline__ float draft_vector_sum(const uint4 &m, float s, float nc, float (&w)[Elt<DT>::kPerVec]) {
+    float z[Elt<DT>::kPerVec];
+    unpack<DT>(m, z);
 #pragma unroll
-    for (int i = 0; i < N; ++i) w[i] = ex2(__fmaf_rn(z[i], s, nc));
+    for (int i = 0; i < Elt<DT>::kPerVec; ++i) w[i] = ex2(__fmaf_rn(z[i], s, nc));
+    return ordered_sum(w);
 }
 
+__device__ __forceinline__ DraftPart load_part(const DraftPart *p) {
+    const double2 raw = __ldcg(reinterpret_cast<const double2 *>(p));
+    return *reinterpret_cast<const DraftPart *>(&raw);
+}
+__device__ __forceinline__ void store_part(DraftPart *p, const DraftPart &v) {
+    __stcg(reinterpret_cast<double2 *>(p), *reinterpret_cast<const double2 *>(&v));
+}
+__device__ __forceinline__ bool better(float b2, int i2, float best, int idx) {   // larger logit, then lower id
+    return i2 != INT_MAX && (idx == INT_MAX || b2 > best || (b2 == best && i2 < idx));
+}
 // 2^k * x for an integer-valued k >= 0
 __device__ __forceinline__ double scale_up(double x, float k) { return scalbn(x, static_cast<int>(k)); }
 
+// The id of one row from its strips' (c, S), by one CTA.
 template <int DT>
-__global__ void __launch_bounds__(kThreads) tli_draft_kernel(const DraftParams P) {
+__device__ void draft_select(const DraftParams &P, int row, const RowView<DT> &rv, float tau) {
     constexpr int EPV = Elt<DT>::kPerVec;
-    __shared__ double sm_red[kWarps];
-    __shared__ float sm_max[kWarps];
-    __shared__ int sm_idx[kWarps];
-    __shared__ int sm_flag, sm_last;
-    __shared__ double sm_tiles[kMaxTiles];
-    __shared__ float sm_ref[kMaxTiles];
-    __shared__ float sm_seg[kVecPerTile];
+    __shared__ double sm_S[kMaxStrips];
+    __shared__ float sm_c[kMaxStrips];
     __shared__ double sm_warp_tot[kWarps];
-    __shared__ int sm_tile, sm_found, sm_lastpos, sm_none;
+    __shared__ float sm_wmax[kWarps];
+    __shared__ int sm_widx[kWarps];
+    __shared__ int sm_flag, sm_found, sm_lastpos, sm_none;
     __shared__ double sm_rem, sm_total;
-    __shared__ float sm_cmax;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int nstrip = P.nstrip;
+    const bool greedy = (tau == 0.f);
+    if (tid == 0) { sm_flag = 0; sm_found = INT_MAX; sm_lastpos = -1; sm_none = 0; }
+    __syncthreads();
+    const int per = (nstrip + kThreads - 1) / kThreads;      // consecutive strips per thread
+    const int i0 = tid * per, i1 = min(i0 + per, nstrip);
+    float cmax = kNegBig; int bidx = INT_MAX; int flags = 0;
+    for (int i = i0; i < i1; ++i) {
+        const DraftPart pt = load_part(P.part + static_cast<size_t>(row) * nstrip + i);
+        sm_S[i] = pt.S; sm_c[i] = pt.c; flags |= pt.flags;
+        if (greedy) {
+            const int i2 = static_cast<int>(pt.S);
+            if (better(pt.c, i2, cmax, bidx)) { cmax = pt.c; bidx = i2; }
+        } else {
+            cmax = fmaxf(cmax, pt.c);
+        }
+    }
+    if (flags) atomicOr(&sm_flag, flags);
+    if (greedy) {
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            const float b2 = __shfl_xor_sync(0xffffffffu, cmax, o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, bidx, o);
+            if (better(b2, i2, cmax, bidx)) { cmax = b2; bidx = i2; }
+        }
+        if (lane == 0) { sm_wmax[warp] = cmax; sm_widx[warp] = bidx; }
+        __syncthreads();
+        if (tid == 0) {
+            float bb = sm_wmax[0]; int ii = sm_widx[0];
+            for (int i = 1; i < kWarps; ++i) if (better(sm_wmax[i], sm_widx[i], bb, ii)) { bb = sm_wmax[i]; ii = sm_widx[i]; }
+            int status = sm_flag, d = ii;
+            if (status & TLI_ROW_NONFINITE) d = -1;
+            else if (ii == INT_MAX) { d = -1; status |= TLI_ROW_FALLBACK; }
+            P.draft_ids[row] = d;
+            if (P.q_out) P.q_out[row] = d >= 0 ? 1.f : 0.f;
+            if (P.status) P.status[row] = status;
+        }
+        return;
+    }
+    // the row's reference, then every strip at that reference
+    cmax = warp_max(cmax);
+    if (lane == 0) sm_wmax[warp] = cmax;
+    __syncthreads();
+    cmax = sm_wmax[0];
+#pragma unroll
+    for (int i = 1; i < kWarps; ++i) cmax = fmaxf(cmax, sm_wmax[i]);
+    double mine = 0.0;
+    for (int i = i0; i < i1; ++i) { const double t = sm_S[i] * pow2_neg_d(sm_c[i] - cmax); sm_S[i] = t; mine += t; }
+    double incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) sm_warp_tot[warp] = incl;
+    __syncthreads();
+    double base = 0.0, R = 0.0;
+#pragma unroll
+    for (int i = 0; i < kWarps; ++i) { if (i < warp) base += sm_warp_tot[i]; R += sm_warp_tot[i]; }
+    int status = 0;
+    if (!isfinite(R)) status = TLI_ROW_NONFINITE;            // a NaN or +inf inside the intersection
+    else if (!(R > 0.0)) status = TLI_ROW_FALLBACK;          // empty intersection, or no mass in it
+    if (status) {
+        if (tid == 0) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = status;
+        }
+        return;
+    }
+    const double target = static_cast<double>(__ldg(P.u + row)) * R;
+    {
+        double run = base + incl - mine;                     // mass before this thread's first strip
+        int cand = INT_MAX, lastpos = -1;
+        for (int i = i0; i < i1; ++i) {
+            const double nx = run + sm_S[i];
+            if (sm_S[i] > 0.0) lastpos = i;
+            if (cand == INT_MAX && nx > target) cand = i;
+            run = nx;
+        }
+        if (cand != INT_MAX) atomicMin(&sm_found, cand);
+        if (lastpos >= 0) atomicMax(&sm_lastpos, lastpos);
+    }
+    __syncthreads();
+    const int found = sm_found;
+    const int T = (found != INT_MAX) ? found : sm_lastpos;   // sm_lastpos >= 0 because R > 0
+    if (T >= i0 && T < i1) {
+        double before = base + incl - mine;
+        for (int i = i0; i < T; ++i) before += sm_S[i];
+        // what is left of the target inside strip T, in the strip's own scale; when rounding left
+        // no strip above the target the walk below ends on the last positive element
+        sm_rem = (found != INT_MAX) ? scale_up(target - before, cmax - sm_c[T]) : INFINITY;
+        sm_total = R;
+    }
+    __syncthreads();
+    if (warp != 0) return;
+
+    // ---- warp 0 walks strip T ----
+    const double rem = sm_rem;
+    const float s = 1.4426950408889634f / tau;
+    const float cT = sm_c[T];
+    const int nvec = rv.nvec();
+    uint4 m[kVecPerThread];
+    float vs[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        uint32_t bits;
+        float w[EPV];
+        m[k] = draft_masked_vector<DT>(P, rv, T * (32 * kVecPerThread) + k * 32 + lane, nvec, bits);
+        vs[k] = draft_vector_sum<DT>(m[k], s, -cT, w);
+    }
+    // vector g = k*32 + lane in address order: mass before it, fp64
+    double carry = 0.0;
+    int cand = INT_MAX, lastpos = -1;
+    double pre_of_cand = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const double mine_v = static_cast<double>(vs[k]);
+        double inc = mine_v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, inc, o);
+            if (lane >= o) inc += up;
+        }
+        const double pre = carry + inc - mine_v;
+        if (vs[k] > 0.f) lastpos = k * 32 + lane;
+        if (cand == INT_MAX && pre + mine_v > rem) { cand = k * 32 + lane; pre_of_cand = pre; }
+        carry += __shfl_sync(0xffffffffu, inc, 31);
+    }
+    const int gfound = __reduce_min_sync(0xffffffffu, cand);
+    const int glast = __reduce_max_sync(0xffffffffu, lastpos);
+    const int G = (gfound != INT_MAX) ? gfound : glast;
+    if (G < 0) {                                             // cannot happen when the strip has positive mass
+        if (lane == 0) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = TLI_ROW_FALLBACK;
+        }
+        return;
+    }
+    if (lane == (G & 31)) {
+        const double rem2 = (gfound != INT_MAX) ? (rem - pre_of_cand) : INFINITY;
+        float w[EPV];
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k)
+            if (k == (G >> 5)) draft_vector_sum<DT>(m[k], s, -cT, w);
+        float runf = 0.f, wp = w[0];
+        int pick = -1, lastw = 0;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+            runf = (i == 0) ? w[0] : __fadd_rn(runf, w[i]);
+            if (w[i] > 0.f) lastw = i;
+            if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
+        }
+        if (pick < 0) pick = lastw;
+#pragma unroll
+        for (int i = 1; i < EPV; ++i) wp = (i == pick) ? w[i] : wp;
+        int id = rv.first_elem(T * (32 * kVecPerThread) + G) + pick;
+        id = min(max(id, 0), P.V_d - 1);
+        P.draft_ids[row] = id;
+        if (P.q_out) P.q_out[row] = static_cast<float>(static_cast<double>(wp) * pow2_neg_d(cT - cmax) / sm_total);
+        if (P.status) P.status[row] = 0;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 6) tli_draft_kernel(const DraftParams P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    __shared__ int sm_last;
     const int row = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int b = row / P.R, r = row - b * P.R;
@@ -1225,65 +1408,71 @@ __global__ void __launch_bounds__(kThreads) tli_draft_kernel(const DraftParams P
         }
         return;
     }
-    const bool greedy = (tau == 0.f);
-    const float s = 1.4426950408889634f / tau;
     const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
     const int nvec = rv.nvec();
-    if (tid == 0) sm_flag = 0;
+    const int strip = tile * kStripsPerTile + warp;
 
-    // ---- this tile ----
-    float z[kVecPerThread][EPV];
-    bool bad = false;
-    float best = -INFINITY; int best_idx = INT_MAX;        // largest logit inside the intersection, lowest id
+    uint4 m[kVecPerThread];
+    uint32_t bits[kVecPerThread];
 #pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = tile * kVecPerTile + k * kThreads + tid;
-        uint32_t bits;
-        draft_vector<DT>(P, rv, v, nvec, z[k], bits, bad);
-        const int e0 = rv.first_elem(v);
+    for (int k = 0; k < kVecPerThread; ++k)
+        m[k] = draft_masked_vector<DT>(P, rv, strip * (32 * kVecPerThread) + k * 32 + lane, nvec, bits[k]);
+    DraftPart pt;
+    if (tau == 0.f) {
+        // largest logit inside the intersection, lowest id; an id inside it counts even at -inf
+        float best = -INFINITY; int idx = INT_MAX; bool bad = false;
 #pragma unroll
-        for (int i = 0; i < EPV; ++i)
-            if (((bits >> i) & 1u) && (best_idx == INT_MAX || z[k][i] > best)) { best = z[k][i]; best_idx = e0 + i; }
-    }
+        for (int k = 0; k < kVecPerThread; ++k) {
+            float z[EPV];
+            unpack<DT>(m[k], z);
+            const int e0 = rv.first_elem(strip * (32 * kVecPerThread) + k * 32 + lane);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        const float b2 = __shfl_xor_sync(0xffffffffu, best, o);
-        const int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
-        if (i2 != INT_MAX && (best_idx == INT_MAX || b2 > best || (b2 == best && i2 < best_idx))) { best = b2; best_idx = i2; }
-    }
-    if (lane == 0) { sm_max[warp] = best; sm_idx[warp] = best_idx; }
-    __syncthreads();
-    if (bad) atomicOr(&sm_flag, static_cast<int>(TLI_ROW_NONFINITE));
-    best = sm_max[0]; best_idx = sm_idx[0];
+            for (int i = 0; i < EPV; ++i)
+                if ((bits[k] >> i) & 1u) {
+                    bad = bad || !(z[i] < INFINITY);
+                    if (idx == INT_MAX || z[i] > best) { best = z[i]; idx = e0 + i; }
+                }
+        }
 #pragma unroll
-    for (int i = 1; i < kWarps; ++i) {
-        const float b2 = sm_max[i]; const int i2 = sm_idx[i];
-        if (i2 != INT_MAX && (best_idx == INT_MAX || b2 > best || (b2 == best && i2 < best_idx))) { best = b2; best_idx = i2; }
-    }
-    const float c_tile = (best_idx == INT_MAX) ? kNegBig : reference_for(best * s);
-    double acc = 0.0;
-    if (!greedy) {
+        for (int o = 16; o > 0; o >>= 1) {
+            const float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+            const int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+            if (better(b2, i2, best, idx)) { best = b2; idx = i2; }
+        }
+        pt.S = static_cast<double>(idx); pt.c = best;
+        pt.flags = __any_sync(0xffffffffu, bad) ? static_cast<int>(TLI_ROW_NONFINITE) : 0;
+    } else {
+        const float s = 1.4426950408889634f / tau;
+        float mx;
+        if constexpr (DT == TLI_BF16) {
+            uint32_t mm = bf16x2_max(bf16x2_max(m[0].x, m[0].y), bf16x2_max(m[0].z, m[0].w));
+#pragma unroll
+            for (int k = 1; k < kVecPerThread; ++k)
+                mm = bf16x2_max(mm, bf16x2_max(bf16x2_max(m[k].x, m[k].y), bf16x2_max(m[k].z, m[k].w)));
+            mx = fmaxf(bf16_lo(mm), bf16_hi(mm));
+        } else {
+            mx = -INFINITY;
+#pragma unroll
+            for (int k = 0; k < kVecPerThread; ++k)
+                mx = fmaxf(mx, fmaxf(fmaxf(__uint_as_float(m[k].x), __uint_as_float(m[k].y)),
+                                     fmaxf(__uint_as_float(m[k].z), __uint_as_float(m[k].w))));
+        }
+        const float c = reference_for(warp_max(mx) * s);
+        double acc = 0.0;
 #pragma unroll
         for (int k = 0; k < kVecPerThread; ++k) {
             float w[EPV];
-            draft_weights(z[k], s, -c_tile, w);
-            acc += static_cast<double>(ordered_sum(w));
+            acc += static_cast<double>(draft_vector_sum<DT>(m[k], s, -c, w));
         }
+        pt.S = warp_sum(acc); pt.c = c; pt.flags = 0;
     }
-    acc = warp_sum(acc);
-    if (lane == 0) sm_red[warp] = acc;
+    if (lane == 0 && strip < P.nstrip) {
+        store_part(P.part + static_cast<size_t>(row) * P.nstrip + strip, pt);
+        if (!P.split) __threadfence();
+    }
+    if (P.split) return;
     __syncthreads();
     if (tid == 0) {
-        double tot = 0.0;
-#pragma unroll
-        for (int i = 0; i < kWarps; ++i) tot += sm_red[i];
-        DraftPart pt;
-        pt.S = greedy ? static_cast<double>(best_idx) : tot;
-        pt.c = greedy ? best : c_tile;
-        pt.flags = sm_flag;
-        DraftPart *dst = P.part + static_cast<size_t>(row) * P.ntile + tile;
-        __stcg(reinterpret_cast<double2 *>(dst), *reinterpret_cast<const double2 *>(&pt));
-        __threadfence();
         const unsigned ticket = atomicAdd(P.cnt + row, 1u);
         sm_last = (ticket == static_cast<unsigned>(P.ntile) - 1);
         if (sm_last) P.cnt[row] = 0;
@@ -1291,150 +1480,20 @@ __global__ void __launch_bounds__(kThreads) tli_draft_kernel(const DraftParams P
     __syncthreads();
     if (!sm_last) return;
     __threadfence();
+    draft_select<DT>(P, row, rv, tau);
+}
 
-    // ---- last CTA of the row: pick the id ----
-    const int ntile = P.ntile;
-    if (tid == 0) { sm_flag = 0; sm_none = 0; }
-    __syncthreads();
-    for (int i = tid; i < ntile; i += kThreads) {
-        const double2 raw = __ldcg(reinterpret_cast<const double2 *>(P.part + static_cast<size_t>(row) * ntile + i));
-        const DraftPart pt = *reinterpret_cast<const DraftPart *>(&raw);
-        sm_tiles[i] = pt.S; sm_ref[i] = pt.c;
-        if (pt.flags) atomicOr(&sm_flag, pt.flags);
-    }
-    __syncthreads();
-    int status = sm_flag;
-    if (greedy) {
-        if (tid == 0) {
-            float bb = -INFINITY; int ii = INT_MAX;
-            for (int i = 0; i < ntile; ++i) {               // tiles in increasing id order: strict > keeps the lowest id
-                const int i2 = static_cast<int>(sm_tiles[i]);
-                if (i2 != INT_MAX && (ii == INT_MAX || sm_ref[i] > bb)) { bb = sm_ref[i]; ii = i2; }
-            }
-            int d = ii;
-            if (status & TLI_ROW_NONFINITE) d = -1;
-            else if (ii == INT_MAX) { d = -1; status |= TLI_ROW_FALLBACK; }
-            P.draft_ids[row] = d;
-            if (P.q_out) P.q_out[row] = d >= 0 ? 1.f : 0.f;
-            if (P.status) P.status[row] = status;
-        }
-        return;
-    }
-    if (tid == 0) {
-        float cmax = kNegBig;
-        for (int i = 0; i < ntile; ++i) cmax = fmaxf(cmax, sm_ref[i]);
-        double R = 0.0;
-        for (int i = 0; i < ntile; ++i) { sm_tiles[i] *= pow2_neg_d(sm_ref[i] - cmax); R += sm_tiles[i]; }
-        if ((status & TLI_ROW_NONFINITE) || !isfinite(R)) { status |= TLI_ROW_NONFINITE; sm_none = 1; }
-        else if (!(R > 0.0)) { status |= TLI_ROW_FALLBACK; sm_none = 1; }
-        else {
-            const double target = static_cast<double>(__ldg(P.u + row)) * R;
-            double run = 0.0, before = 0.0;
-            int T = -1, lastpos = 0;
-            for (int i = 0; i < ntile; ++i) {
-                const double nx = run + sm_tiles[i];
-                if (sm_tiles[i] > 0.0) lastpos = i;
-                if (T < 0 && nx > target) { T = i; before = run; }
-                run = nx;
-            }
-            if (T < 0) { T = lastpos; before = R - sm_tiles[lastpos]; }
-            sm_tile = T;
-            sm_rem = scale_up(target - before, cmax - sm_ref[T]);     // in the tile's own scale
-            sm_total = R; sm_cmax = cmax;
-        }
-        if (sm_none) {
-            P.draft_ids[row] = -1;
-            if (P.q_out) P.q_out[row] = 0.f;
-            if (P.status) P.status[row] = status;
-        }
-        sm_found = INT_MAX; sm_lastpos = -1;
-    }
-    __syncthreads();
-    if (sm_none) return;
-    const int T = sm_tile;
-    const double rem = sm_rem;
-    const float nc = -sm_ref[T];
-    // vector sums of tile T in address order, by the code that formed the tile's sum
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int g = k * kThreads + tid;
-        const int v = T * kVecPerTile + g;
-        float zz[EPV], w[EPV];
-        uint32_t bits; bool ignore = false;
-        draft_vector<DT>(P, rv, v, nvec, zz, bits, ignore);
-        draft_weights(zz, s, nc, w);
-        sm_seg[g] = ordered_sum(w);
-    }
-    __syncthreads();
-    // thread i owns vectors 4i .. 4i+3: block-wide exclusive prefix in fp64
-    double loc[kVecPerThread];
-    double mine = 0.0;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) { loc[k] = static_cast<double>(sm_seg[tid * kVecPerThread + k]); mine += loc[k]; }
-    double incl = mine;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-        const double up = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += up;
-    }
-    if (lane == 31) sm_warp_tot[warp] = incl;
-    __syncthreads();
-    double base = 0.0;
-    for (int i = 0; i < warp; ++i) base += sm_warp_tot[i];
-    double run = base + incl - mine;                       // mass before this thread's first vector
-    int cand = INT_MAX, lastpos = -1;
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const double nx = run + loc[k];
-        if (loc[k] > 0.0) lastpos = tid * kVecPerThread + k;
-        if (cand == INT_MAX && nx > rem) cand = tid * kVecPerThread + k;
-        run = nx;
-    }
-    if (cand != INT_MAX) atomicMin(&sm_found, cand);
-    if (lastpos >= 0) atomicMax(&sm_lastpos, lastpos);
-    __syncthreads();
-    const int found = sm_found;
-    const int G = (found != INT_MAX) ? found : sm_lastpos;
-    if (G < 0) {                                           // cannot happen when the tile has positive mass
-        if (tid == 0) {
-            P.draft_ids[row] = -1;
-            if (P.q_out) P.q_out[row] = 0.f;
-            if (P.status) P.status[row] = status | TLI_ROW_FALLBACK;
-        }
-        return;
-    }
-    if (tid == G / kVecPerThread) {
-        // walk the elements of vector G with the running fp32 sum that formed its total; when
-        // rounding left no vector above the target, take the last positive element instead
-        double before = 0.0;
-        if (found != INT_MAX) {
-            before = base + incl - mine;
-            for (int k = 0; k < G - tid * kVecPerThread; ++k) before += loc[k];
-        }
-        const double rem2 = (found != INT_MAX) ? (rem - before) : INFINITY;
-        const int v = T * kVecPerTile + G;
-        float zz[EPV], w[EPV];
-        uint32_t bits; bool ignore = false;
-        draft_vector<DT>(P, rv, v, nvec, zz, bits, ignore);
-        draft_weights(zz, s, nc, w);
-        float runf = 0.f;
-        int pick = -1, lastw = 0;
-#pragma unroll
-        for (int i = 0; i < EPV; ++i) {
-            runf = (i == 0) ? w[0] : __fadd_rn(runf, w[i]);
-            if (w[i] > 0.f) lastw = i;
-            if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
-        }
-        if (pick < 0) pick = lastw;
-        float wp = w[0];
-#pragma unroll
-        for (int i = 1; i < EPV; ++i) wp = (i == pick) ? w[i] : wp;
-        int id = rv.first_elem(v) + pick;
-        id = min(max(id, 0), P.V_d - 1);
-        P.draft_ids[row] = id;
-        if (P.q_out) P.q_out[row] = static_cast<float>(static_cast<double>(wp) * pow2_neg_d(sm_ref[T] - sm_cmax) / sm_total);
-        if (P.status) P.status[row] = status;
-    }
+// Large batches: the selections as a kernel of their own, one CTA per row, so that the tile CTAs
+// carry neither a fence nor a ticket.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_draft_select_kernel(const DraftParams P) {
+    const int row = blockIdx.x;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int b = row / P.R, r = row - b * P.R;
+    const float tau = __ldg(P.tau + b);
+    if (!(tau >= 0.f) || isinf(tau)) return;                 // the tile kernel has written this row
+    const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
+    draft_select<DT>(P, row, rv, tau);
 }
 
 // ---------------------------------------------------------------------------
@@ -2385,8 +2444,8 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream) {
 size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32_t dtype) {
     if (!ctx || B < 1 || R < 1 || static_cast<long long>(B) * R > TLI_MAX_B) return 0;
     if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
-    const size_t ntile = static_cast<size_t>(chunks_per_row(ctx->V_d, dtype, kVecPerTile));
-    return align_up(sizeof(DraftPart) * static_cast<size_t>(B) * R * ntile, 256);
+    const size_t nstrip = static_cast<size_t>(chunks_per_row(ctx->V_d, dtype, kVecPerTile)) * kStripsPerTile;
+    return align_up(sizeof(DraftPart) * static_cast<size_t>(B) * R * nstrip, 256);
 }
 
 int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *a, void *cuda_stream) {
@@ -2404,17 +2463,33 @@ int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *a, void *cuda_stream) {
     DraftParams P;
     P.B = a->B; P.R = a->R; P.V_d = ctx->V_d;
     P.ntile = chunks_per_row(ctx->V_d, a->dtype, kVecPerTile);
+    P.nstrip = P.ntile * kStripsPerTile;
+    const int rows = a->B * a->R;
+    // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
+    P.split = (static_cast<long long>(rows) * P.ntile >= 4096) ? 1 : 0;
     P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sr = a->d_stride_r;
     P.maskbits = ctx->d_mask; P.tau = a->temperature; P.u = a->uniforms;
     P.draft_ids = a->draft_ids; P.q_out = a->q_draft; P.status = a->draft_status;
     P.part = reinterpret_cast<DraftPart *>(a->workspace);
     P.cnt = ctx->d_counters + (TLI_MAX_B + 1);           // the sampling pass's tickets: zero between calls
-    const dim3 grid(static_cast<unsigned>(P.ntile), static_cast<unsigned>(a->B * a->R));
+    const dim3 grid(static_cast<unsigned>(P.ntile), static_cast<unsigned>(rows));
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (a->dtype == TLI_F32) tli_draft_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(P);
     else tli_draft_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(P);
-    const cudaError_t e = cudaGetLastError();
+    cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_kernel");
+    if (P.split) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.gridDim = dim3(static_cast<unsigned>(rows)); cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = 0; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+        if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_F32>, P);
+        else e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_BF16>, P);
+        if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_select_kernel");
+    }
     return TLI_OK;
 }
 

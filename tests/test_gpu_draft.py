@@ -158,16 +158,22 @@ def test_empty_intersection_bad_temperature_and_nonfinite_rows():
     bad = run_gpu(z, id_map, [-1.0, np.nan, np.inf, 1.0], u, V_t)
     np.testing.assert_array_equal(bad["draft_ids"][:3], -1)
     assert (bad["draft_status"][:3] == tli.TLI_ROW_BAD_TEMPERATURE).all() and (bad["draft_status"][3] == 0).all()
-    z2 = z.copy()
-    z2[1, 0, 77] = np.nan
-    z2[2, 1, 4999] = np.inf
-    nf = run_gpu(z2, id_map, tau, u, V_t)
-    assert nf["draft_ids"][1, 0] == -1 and nf["draft_status"][1, 0] == tli.TLI_ROW_NONFINITE
-    assert nf["draft_ids"][2, 1] == -1 and nf["draft_status"][2, 1] == tli.TLI_ROW_NONFINITE
-    ok = np.ones((4, 2), bool)
-    ok[1, 0] = ok[2, 1] = False
+    inside, outside = np.flatnonzero(id_map >= 0), np.flatnonzero(id_map < 0)
     ref = run_gpu(z, id_map, tau, u, V_t)
-    np.testing.assert_array_equal(nf["draft_ids"][ok], ref["draft_ids"][ok])
+    z2 = z.copy()
+    z2[1, 0, inside[7]] = np.nan
+    z2[2, 1, inside[-1]] = np.inf
+    z2[0, 0, outside[3]] = np.nan             # outside the intersection: does not enter q', is not examined
+    z2[3, 1, outside[-1]] = np.inf
+    for t in (tau, np.zeros(4, np.float32)):
+        nf = run_gpu(z2, id_map, t, u, V_t)
+        assert nf["draft_ids"][1, 0] == -1 and nf["draft_status"][1, 0] == tli.TLI_ROW_NONFINITE
+        assert nf["draft_ids"][2, 1] == -1 and nf["draft_status"][2, 1] == tli.TLI_ROW_NONFINITE
+        ok = np.ones((4, 2), bool)
+        ok[1, 0] = ok[2, 1] = False
+        assert (nf["draft_status"][ok] == 0).all()
+        if t is tau:
+            np.testing.assert_array_equal(nf["draft_ids"][ok], ref["draft_ids"][ok])
 
 
 def test_minus_infinity_is_a_token_of_probability_zero():
