@@ -2,7 +2,7 @@
 
 ctypes front end of the fp64 CPU oracle in ``tli_oracle.c`` (Algorithms 4 and 5
 of the paper: ``verify`` for the verification half, ``draft`` for drawing the
-draft ids from q').  Only tests, the smoke check and the benchmark's CPU-baseline
+draft ids from q') and of Algorithm 2's exact-match verification (``slem``).  Only tests, the smoke check and the benchmark's CPU-baseline
 legs may import this package; the CUDA library never does, and this package
 imports nothing from it.
 """
@@ -59,6 +59,18 @@ class _DraftArgs(ctypes.Structure):
     ]
 
 
+class _SlemArgs(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("M", ctypes.c_int32), ("V_t", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("candidates", ctypes.c_void_p), ("lengths", ctypes.c_void_p),
+        ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p), ("probe_token", ctypes.c_void_p),
+        ("sampled", ctypes.c_void_p), ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p), ("cdf_lo", ctypes.c_void_p), ("cdf_hi", ctypes.c_void_p),
+        ("probe_lo", ctypes.c_void_p), ("probe_hi", ctypes.c_void_p), ("probe_w", ctypes.c_void_p),
+    ]
+
+
 def build(force: bool = False) -> str:
     """Compile ``tli_oracle.c`` with gcc -O2 into ``liboracle.so`` beside it."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
@@ -82,6 +94,8 @@ def _load():
         lib.oracle_tli_distributions.restype = ctypes.c_int
         lib.oracle_tli_draft.argtypes = [ctypes.POINTER(_DraftArgs), ctypes.c_int32, ctypes.c_int32]
         lib.oracle_tli_draft.restype = ctypes.c_int
+        lib.oracle_slem_verify.argtypes = [ctypes.POINTER(_SlemArgs), ctypes.c_int32, ctypes.c_int32]
+        lib.oracle_slem_verify.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -238,6 +252,58 @@ def draft(drafter_logits, id_map, temperature, uniforms, probe_id=None, threads:
         rc = lib.oracle_tli_draft(ctypes.byref(args), lo_hi[0], lo_hi[1])
         if rc != 0:
             raise RuntimeError("oracle_tli_draft failed with code %d" % rc)
+
+    if threads == 1:
+        run((0, B))
+    else:
+        cuts = [(B * i) // threads for i in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(run, [(cuts[i], cuts[i + 1]) for i in range(threads)]))
+    return out
+
+
+def slem(target_logits, candidates, temperature, uniforms, lengths=None, probe_token=None,
+         threads: int = 1) -> Dict[str, np.ndarray]:
+    """Algorithm 2's verification: sample t'_j from each of the M+1 target rows, first mismatch with
+    ``candidates`` (int32 [B,M], the re-tokenised drafts).  Returns ``sampled`` (int32 [B,M+1]),
+    ``accepted``, ``next_token``, ``flags`` (int32 [B]), ``cdf_lo``, ``cdf_hi`` (float64 [B,M+1]) and,
+    with ``probe_token`` (int32 [B,M+1]), ``probe_lo/hi/w``."""
+    lib = _load()
+    zt = np.asarray(target_logits)
+    if zt.dtype == np.float32:
+        dtype = F32
+    elif zt.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must be float32 or uint16 bfloat16 bit patterns")
+    if zt.ndim != 3 or zt.strides[2] != zt.itemsize:
+        raise ValueError("target logits must be [B,M+1,V_t] with a contiguous vocabulary axis")
+    B, M1, V_t = zt.shape
+    M = M1 - 1
+    cand = np.ascontiguousarray(candidates, dtype=np.int32).reshape(B, M)
+    tau = np.ascontiguousarray(temperature, dtype=np.float32).reshape(B)
+    u = np.ascontiguousarray(uniforms, dtype=np.float32).reshape(B, M + 1)
+    ln = None if lengths is None else np.ascontiguousarray(lengths, dtype=np.int32).reshape(B)
+    probe = None if probe_token is None else np.ascontiguousarray(probe_token, dtype=np.int32).reshape(B, M + 1)
+    out: Dict[str, np.ndarray] = {
+        "sampled": np.zeros((B, M + 1), np.int32), "accepted": np.zeros(B, np.int32),
+        "next_token": np.zeros(B, np.int32), "flags": np.zeros(B, np.int32),
+        "cdf_lo": np.zeros((B, M + 1), np.float64), "cdf_hi": np.zeros((B, M + 1), np.float64),
+    }
+    if probe is not None:
+        out.update(probe_lo=np.zeros((B, M + 1), np.float64), probe_hi=np.zeros((B, M + 1), np.float64),
+                   probe_w=np.zeros((B, M + 1), np.float64))
+    args = _SlemArgs(B, M, V_t, dtype, zt.ctypes.data, zt.strides[0] // zt.itemsize, zt.strides[1] // zt.itemsize,
+                     _ptr(cand), _ptr(ln), _ptr(tau), _ptr(u), _ptr(probe),
+                     _ptr(out["sampled"]), _ptr(out["accepted"]), _ptr(out["next_token"]), _ptr(out["flags"]),
+                     _ptr(out["cdf_lo"]), _ptr(out["cdf_hi"]),
+                     _ptr(out.get("probe_lo")), _ptr(out.get("probe_hi")), _ptr(out.get("probe_w")))
+    threads = max(1, min(int(threads), B))
+
+    def run(lo_hi):
+        rc = lib.oracle_slem_verify(ctypes.byref(args), lo_hi[0], lo_hi[1])
+        if rc != 0:
+            raise RuntimeError("oracle_slem_verify failed with code %d" % rc)
 
     if threads == 1:
         run((0, B))

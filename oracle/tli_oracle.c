@@ -40,7 +40,9 @@
  * fusion or reordering.
  *
  * The file also holds the drafting side of the same algorithms
- * (oracle_tli_draft, at the end): drawing the draft ids from q'.
+ * (oracle_tli_draft): drawing the draft ids from q', and the verification step
+ * of Algorithm 2, exact matching against sampled target tokens
+ * (oracle_slem_verify); both at the end.
  *
  * Parity status: every function here is pinned by tests that do not use this
  * file's own formulas (worked example, brute-force losslessness on tiny
@@ -487,5 +489,117 @@ int oracle_tli_draft(const oracle_draft_args *a, int32_t row_begin, int32_t row_
         if (a->flags) a->flags[b] = flags;
     }
     free(q); free(qp);
+    return 0;
+}
+
+/*
+ * Algorithm 2 (string-level exact matching), the part after the drafts have
+ * been re-tokenised into target ids t_1..t_m: sample t'_j from each of the
+ * m+1 target rows (p_j = softmax(row j / tau); inverse CDF in increasing
+ * target-id order with the uniform u[b, j]; tau == 0: the lowest id attaining
+ * the maximum), find the first j with t'_j != t_j (j = m+1 if none), accept
+ * t_1..t_{j-1} and emit t'_j.  accepted = j-1 in [0, m], next_token = t'_j.
+ * Sequences may have different m (lengths[b] <= M); rows beyond m are not
+ * sampled (-1).  A non-finite logit in a row that is sampled, or an invalid
+ * temperature, flags the sequence (accepted = 0, next_token = 0).  Parity
+ * status: pinned by a chi-square of the sampled ids against the softmax, by
+ * the closed-form match probability p_j(t_j), by numpy's cumulative-sum
+ * search, by brute force over all candidate strings on a tiny vocabulary, and
+ * at tau == 0 by agreement with the verification oracle under an identity map.
+ */
+typedef struct {
+    int32_t B, M, V_t, dtype;
+    const void *target_logits;  /* [B, M+1, V_t], strides in elements */
+    int64_t t_stride_b, t_stride_k;
+    const int32_t *candidates;  /* [B, M] target ids of the re-tokenised drafts */
+    const int32_t *lengths;     /* [B] m_b in [0, M], or NULL for m_b = M */
+    const float *temperature;   /* [B] */
+    const float *uniforms;      /* [B, M+1] */
+    const int32_t *probe_token; /* [B, M+1] or NULL */
+    /* outputs */
+    int32_t *sampled;           /* [B, M+1] t'_j; -1 for rows that are not sampled */
+    int32_t *accepted;          /* [B] */
+    int32_t *next_token;        /* [B] */
+    int32_t *flags;             /* [B] */
+    double *cdf_lo, *cdf_hi;    /* [B, M+1] normalised CDF around t'_j */
+    double *probe_lo, *probe_hi, *probe_w; /* [B, M+1] (only if probe_token) */
+} oracle_slem_args;
+
+int oracle_slem_verify(const oracle_slem_args *a, int32_t row_begin, int32_t row_end)
+{
+    if (!a || a->B < 1 || a->M < 0 || a->V_t < 1) return -1;
+    if (a->dtype != ORACLE_F32 && a->dtype != ORACLE_BF16) return -1;
+    if (row_begin < 0 || row_end > a->B || row_begin > row_end) return -1;
+    const int V = a->V_t, M = a->M;
+    double *p = (double *)malloc(sizeof(double) * (size_t)V);
+    if (!p) return -3;
+    for (int b = row_begin; b < row_end; ++b) {
+        const double tau = (double)a->temperature[b];
+        int m = a->lengths ? a->lengths[b] : M;
+        int flags = 0;
+        if (m < 0) m = 0;
+        if (m > M) m = M;
+        for (int j = 0; j <= M; ++j) {
+            const int64_t o = (int64_t)b * (M + 1) + j;
+            a->sampled[o] = -1;
+            if (a->cdf_lo) a->cdf_lo[o] = 0.0;
+            if (a->cdf_hi) a->cdf_hi[o] = 0.0;
+        }
+        if (!(tau >= 0.0) || isinf(tau)) flags |= FLAG_BAD_TEMPERATURE;
+        for (int j = 0; j <= m && !flags; ++j) {
+            const int64_t o = (int64_t)b * (M + 1) + j;
+            const int64_t off = (int64_t)b * a->t_stride_b + (int64_t)j * a->t_stride_k;
+            if (tau == 0.0) {
+                int finite = 1;
+                for (int t = 0; t < V; ++t)
+                    if (!isfinite(load_logit(a->target_logits, a->dtype, off + t))) finite = 0;
+                if (!finite) { flags |= FLAG_NONFINITE; break; }
+                a->sampled[o] = argmax_row(a->target_logits, a->dtype, off, V);
+                if (a->cdf_hi) a->cdf_hi[o] = 1.0;
+                continue;
+            }
+            if (!softmax_row(a->target_logits, a->dtype, off, V, tau, p)) { flags |= FLAG_NONFINITE; break; }
+            double total = 0.0;
+            for (int t = 0; t < V; ++t) total += p[t];
+            const double target = (double)a->uniforms[o] * total;
+            double C = 0.0, C_before = 0.0, hi = 1.0;
+            int found = -1, last_pos = 0;
+            for (int t = 0; t < V; ++t) {
+                double Cn = C + p[t];
+                if (p[t] > 0.0) last_pos = t;
+                if (found < 0 && Cn > target) { found = t; C_before = C; hi = Cn / total; }
+                C = Cn;
+            }
+            if (found < 0) { found = last_pos; C_before = C - p[last_pos]; hi = 1.0; }
+            a->sampled[o] = found;
+            if (a->cdf_lo) a->cdf_lo[o] = C_before / total;
+            if (a->cdf_hi) a->cdf_hi[o] = hi;
+            if (a->probe_token) {
+                int g = a->probe_token[o];
+                double plo = 0.0, phi = 0.0, pw = 0.0;
+                if (g >= 0 && g < V) {
+                    double Cc = 0.0;
+                    for (int t = 0; t < g; ++t) Cc += p[t];
+                    plo = Cc / total; phi = (Cc + p[g]) / total; pw = p[g] / total;
+                }
+                if (a->probe_lo) a->probe_lo[o] = plo;
+                if (a->probe_hi) a->probe_hi[o] = phi;
+                if (a->probe_w) a->probe_w[o] = pw;
+            }
+        }
+        int n = 0, next = 0;
+        if (!flags) {
+            n = m;
+            for (int j = 0; j < m; ++j)
+                if (a->sampled[(int64_t)b * (M + 1) + j] != a->candidates[(int64_t)b * M + j]) { n = j; break; }
+            next = a->sampled[(int64_t)b * (M + 1) + n];
+        } else {
+            for (int j = 0; j <= M; ++j) a->sampled[(int64_t)b * (M + 1) + j] = -1;
+        }
+        a->accepted[b] = n;
+        a->next_token[b] = next;
+        if (a->flags) a->flags[b] = flags;
+    }
+    free(p);
     return 0;
 }
