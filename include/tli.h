@@ -236,6 +236,55 @@ size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32
  */
 int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *args, void *cuda_stream);
 
+typedef struct {
+    int32_t B;      /* sequences, >= 1 */
+    int32_t M;      /* re-tokenised drafts per sequence (at most), 0 .. TLI_MAX_K; B * (M+1) <= TLI_MAX_B */
+    int32_t dtype;  /* TLI_F32 or TLI_BF16 */
+
+    /* [device] target logits [B, M+1, V_t]: row j is the target distribution
+     * after the prompt and candidates t_1 .. t_j (Algorithm 2's single
+     * batched target pass).  Strides in elements; vocabulary axis contiguous. */
+    const void *target_logits;
+    int64_t t_stride_b, t_stride_k;
+
+    const int32_t *candidates;  /* [device] int32[B, M]: the drafts re-tokenised into target ids t_1 .. t_m */
+    const int32_t *lengths;     /* [device] int32[B]: m_b in [0, M] (re-tokenisation gives each sequence its
+                                 * own count); NULL = M for all.  Rows beyond m_b are not read */
+    const float *temperature;   /* [device] float[B]; 0 = arg-max */
+    const float *uniforms;      /* [device] float[B, M+1] in [0, 1): one per target row */
+
+    int32_t *accepted;          /* [device] out int32[B]: matched candidates, 0 .. m_b */
+    int32_t *next_token;        /* [device] out int32[B]: the sampled token at the first mismatch
+                                 * (the bonus token t'_{m+1} when all m_b match) */
+    int32_t *sampled;           /* [device] out int32[B, M+1]: every sampled token t'_j, -1 for rows
+                                 * beyond m_b and for flagged sequences; may be NULL */
+    int32_t *row_status;        /* [device] out int32[B] of TLI_ROW_* bits (NONFINITE, FALLBACK = a row
+                                 * without mass, BAD_TEMPERATURE); may be NULL */
+
+    void *workspace;            /* [device] scratch, 256-byte aligned, >= tli_slem_workspace_bytes() */
+    size_t workspace_bytes;
+} tli_slem_args;
+
+/* Bytes of device scratch tli_slem_verify() needs for (B, M, dtype); 0 on bad arguments. */
+size_t tli_slem_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t M, int32_t dtype);
+
+/*
+ * Exact-match verification, the device part of Algorithm 2 (string-level exact
+ * matching): the drafts have been decoded to text and re-tokenised into target
+ * ids t_1 .. t_m by the caller; this call samples a token t'_j from each of
+ * the m+1 target rows (p_j = softmax(row j / tau), inverse CDF in increasing
+ * target-id order with uniforms[b,j]; tau == 0: the lowest id attaining the
+ * maximum), finds the first j with t'_j != t_j and reports accepted = j - 1
+ * and next_token = t'_j (j = m+1, the bonus token, if every candidate
+ * matched).  The id map of the context plays no part; rows have the context's
+ * V_t entries.  One pass over the logits of rows 0 .. m_b; arithmetic and the
+ * handling of -inf / NaN / +inf as in tli_verify().  A flagged sequence
+ * reports accepted = 0, next_token = 0.  Asynchronous on the stream, allocates
+ * nothing, uses the context's counters (no overlap with another call on the
+ * same context).  Errors as for tli_verify().
+ */
+int tli_slem_verify(tli_ctx *ctx, const tli_slem_args *args, void *cuda_stream);
+
 /*
  * Measurement hook: the three-kernel form of tli_verify() (see tli_set_fused)
  * with CUDA events recorded on `cuda_stream` around each kernel.  Blocks until

@@ -1165,9 +1165,10 @@ struct __align__(16) DraftPart {
     int flags;     // temperature 0: TLI_ROW_NONFINITE if an id inside the intersection holds NaN or +inf
 };
 struct DraftParams {
-    int B, R, V_d, ntile, nstrip, split;
+    int B, R, V_d, ntile, nstrip, split;     // V_d: length of a row (the target vocabulary when no mask is given)
     const void *zd; long long d_sb, d_sr;
-    const uint32_t *maskbits;
+    const uint32_t *maskbits;                // ids that can be drawn; NULL: every id of the row
+    const int *lengths;                      // NULL, or per sequence the last row to sample (rows beyond it get -1)
     const float *tau; const float *u;
     int *draft_ids; float *q_out; int *status;
     DraftPart *part;               // [B*R][nstrip]
@@ -1182,7 +1183,15 @@ __device__ __forceinline__ uint4 draft_masked_vector(const DraftParams &P, const
     bits = 0u;
     if (v >= nvec) return make_uint4(NI, NI, NI, NI);
     uint4 raw = rv.load(v);
-    bits = mask_bits(P.maskbits, rv.first_elem(v));
+    const int e0 = rv.first_elem(v);
+    if (P.maskbits == nullptr) {                           // no mask: the elements inside the row (load() gave -inf elsewhere)
+        constexpr int EPV = Elt<DT>::kPerVec;
+        bits = (1u << EPV) - 1u;
+        if (e0 < 0) bits &= ~((1u << (-e0)) - 1u);
+        if (e0 + EPV > rv.V) bits &= (1u << (rv.V - e0)) - 1u;
+        return raw;
+    }
+    bits = mask_bits(P.maskbits, e0);
     if constexpr (DT == TLI_BF16) {
         mask_bf16_vector(raw, bits);
     } else {
@@ -1408,6 +1417,14 @@ __global__ void __launch_bounds__(kThreads, 6) tli_draft_kernel(const DraftParam
         }
         return;
     }
+    if (P.lengths && r > __ldg(P.lengths + b)) {               // not a row of this sequence
+        if (tile == 0 && tid == 0) {
+            P.draft_ids[row] = -1;
+            if (P.q_out) P.q_out[row] = 0.f;
+            if (P.status) P.status[row] = 0;
+        }
+        return;
+    }
     const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
     const int nvec = rv.nvec();
     const int strip = tile * kStripsPerTile + warp;
@@ -1492,8 +1509,43 @@ __global__ void __launch_bounds__(kThreads) tli_draft_select_kernel(const DraftP
     const int b = row / P.R, r = row - b * P.R;
     const float tau = __ldg(P.tau + b);
     if (!(tau >= 0.f) || isinf(tau)) return;                 // the tile kernel has written this row
+    if (P.lengths && r > __ldg(P.lengths + b)) return;       // this one too
     const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
     draft_select<DT>(P, row, rv, tau);
+}
+
+// Algorithm 2's comparison: the drafts re-tokenised into target ids against the tokens sampled from
+// the target rows; one thread per sequence.
+struct SlemParams {
+    int B, M;
+    const int *candidates; const int *lengths; const float *tau;
+    int *sampled;              // [B, M+1], written by the sampling kernels
+    const int *row_flags;      // [B, M+1]
+    int *accepted; int *next_token; int *status;
+};
+__global__ void __launch_bounds__(128) tli_slem_match_kernel(const SlemParams P) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= P.B) return;
+    const float tau = __ldg(P.tau + b);
+    int m = P.lengths ? __ldg(P.lengths + b) : P.M;
+    m = min(max(m, 0), P.M);
+    int *t = P.sampled + static_cast<size_t>(b) * (P.M + 1);
+    int flags = 0;
+    if (!(tau >= 0.f) || isinf(tau)) flags = TLI_ROW_BAD_TEMPERATURE;
+    else for (int j = 0; j <= m; ++j) flags |= __ldcg(P.row_flags + static_cast<size_t>(b) * (P.M + 1) + j);
+    int n = 0, next = 0;
+    if (flags) {
+        for (int j = 0; j <= P.M; ++j) t[j] = -1;
+    } else {
+        n = m;
+        for (int j = 0; j < m; ++j)
+            if (__ldcg(t + j) != __ldg(P.candidates + static_cast<size_t>(b) * P.M + j)) { n = j; break; }
+        next = __ldcg(t + n);
+    }
+    P.accepted[b] = n;
+    P.next_token[b] = next;
+    if (P.status) P.status[b] = flags;
 }
 
 // ---------------------------------------------------------------------------
@@ -2448,6 +2500,33 @@ size_t tli_draft_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t R, int32
     return align_up(sizeof(DraftPart) * static_cast<size_t>(B) * R * nstrip, 256);
 }
 
+// The sampling kernels on `rows` = B * R rows: tiles, then (large batches) the selections.
+static int launch_row_sampler(DraftParams &P, int dtype, cudaStream_t stream) {
+    const int rows = P.B * P.R;
+    P.ntile = chunks_per_row(P.V_d, dtype, kVecPerTile);
+    P.nstrip = P.ntile * kStripsPerTile;
+    // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
+    P.split = (static_cast<long long>(rows) * P.ntile >= 4096) ? 1 : 0;
+    const dim3 grid(static_cast<unsigned>(P.ntile), static_cast<unsigned>(rows));
+    if (dtype == TLI_F32) tli_draft_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(P);
+    else tli_draft_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(P);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_kernel");
+    if (P.split) {
+        cudaLaunchConfig_t cfg;
+        memset(&cfg, 0, sizeof cfg);
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.gridDim = dim3(static_cast<unsigned>(rows)); cfg.blockDim = dim3(kThreads);
+        cfg.dynamicSmemBytes = 0; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+        if (dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_F32>, P);
+        else e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_BF16>, P);
+        if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_select_kernel");
+    }
+    return TLI_OK;
+}
+
 int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *a, void *cuda_stream) {
     if (!ctx || !a) return TLI_ERR_ARG;
     if (a->B < 1 || a->R < 1) return TLI_ERR_ARG;
@@ -2462,34 +2541,74 @@ int tli_draft_sample(tli_ctx *ctx, const tli_draft_args *a, void *cuda_stream) {
         return TLI_ERR_WORKSPACE;
     DraftParams P;
     P.B = a->B; P.R = a->R; P.V_d = ctx->V_d;
-    P.ntile = chunks_per_row(ctx->V_d, a->dtype, kVecPerTile);
-    P.nstrip = P.ntile * kStripsPerTile;
-    const int rows = a->B * a->R;
-    // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
-    P.split = (static_cast<long long>(rows) * P.ntile >= 4096) ? 1 : 0;
     P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sr = a->d_stride_r;
-    P.maskbits = ctx->d_mask; P.tau = a->temperature; P.u = a->uniforms;
+    P.maskbits = ctx->d_mask; P.lengths = nullptr; P.tau = a->temperature; P.u = a->uniforms;
     P.draft_ids = a->draft_ids; P.q_out = a->q_draft; P.status = a->draft_status;
     P.part = reinterpret_cast<DraftPart *>(a->workspace);
     P.cnt = ctx->d_counters + (TLI_MAX_B + 1);           // the sampling pass's tickets: zero between calls
-    const dim3 grid(static_cast<unsigned>(P.ntile), static_cast<unsigned>(rows));
+    return launch_row_sampler(P, a->dtype, reinterpret_cast<cudaStream_t>(cuda_stream));
+}
+
+namespace {
+struct SlemLayout { size_t part, sampled, flags, total; };
+SlemLayout slem_layout(int B, int M, int V_t, int dtype) {
+    SlemLayout L;
+    const size_t rows = static_cast<size_t>(B) * (M + 1);
+    const size_t nstrip = static_cast<size_t>(chunks_per_row(V_t, dtype, kVecPerTile)) * kStripsPerTile;
+    size_t off = 0;
+    L.part = off;    off = align_up(off + sizeof(DraftPart) * rows * nstrip, 256);
+    L.sampled = off; off = align_up(off + sizeof(int) * rows, 256);
+    L.flags = off;   off = align_up(off + sizeof(int) * rows, 256);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t tli_slem_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t M, int32_t dtype) {
+    if (!ctx || B < 1 || M < 0 || M > TLI_MAX_K || static_cast<long long>(B) * (M + 1) > TLI_MAX_B) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    return slem_layout(B, M, ctx->V_t, dtype).total;
+}
+
+int tli_slem_verify(tli_ctx *ctx, const tli_slem_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->M < 0) return TLI_ERR_ARG;
+    if (a->M > TLI_MAX_K || static_cast<long long>(a->B) * (a->M + 1) > TLI_MAX_B) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->target_logits || !a->temperature || !a->uniforms || !a->accepted || !a->next_token) return TLI_ERR_ARG;
+    if (a->M > 0 && !a->candidates) return TLI_ERR_ARG;
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(a->target_logits) % elt) return TLI_ERR_ARG;
+    if (a->t_stride_b < 0 || a->t_stride_k < 0) return TLI_ERR_ARG;
+    const SlemLayout L = slem_layout(a->B, a->M, ctx->V_t, a->dtype);
+    if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
+        return TLI_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(a->workspace);
+    int *sampled = a->sampled ? a->sampled : reinterpret_cast<int *>(ws + L.sampled);
+    int *flags = reinterpret_cast<int *>(ws + L.flags);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
-    if (a->dtype == TLI_F32) tli_draft_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(P);
-    else tli_draft_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(P);
-    cudaError_t e = cudaGetLastError();
-    if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_kernel");
-    if (P.split) {
-        cudaLaunchConfig_t cfg;
-        memset(&cfg, 0, sizeof cfg);
-        cudaLaunchAttribute attr[1];
-        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-        attr[0].val.programmaticStreamSerializationAllowed = 1;
-        cfg.gridDim = dim3(static_cast<unsigned>(rows)); cfg.blockDim = dim3(kThreads);
-        cfg.dynamicSmemBytes = 0; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
-        if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_F32>, P);
-        else e = cudaLaunchKernelEx(&cfg, tli_draft_select_kernel<TLI_BF16>, P);
-        if (e != cudaSuccess) return cuda_fail(e, "launch tli_draft_select_kernel");
-    }
+    DraftParams P;
+    P.B = a->B; P.R = a->M + 1; P.V_d = ctx->V_t;
+    P.zd = a->target_logits; P.d_sb = a->t_stride_b; P.d_sr = a->t_stride_k;
+    P.maskbits = nullptr; P.lengths = a->lengths; P.tau = a->temperature; P.u = a->uniforms;
+    P.draft_ids = sampled; P.q_out = nullptr; P.status = flags;
+    P.part = reinterpret_cast<DraftPart *>(ws + L.part);
+    P.cnt = ctx->d_counters + (TLI_MAX_B + 1);
+    const int rc = launch_row_sampler(P, a->dtype, stream);
+    if (rc != TLI_OK) return rc;
+    SlemParams Q;
+    Q.B = a->B; Q.M = a->M; Q.candidates = a->candidates; Q.lengths = a->lengths; Q.tau = a->temperature;
+    Q.sampled = sampled; Q.row_flags = flags;
+    Q.accepted = a->accepted; Q.next_token = a->next_token; Q.status = a->row_status;
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.gridDim = dim3(static_cast<unsigned>((a->B + 127) / 128)); cfg.blockDim = dim3(128);
+    cfg.dynamicSmemBytes = 0; cfg.stream = stream; cfg.attrs = attr; cfg.numAttrs = 1;
+    const cudaError_t e = cudaLaunchKernelEx(&cfg, tli_slem_match_kernel, Q);
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_slem_match_kernel");
     return TLI_OK;
 }
 

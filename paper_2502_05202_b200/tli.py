@@ -38,7 +38,7 @@ TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
 EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
-           "tli_draft_workspace_bytes", "tli_draft_sample",
+           "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -61,6 +61,18 @@ class tli_draft_args(ctypes.Structure):
         ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_r", ctypes.c_int64),
         ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
         ("draft_ids", ctypes.c_void_p), ("q_draft", ctypes.c_void_p), ("draft_status", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+    ]
+
+
+class tli_slem_args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("M", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("candidates", ctypes.c_void_p), ("lengths", ctypes.c_void_p),
+        ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("sampled", ctypes.c_void_p),
+        ("row_status", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
 
@@ -102,6 +114,10 @@ def load() -> ctypes.CDLL:
         lib.tli_draft_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_draft_sample.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_draft_args), ctypes.c_void_p]
         lib.tli_draft_sample.restype = ctypes.c_int
+        lib.tli_slem_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_slem_workspace_bytes.restype = ctypes.c_size_t
+        lib.tli_slem_verify.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_slem_args), ctypes.c_void_p]
+        lib.tli_slem_verify.restype = ctypes.c_int
         lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_fused.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
@@ -231,6 +247,43 @@ def tli_draft_sample(ctx: int, args: tli_draft_args, stream: Optional[int] = Non
         raise TLIError(rc, "tli_draft_sample")
 
 
+def tli_slem_workspace_bytes(ctx: int, B: int, M: int, dtype: int) -> int:
+    return int(load().tli_slem_workspace_bytes(ctx, B, M, dtype))
+
+
+def make_slem_args(target_logits: torch.Tensor, candidates: torch.Tensor, temperature: torch.Tensor,
+                   uniforms: torch.Tensor, accepted: torch.Tensor, next_token: torch.Tensor, workspace: torch.Tensor,
+                   lengths: Optional[torch.Tensor] = None, sampled: Optional[torch.Tensor] = None,
+                   row_status: Optional[torch.Tensor] = None) -> tli_slem_args:
+    """Fill a tli_slem_args from device tensors (no copies; the tensors must outlive the call)."""
+    B, M1, _ = target_logits.shape
+    M = M1 - 1
+    dt = _logit_dtype(target_logits)
+    if target_logits.stride(2) != 1:
+        raise ValueError("the vocabulary axis must be contiguous")
+    for name, t, dtype, shape in (("candidates", candidates, torch.int32, (B, M)),
+                                  ("temperature", temperature, torch.float32, (B,)),
+                                  ("uniforms", uniforms, torch.float32, (B, M + 1)),
+                                  ("accepted", accepted, torch.int32, (B,)),
+                                  ("next_token", next_token, torch.int32, (B,))):
+        if t.dtype != dtype or tuple(t.shape) != shape or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous %s tensor of shape %s" % (name, dtype, shape))
+    opt = lambda t: None if t is None else t.data_ptr()
+    return tli_slem_args(B, M, dt, target_logits.data_ptr(), target_logits.stride(0), target_logits.stride(1),
+                         candidates.data_ptr(), opt(lengths), temperature.data_ptr(), uniforms.data_ptr(),
+                         accepted.data_ptr(), next_token.data_ptr(), opt(sampled), opt(row_status),
+                         workspace.data_ptr(), workspace.numel() * workspace.element_size())
+
+
+def tli_slem_verify(ctx: int, args: tli_slem_args, stream: Optional[int] = None) -> None:
+    """tli_slem_verify() on ``stream`` (a cudaStream_t as int; default: torch's current stream)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_slem_verify(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_slem_verify")
+
+
 def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
     """tli_verify_profile(): blocks; returns ms of (statistics kernel, decision kernel, sampling kernel)."""
     if stream is None:
@@ -305,6 +358,25 @@ class Verifier:
         args = make_draft_args(drafter_logits, temperature, uniforms, out["draft_ids"], self._ws,
                                out["q_draft"], out["draft_status"])
         tli_draft_sample(self.ctx, args)
+        return out
+
+    def slem(self, target_logits, candidates, temperature, uniforms, lengths=None) -> Dict[str, torch.Tensor]:
+        """Exact-match verification of re-tokenised drafts ``candidates`` [B,M] against tokens sampled
+        from ``target_logits`` [B,M+1,V_t]; returns device tensors."""
+        B, M1, _ = target_logits.shape
+        dev = self.device
+        out = {"accepted": torch.empty(B, dtype=torch.int32, device=dev),
+               "next_token": torch.empty(B, dtype=torch.int32, device=dev),
+               "sampled": torch.empty(B, M1, dtype=torch.int32, device=dev),
+               "row_status": torch.empty(B, dtype=torch.int32, device=dev)}
+        need = tli_slem_workspace_bytes(self.ctx, B, M1 - 1, _logit_dtype(target_logits))
+        if need == 0:
+            raise TLIError(TLI_ERR_UNSUPPORTED, "tli_slem_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        args = make_slem_args(target_logits, candidates, temperature, uniforms, out["accepted"], out["next_token"],
+                              self._ws, lengths, out["sampled"], out["row_status"])
+        tli_slem_verify(self.ctx, args)
         return out
 
     def verify(self, target_logits, drafter_logits, draft_ids, temperature, uniforms,
