@@ -309,6 +309,32 @@ class GpuCase:
         return {"ms_per_call": ms, "rows_per_s": cfg.B * cfg.K / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
                 "rows_per_call": cfg.B * cfg.K, "bytes_per_call": nbytes, "greedy_sequences": greedy}
 
+    def slem_timing(self, steps):
+        """tli_slem_verify() on this workload's target logits (candidates: the drafts carried to target ids)."""
+        import numpy as np
+        torch, tli, cfg = self.torch, self.tli, self.cfg
+        dev = self.zt[0].device
+        cand = torch.from_numpy(self.batch["id_map"][self.batch["draft_ids"]].astype(np.int32)).to(dev)
+        acc = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+        nxt = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+        st = torch.empty(cfg.B, dtype=torch.int32, device=dev)
+        need = tli.tli_slem_workspace_bytes(self.ver.ctx, cfg.B, cfg.K, tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16)
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        args = [tli.make_slem_args(z, cand, self.tau, self.u, acc, nxt, ws, row_status=st) for z in self.zt]
+        n = [0]
+
+        def step():
+            tli.tli_slem_verify(self.ver.ctx, args[n[0] % len(args)], self.stream)
+            n[0] += 1
+        for _ in range(3 + len(args)):
+            step()
+        ms = timed(torch, None, steps, step, 1) / steps
+        assert int(st.abs().sum()) == 0, "row_status not clean on benchmark inputs"
+        nbytes = cfg.elt * cfg.B * (cfg.K + 1) * cfg.V_t
+        return {"ms_per_call": ms, "positions_per_s": cfg.B * cfg.K / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
+                "rows_per_call": cfg.B * (cfg.K + 1), "bytes_per_call": nbytes,
+                "mean_accepted": float(acc.float().mean().item())}
+
     def e2e_bytes(self):
         h = self.host
         h2d = sum(h[k].numel() * h[k].element_size() for k in ("zt", "zd", "draft", "tau", "u"))
@@ -403,6 +429,7 @@ def gpu_arm(args):
     ms_stats, ms_decide, ms_sample = case.profile(args.steps)
     calls = call_timings(case, torch, args.steps)
     draft = case.draft_timing(max(args.steps, 20)) if world == 1 else None
+    slem = case.slem_timing(max(args.steps, 20)) if world == 1 else None
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
@@ -430,6 +457,7 @@ def gpu_arm(args):
         "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
         "per_call": calls,
         "draft_sample": draft,
+        "slem_verify": slem,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
@@ -449,7 +477,7 @@ def gpu_arm(args):
                 per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
                             "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
                             "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls,
-                            "draft_sample": draft})
+                            "draft_sample": draft, "slem_verify": slem})
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
@@ -460,6 +488,7 @@ def gpu_arm(args):
             a, d, b = k.profile(min(steps, 50))
             kc = call_timings(k, torch, steps)
             kc["draft_sample"] = k.draft_timing(steps)
+            kc["slem_verify"] = k.slem_timing(steps)
             k.check()
             per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
                         "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
