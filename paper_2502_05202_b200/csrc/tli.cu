@@ -876,7 +876,10 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
 // Weights of the elements of vector v of the sampled target row:
 // p(t), or max(0, p(t) - q'(inv[t])) for the residual.  The same code feeds the
 // tile sums and every rescan, so the levels of the CDF walk agree bit for bit.
-template <int DT>
+// LEAN: the caller knows that the vector lies wholly inside the row and that its first id is a
+// multiple of four (true for every vector of a tile that is not at an end of an aligned row), which
+// takes the checks and the element-wise loads out of the code.
+template <int DT, bool LEAN = false>
 __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
                                                     const void *zd_row, float (&w)[Elt<DT>::kPerVec]) {
     constexpr int EPV = Elt<DT>::kPerVec;
@@ -886,7 +889,7 @@ __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSe
 #pragma unroll
     for (int i = 0; i < EPV; ++i) x[i] = -1;
     if (sel.mode == MODE_RESIDUAL) {
-        if (e0 >= 0 && e0 + EPV <= P.V_t && (e0 & 3) == 0) {
+        if (LEAN || (e0 >= 0 && e0 + EPV <= P.V_t && (e0 & 3) == 0)) {
 #pragma unroll
             for (int i = 0; i < EPV; i += 4) {
                 const int4 q = __ldg(reinterpret_cast<const int4 *>(P.inv + e0 + i));
@@ -914,11 +917,11 @@ __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSe
     }
 }
 
-template <int DT>
+template <int DT, bool LEAN = false>
 __device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
                                                const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
-    const uint4 raw = rt.load(v);
-    vector_weights_from<DT>(P, sel, raw, rt.first_elem(v), zd_row, w);
+    const uint4 raw = LEAN ? __ldg(rt.vec0 + v) : rt.load(v);
+    vector_weights_from<DT, LEAN>(P, sel, raw, rt.first_elem(v), zd_row, w);
 }
 
 template <int N> __device__ __forceinline__ float ordered_sum(const float (&w)[N]) {
@@ -936,13 +939,25 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int nvec = rt.nvec();
     double acc = 0.0;
+    const int v_first = tile * kVecPerTile;
+    const bool lean = (rt.head & 3) == 0 && rt.first_elem(v_first) >= 0 &&
+                      rt.first_elem(v_first + kVecPerTile - 1) + EPV <= rt.V;        // the same for the whole CTA
+    if (lean) {
 #pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = tile * kVecPerTile + k * kThreads + tid;
-        if (v < nvec) {
+        for (int k = 0; k < kVecPerThread; ++k) {
             float w[EPV];
-            vector_weights<DT>(P, sel, rt, zd_row, v, w);
+            vector_weights<DT, true>(P, sel, rt, zd_row, v_first + k * kThreads + tid, w);
             acc += static_cast<double>(ordered_sum(w));
+        }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const int v = v_first + k * kThreads + tid;
+            if (v < nvec) {
+                float w[EPV];
+                vector_weights<DT>(P, sel, rt, zd_row, v, w);
+                acc += static_cast<double>(ordered_sum(w));
+            }
         }
     }
     acc = warp_sum(acc);
@@ -1176,19 +1191,23 @@ struct DraftParams {
 };
 
 // Vector v of a drafter row with the ids outside the intersection (and outside the row) set to -inf.
-template <int DT>
+// INTERIOR: the caller knows that the vector lies wholly inside the row (a whole strip does, for all
+// but the two ends of a row), which takes the checks and the element-wise loads out of the code.
+template <int DT, bool INTERIOR>
 __device__ __forceinline__ uint4 draft_masked_vector(const DraftParams &P, const RowView<DT> &rv, int v, int nvec,
                                                      uint32_t &bits) {
     constexpr uint32_t NI = Elt<DT>::kNegInfWord;
+    constexpr int EPV = Elt<DT>::kPerVec;
     bits = 0u;
-    if (v >= nvec) return make_uint4(NI, NI, NI, NI);
-    uint4 raw = rv.load(v);
+    if (!INTERIOR && v >= nvec) return make_uint4(NI, NI, NI, NI);
+    uint4 raw = INTERIOR ? __ldg(rv.vec0 + v) : rv.load(v);
     const int e0 = rv.first_elem(v);
     if (P.maskbits == nullptr) {                           // no mask: the elements inside the row (load() gave -inf elsewhere)
-        constexpr int EPV = Elt<DT>::kPerVec;
         bits = (1u << EPV) - 1u;
-        if (e0 < 0) bits &= ~((1u << (-e0)) - 1u);
-        if (e0 + EPV > rv.V) bits &= (1u << (rv.V - e0)) - 1u;
+        if (!INTERIOR) {
+            if (e0 < 0) bits &= ~((1u << (-e0)) - 1u);
+            if (e0 + EPV > rv.V) bits &= (1u << (rv.V - e0)) - 1u;
+        }
         return raw;
     }
     bits = mask_bits(P.maskbits, e0);
@@ -1199,6 +1218,22 @@ __device__ __forceinline__ uint4 draft_masked_vector(const DraftParams &P, const
         raw.z = (bits & 4u) ? raw.z : NI; raw.w = (bits & 8u) ? raw.w : NI;
     }
     return raw;
+}
+
+// This lane's kVecPerThread vectors of strip `strip` (vector k*32 + lane of the strip's 128).
+template <int DT>
+__device__ __forceinline__ void draft_load_strip(const DraftParams &P, const RowView<DT> &rv, int strip, int nvec, int lane,
+                                                 uint4 (&m)[kVecPerThread], uint32_t (&bits)[kVecPerThread]) {
+    const int v0 = strip * (32 * kVecPerThread);
+    const bool interior = rv.first_elem(v0) >= 0 &&
+                          rv.first_elem(v0 + 32 * kVecPerThread - 1) + Elt<DT>::kPerVec <= rv.V;
+    if (interior) {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) m[k] = draft_masked_vector<DT, true>(P, rv, v0 + k * 32 + lane, nvec, bits[k]);
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) m[k] = draft_masked_vector<DT, false>(P, rv, v0 + k * 32 + lane, nvec, bits[k]);
+    }
 }
 
 // fp32 sum, in element order, of the weights 2^(z*s + nc) of one masked vector; the weights in w[]
@@ -1340,11 +1375,13 @@ __device__ void draft_select(const DraftParams &P, int row, const RowView<DT> &r
     const int nvec = rv.nvec();
     uint4 m[kVecPerThread];
     float vs[kVecPerThread];
+    {
+        uint32_t bits[kVecPerThread];
+        draft_load_strip<DT>(P, rv, T, nvec, lane, m, bits);
+    }
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
-        uint32_t bits;
         float w[EPV];
-        m[k] = draft_masked_vector<DT>(P, rv, T * (32 * kVecPerThread) + k * 32 + lane, nvec, bits);
         vs[k] = draft_vector_sum<DT>(m[k], s, -cT, w);
     }
     // vector g = k*32 + lane in address order: mass before it, fp64
@@ -1431,9 +1468,7 @@ __global__ void __launch_bounds__(kThreads, 6) tli_draft_kernel(const DraftParam
 
     uint4 m[kVecPerThread];
     uint32_t bits[kVecPerThread];
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k)
-        m[k] = draft_masked_vector<DT>(P, rv, strip * (32 * kVecPerThread) + k * 32 + lane, nvec, bits[k]);
+    draft_load_strip<DT>(P, rv, strip, nvec, lane, m, bits);
     DraftPart pt;
     if (tau == 0.f) {
         // largest logit inside the intersection, lowest id; an id inside it counts even at -inf
