@@ -1454,7 +1454,7 @@ __global__ void __launch_bounds__(kThreads, 6) tli_draft_kernel(const DraftParam
         }
         return;
     }
-    if (P.lengths && r > __ldg(P.lengths + b)) {               // not a row of this sequence
+    if (P.lengths && r > max(__ldg(P.lengths + b), 0)) {        // not a row of this sequence
         if (tile == 0 && tid == 0) {
             P.draft_ids[row] = -1;
             if (P.q_out) P.q_out[row] = 0.f;
@@ -1544,7 +1544,7 @@ __global__ void __launch_bounds__(kThreads) tli_draft_select_kernel(const DraftP
     const int b = row / P.R, r = row - b * P.R;
     const float tau = __ldg(P.tau + b);
     if (!(tau >= 0.f) || isinf(tau)) return;                 // the tile kernel has written this row
-    if (P.lengths && r > __ldg(P.lengths + b)) return;       // this one too
+    if (P.lengths && r > max(__ldg(P.lengths + b), 0)) return;   // this one too
     const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(r) * P.d_sr, P.V_d);
     draft_select<DT>(P, row, rv, tau);
 }
