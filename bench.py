@@ -175,7 +175,7 @@ def reference_arm(args):
 
 def stats_kernel_traffic(cfg):
     """DRAM bytes (read + write) of one tli_stats_kernel launch from the committed ncu capture
-    (profiles/stats_kernel_cfg3_b64_cfg2.md): cfg3 with B=64 moved 459 066 112 + 4 182 016 bytes;
+    (kept as a summary beside the other profiles): cfg3 with B=64 moved 459 066 112 + 4 182 016 bytes;
     traffic is proportional to B, so the full batch is 4 x that.  None for the other workloads and
     to be set back to None whenever the kernel changes."""
     if cfg.name == "cfg3" and cfg.B % 64 == 0:
