@@ -44,6 +44,7 @@ class _Args(ctypes.Structure):
         ("thr", ctypes.c_void_p), ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
         ("cdf_lo", ctypes.c_void_p), ("cdf_hi", ctypes.c_void_p), ("total", ctypes.c_void_p),
         ("probe_lo", ctypes.c_void_p), ("probe_hi", ctypes.c_void_p), ("probe_w", ctypes.c_void_p),
+        ("draft_lengths", ctypes.c_void_p),
     ]
 
 
@@ -108,7 +109,7 @@ class _Call:
     """Keeps the numpy arrays of one call alive next to the C struct."""
 
     def __init__(self, target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
-                 force_accept=None, probe_token=None):
+                 force_accept=None, probe_token=None, draft_lengths=None):
         zt = np.asarray(target_logits)
         zd = np.asarray(drafter_logits)
         if zt.dtype == np.float32 and zd.dtype == np.float32:
@@ -135,6 +136,7 @@ class _Call:
             raise ValueError("id_map must be [V_d]")
         self.force = None if force_accept is None else np.ascontiguousarray(force_accept, dtype=np.int8).reshape(B, K)
         self.probe = None if probe_token is None else np.ascontiguousarray(probe_token, dtype=np.int32).reshape(B)
+        self.lengths = None if draft_lengths is None else np.ascontiguousarray(draft_lengths, dtype=np.int32).reshape(B)
         self.out: Dict[str, np.ndarray] = {
             "accepted": np.zeros(B, np.int32), "next_token": np.zeros(B, np.int32),
             "flags": np.zeros(B, np.int32),
@@ -158,11 +160,12 @@ class _Call:
             _ptr(o["thr"]), _ptr(o["p_draft"]), _ptr(o["q_draft"]),
             _ptr(o["cdf_lo"]), _ptr(o["cdf_hi"]), _ptr(o["total"]),
             _ptr(o.get("probe_lo")), _ptr(o.get("probe_hi")), _ptr(o.get("probe_w")),
+            _ptr(self.lengths),
         )
 
 
 def verify(target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
-           force_accept=None, probe_token=None, threads: int = 1) -> Dict[str, np.ndarray]:
+           force_accept=None, probe_token=None, threads: int = 1, draft_lengths=None) -> Dict[str, np.ndarray]:
     """Run the oracle on a whole batch.
 
     Logits are float32 arrays or uint16 arrays holding bfloat16 bit patterns;
@@ -171,11 +174,14 @@ def verify(target_logits, drafter_logits, id_map, draft_ids, temperature, unifor
     threads; the arithmetic per row is unchanged.  Returns a dict with
     ``accepted``, ``next_token``, ``flags`` (int32 [B]), ``thr``, ``p_draft``,
     ``q_draft`` (float64 [B,K]), ``cdf_lo``, ``cdf_hi``, ``total`` (float64
-    [B]) and, when ``probe_token`` is given, ``probe_lo/hi/w``.
+    [B]) and, when ``probe_token`` is given, ``probe_lo/hi/w``.  With
+    ``draft_lengths`` (int32 [B], 0..K) only that many drafts of a sequence
+    count and its extra token comes from target row ``draft_lengths[b]`` when
+    all of them are accepted.
     """
     lib = _load()
     call = _Call(target_logits, drafter_logits, id_map, draft_ids, temperature, uniforms,
-                 force_accept, probe_token)
+                 force_accept, probe_token, draft_lengths)
     B = call.B
     threads = max(1, min(int(threads), B))
 

@@ -93,6 +93,9 @@ typedef struct {
     double *probe_lo;           /* [B] (only if probe_token) */
     double *probe_hi;           /* [B] */
     double *probe_w;            /* [B] normalised weight of the probed token */
+    /* optional input, last so that older callers' layouts stay valid */
+    const int32_t *draft_lengths; /* [B] or NULL: drafts of sequence b that count, 0..K; the extra token
+                                   * then comes from target row draft_lengths[b] when all of them are accepted */
 } oracle_args;
 
 static double load_logit(const void *base, int dtype, int64_t idx)
@@ -216,7 +219,10 @@ int oracle_tli_verify(const oracle_args *a, int32_t row_begin, int32_t row_end)
         const int64_t t_off = (int64_t)b * a->t_stride_b;
         const int64_t d_off = (int64_t)b * a->d_stride_b;
         int flags = 0;
-        int n = K;
+        int Kb = a->draft_lengths ? a->draft_lengths[b] : K;   /* drafts of this sequence */
+        if (Kb < 0) Kb = 0;
+        if (Kb > K) Kb = K;
+        int n = Kb;
         int next = 0;
         double lo = 0.0, hi = 0.0, R = 0.0;
         for (int j = 0; j < K; ++j) {
@@ -233,7 +239,7 @@ int oracle_tli_verify(const oracle_args *a, int32_t row_begin, int32_t row_end)
 
         if (tau == 0.0) {
             /* arg-max limit: exact match of map[d_j] with the row's arg-max */
-            for (int j = 0; j < K; ++j) {
+            for (int j = 0; j < Kb; ++j) {
                 int aj = argmax_row(a->target_logits, a->dtype, t_off + (int64_t)j * a->t_stride_k, V_t);
                 int32_t x = a->draft_ids[(int64_t)b * K + j];
                 int ok;
@@ -245,15 +251,15 @@ int oracle_tli_verify(const oracle_args *a, int32_t row_begin, int32_t row_end)
                 acc[j] = ok;
                 if (a->thr) a->thr[(int64_t)b * K + j] = ok ? 1.0 : 0.0;
             }
-            n = K;
-            for (int j = 0; j < K; ++j) if (!acc[j]) { n = j; break; }
+            n = Kb;
+            for (int j = 0; j < Kb; ++j) if (!acc[j]) { n = j; break; }
             next = argmax_row(a->target_logits, a->dtype, t_off + (int64_t)n * a->t_stride_k, V_t);
             lo = 0.0; hi = 1.0; R = 1.0;
             goto row_done;
         }
 
         /* acceptance tests, Algorithm 5 with (p, q') */
-        for (int j = 0; j < K; ++j) {
+        for (int j = 0; j < Kb; ++j) {
             int ok_sc, empty;
             if (!softmax_row(a->target_logits, a->dtype, t_off + (int64_t)j * a->t_stride_k, V_t, tau, p) ||
                 !qprime_row(a, d_off + (int64_t)j * a->d_stride_k, tau, q, qp, &ok_sc, &empty)) {
@@ -283,14 +289,14 @@ int oracle_tli_verify(const oracle_args *a, int32_t row_begin, int32_t row_end)
         if (flags & FLAG_NONFINITE) { n = 0; next = 0; goto row_done; }
 
         /* number of accepted drafts */
-        n = K;
-        for (int j = 0; j < K; ++j) if (!acc[j]) { n = j; break; }
+        n = Kb;
+        for (int j = 0; j < Kb; ++j) if (!acc[j]) { n = j; break; }
 
         /* distribution of the extra token */
         if (!softmax_row(a->target_logits, a->dtype, t_off + (int64_t)n * a->t_stride_k, V_t, tau, p)) {
             flags |= FLAG_NONFINITE; n = 0; next = 0; goto row_done;
         }
-        if (n < K) {
+        if (n < Kb) {
             int ok_sc, empty;
             if (!qprime_row(a, d_off + (int64_t)n * a->d_stride_k, tau, q, qp, &ok_sc, &empty)) {
                 flags |= FLAG_NONFINITE; n = 0; next = 0; goto row_done;

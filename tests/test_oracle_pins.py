@@ -10,6 +10,7 @@ import scipy.special
 import scipy.stats
 
 import oracle
+from paper_2502_05202_b200 import workload as wl
 
 GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
 ONE_M = np.float32(1.0 - 2.0 ** -24)   # the largest uniform the ABI allows
@@ -474,3 +475,30 @@ def test_oracle_catches_a_planted_wrong_denominator():
     np.add.at(dist, id_map[inside], qp[inside] * a_wrong)
     dist += (qp[inside] * (1 - a_wrong)).sum() * r_wrong
     assert np.abs(dist - p).max() > 1e-3
+
+
+def test_ragged_draft_counts_equal_truncated_batches():
+    """draft_lengths[b] = m: the result is that of the same sequence given with K = m drafts (rows and
+    uniforms beyond m dropped, the last uniform kept); m = 0 is one draw from target row 0."""
+    cfg = wl.tiny_config(B=12, K=5, V_t=60, V_d=50, dtype=wl.F32, f_mapped=0.7, sigma_d=0.3,
+                         temperatures=(0.0, 0.8, 1.0), seed=77)
+    b = wl.make_batch(cfg)
+    lengths = np.array([0, 1, 2, 3, 4, 5, 5, 3, 0, 2, 1, 4], np.int32)
+    rag = oracle.verify(b["target_logits"], b["drafter_logits"], b["id_map"], b["draft_ids"], b["temperature"],
+                        b["uniforms"], draft_lengths=lengths)
+    full = oracle.verify(b["target_logits"], b["drafter_logits"], b["id_map"], b["draft_ids"], b["temperature"],
+                         b["uniforms"])
+    assert (rag["accepted"] <= lengths).all() and rag["accepted"].max() >= 2
+    for i, m in enumerate(lengths):
+        u = np.concatenate([b["uniforms"][i:i + 1, :m], b["uniforms"][i:i + 1, -1:]], axis=1)
+        if m == 0:
+            one = oracle.slem(b["target_logits"][i:i + 1, :1], np.zeros((1, 0), np.int32), b["temperature"][i:i + 1], u)
+            assert rag["accepted"][i] == 0 and rag["next_token"][i] == one["next_token"][0]
+            continue
+        sub = oracle.verify(b["target_logits"][i:i + 1, :m + 1], b["drafter_logits"][i:i + 1, :m], b["id_map"],
+                            b["draft_ids"][i:i + 1, :m], b["temperature"][i:i + 1], u)
+        assert sub["accepted"][0] == rag["accepted"][i] and sub["next_token"][0] == rag["next_token"][i]
+        np.testing.assert_array_equal(sub["thr"][0], rag["thr"][i, :m])
+        assert (rag["thr"][i, m:] == 0).all() and (rag["q_draft"][i, m:] == 0).all()
+        if m == cfg.K:
+            assert rag["accepted"][i] == full["accepted"][i] and rag["next_token"][i] == full["next_token"][i]
