@@ -124,6 +124,14 @@ typedef struct {
     void *workspace;            /* [device] scratch, 256-byte aligned, >= tli_workspace_bytes();
                                  * contents need no initialisation and are garbage afterwards */
     size_t workspace_bytes;
+
+    const int32_t *draft_lengths; /* [device] int32[B] or NULL.  Algorithm 5's lookahead given per
+                                 * sequence: only the first draft_lengths[b] (0 .. K) drafts of
+                                 * sequence b count; its later drafter rows and its target rows beyond
+                                 * row draft_lengths[b] are not read, and when all counted drafts are
+                                 * accepted the extra token is drawn from target row draft_lengths[b].
+                                 * The extra token still uses uniforms[b, K].  NULL = K for all.
+                                 * Not available in the fused form (TLI_ERR_UNSUPPORTED) */
 } tli_verify_args;
 
 /*

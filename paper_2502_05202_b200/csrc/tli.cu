@@ -71,6 +71,7 @@ struct Params {
     const void *zd; long long d_sb, d_sk;
     const int *map; const int *inv; const uint32_t *maskbits; int n_mapped;
     const int *draft; const float *tau; const float *u;
+    const int *draft_len;    // NULL, or per sequence how many of its K drafts count (three-kernel form only)
     int *accepted; int *next_token; int *status; float *p_out; float *q_out;
     float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
     unsigned *cnt_stats; unsigned *cnt_sample;
@@ -288,15 +289,16 @@ __device__ __forceinline__ Segment decode_segment(const Params &P, long long id)
     int item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
     g.tau = __ldg(P.tau + g.b);
     const bool bad = !(g.tau >= 0.f) || isinf(g.tau);
+    const int m = P.draft_len ? min(max(__ldg(P.draft_len + g.b), 0), P.K) : P.K;    // drafts of this sequence
     int nchunk;
     if (item < (P.K + 1) * P.nst) {
         g.row = item / P.nst; g.seg = item - g.row * P.nst; nchunk = P.nct;
-        g.skip = bad;
+        g.skip = bad || g.row > m;               // target rows 0..m: m drafts and the bonus position
     } else {
         item -= (P.K + 1) * P.nst;
         const int j = item / P.nsd;
         g.row = P.K + 1 + j; g.seg = item - j * P.nsd; nchunk = P.ncd;
-        g.skip = bad || g.tau == 0.f;
+        g.skip = bad || g.tau == 0.f || j >= m;
     }
     g.chunk0 = g.seg * P.cps;
     g.chunk1 = min(g.chunk0 + P.cps, nchunk);
@@ -721,6 +723,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
     __shared__ int sm_accept[TLI_MAX_K];
     __shared__ int sm_flags;
     const int K = P.K;
+    const int Kb = P.draft_len ? min(max(__ldg(P.draft_len + b), 0), K) : K;     // drafts of this sequence that count
     if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
         if (tid == 0) {
             P.accepted[b] = 0; P.next_token[b] = 0;
@@ -738,7 +741,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
     // the drafted token's two logits and its target id: loads in flight while the rows are combined
     int g_x = -1, g_t = -1, g_fl = 0;
     float g_zt = 0.f, g_zd = 0.f;
-    if (tid < K) {
+    if (tid < Kb) {
         g_x = P.draft[static_cast<size_t>(b) * K + tid];
         if (g_x < 0 || g_x >= P.V_d) g_fl |= TLI_ROW_DRAFT_RANGE;
         else { g_t = __ldg(P.map + g_x); if (g_t < 0) g_fl |= TLI_ROW_DRAFT_UNMAPPED; }
@@ -747,7 +750,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
             g_zd = load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(tid) * P.d_sk + g_x);
         }
     }
-    const int nrows = greedy ? (K + 1) : (2 * K + 1);
+    const int nrows = greedy ? (K + 1) : (2 * K + 1);      // rows beyond the sequence's own drafts have no partials
     if (tid == K) sm_u_last = u_mine;
     if (tid == 0) {
         int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
@@ -764,7 +767,8 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         const int r = r0 + (tid >> 3);
         const int sub = tid & 7;
         const bool is_t = r <= K;
-        const int nseg = (r >= nrows) ? 0 : (is_t ? P.nst : P.nsd);
+        const bool mine = r < nrows && (is_t ? r <= Kb : r - K - 1 < Kb);
+        const int nseg = !mine ? 0 : (is_t ? P.nst : P.nsd);
         const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
                                   : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
         if (greedy) {
@@ -804,7 +808,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
     __syncthreads();
 
     const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
-    if (tid < K) {
+    if (tid < Kb) {
         const int j = tid;
         int ok = 0, fl = g_fl;
         float pv = 0.f, qv = 0.f;
@@ -831,16 +835,19 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         if (fl) atomicOr(&sm_flags, fl);
         if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
         if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+    } else if (tid < K) {
+        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
+        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
     }
     // the bonus row's sum must be usable too
-    if (tid == K && !greedy) {
-        const double S_t = sm_s[K];
+    if (tid == Kb && !greedy) {
+        const double S_t = sm_s[Kb];
         if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
     }
     __syncthreads();
     if (tid == 0) {
-        int n = K;
-        for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
+        int n = Kb;
+        for (int j = 0; j < Kb; ++j) if (!sm_accept[j]) { n = j; break; }
         int fl = sm_flags;
         RowSel sel;
         sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
@@ -853,7 +860,7 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         } else {
             sel.c_t = sm_c[n];
             sel.rs_t = static_cast<float>(1.0 / sm_s[n]);
-            if (n < K) {
+            if (n < Kb) {
                 const double S_d = sm_s[K + 1 + n];
                 sel.mode = MODE_RESIDUAL;
                 sel.c_d = sm_c[K + 1 + n];
@@ -2439,6 +2446,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
         return TLI_ERR_ARG;
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
+    if (a->draft_lengths && ctx->fused) return TLI_ERR_UNSUPPORTED;     // the fused form takes whole batches only
     const Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
         return TLI_ERR_WORKSPACE;
@@ -2449,6 +2457,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sk = a->d_stride_k;
     P.map = ctx->d_map; P.inv = ctx->d_inv; P.maskbits = ctx->d_mask; P.n_mapped = ctx->n_mapped;
     P.draft = a->draft_ids; P.tau = a->temperature; P.u = a->uniforms;
+    P.draft_len = a->draft_lengths;
     P.accepted = a->accepted; P.next_token = a->next_token; P.status = a->row_status;
     P.p_out = a->p_draft; P.q_out = a->q_draft;
     char *ws = reinterpret_cast<char *>(a->workspace);

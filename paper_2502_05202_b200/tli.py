@@ -52,6 +52,7 @@ class tli_verify_args(ctypes.Structure):
         ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
         ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+        ("draft_lengths", ctypes.c_void_p),
     ]
 
 
@@ -165,7 +166,8 @@ def _logit_dtype(t: torch.Tensor) -> int:
 def make_args(target_logits: torch.Tensor, drafter_logits: torch.Tensor, draft_ids: torch.Tensor,
               temperature: torch.Tensor, uniforms: torch.Tensor, accepted: torch.Tensor,
               next_token: torch.Tensor, workspace: torch.Tensor, row_status: Optional[torch.Tensor] = None,
-              p_draft: Optional[torch.Tensor] = None, q_draft: Optional[torch.Tensor] = None) -> tli_verify_args:
+              p_draft: Optional[torch.Tensor] = None, q_draft: Optional[torch.Tensor] = None,
+              draft_lengths: Optional[torch.Tensor] = None) -> tli_verify_args:
     """Fill a tli_verify_args from device tensors (no copies; the tensors must outlive the call)."""
     B, K1, _ = target_logits.shape
     K = K1 - 1
@@ -190,7 +192,7 @@ def make_args(target_logits: torch.Tensor, drafter_logits: torch.Tensor, draft_i
         drafter_logits.data_ptr(), drafter_logits.stride(0), drafter_logits.stride(1),
         draft_ids.data_ptr(), temperature.data_ptr(), uniforms.data_ptr(),
         accepted.data_ptr(), next_token.data_ptr(), opt(row_status), opt(p_draft), opt(q_draft),
-        workspace.data_ptr(), workspace.numel() * workspace.element_size())
+        workspace.data_ptr(), workspace.numel() * workspace.element_size(), opt(draft_lengths))
 
 
 def tli_verify(ctx: int, args: tli_verify_args, stream: Optional[int] = None) -> None:
@@ -380,7 +382,7 @@ class Verifier:
         return out
 
     def verify(self, target_logits, drafter_logits, draft_ids, temperature, uniforms,
-               diagnostics: bool = True) -> Dict[str, torch.Tensor]:
+               diagnostics: bool = True, draft_lengths=None) -> Dict[str, torch.Tensor]:
         """One call on torch's current stream; returns device tensors (no synchronisation)."""
         B, K1, _ = target_logits.shape
         K = K1 - 1
@@ -394,6 +396,6 @@ class Verifier:
         ws = self.workspace(B, K, _logit_dtype(target_logits))
         args = make_args(target_logits, drafter_logits, draft_ids, temperature, uniforms,
                          out["accepted"], out["next_token"], ws, out["row_status"],
-                         out.get("p_draft"), out.get("q_draft"))
+                         out.get("p_draft"), out.get("q_draft"), draft_lengths)
         tli_verify(self.ctx, args)
         return out

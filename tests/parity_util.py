@@ -36,6 +36,8 @@ def to_device(batch: Dict[str, np.ndarray], device="cuda") -> Dict[str, torch.Te
             t = t.view(torch.bfloat16)
         out[k] = t.to(device)
     out["draft_ids"] = torch.from_numpy(batch["draft_ids"]).to(device)
+    out["draft_lengths"] = (torch.from_numpy(np.asarray(batch["draft_lengths"], np.int32)).to(device)
+                            if batch.get("draft_lengths") is not None else None)
     out["temperature"] = torch.from_numpy(batch["temperature"]).to(device)
     out["uniforms"] = torch.from_numpy(batch["uniforms"]).to(device)
     return out
@@ -50,7 +52,7 @@ def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = Non
 
     def once(v):
         out = v.verify(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"],
-                       dev["temperature"], dev["uniforms"])
+                       dev["temperature"], dev["uniforms"], draft_lengths=dev.get("draft_lengths"))
         torch.cuda.synchronize()
         return {k: x.cpu().numpy() for k, x in out.items()}
 
@@ -59,7 +61,8 @@ def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = Non
     V_t = batch["target_logits"].shape[2]
     V_d = batch["drafter_logits"].shape[2]
     res = None
-    for fused in (False, True):
+    forms = (False,) if batch.get("draft_lengths") is not None else (False, True)   # ragged counts: three kernels only
+    for fused in forms:
         v = tli.Verifier(V_t, V_d, batch["id_map"], fused=fused)
         r = once(v)
         r2 = once(v)                                  # a second call on the same context: counters came back to zero
@@ -75,7 +78,8 @@ def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = Non
 
 def run_oracle(batch: Dict[str, np.ndarray], threads: int = 8, **kw) -> Dict[str, np.ndarray]:
     return oracle.verify(batch["target_logits"], batch["drafter_logits"], batch["id_map"], batch["draft_ids"],
-                         batch["temperature"], batch["uniforms"], threads=threads, **kw)
+                         batch["temperature"], batch["uniforms"], threads=threads,
+                         draft_lengths=batch.get("draft_lengths"), **kw)
 
 
 @dataclass
@@ -101,7 +105,8 @@ def _sub(batch, rows):
     rows = np.asarray(rows)
     return {"target_logits": batch["target_logits"][rows], "drafter_logits": batch["drafter_logits"][rows],
             "id_map": batch["id_map"], "draft_ids": batch["draft_ids"][rows],
-            "temperature": batch["temperature"][rows], "uniforms": batch["uniforms"][rows]}
+            "temperature": batch["temperature"][rows], "uniforms": batch["uniforms"][rows],
+            "draft_lengths": None if batch.get("draft_lengths") is None else np.asarray(batch["draft_lengths"])[rows]}
 
 
 def compare(batch: Dict[str, np.ndarray], gpu: Dict[str, np.ndarray], orc: Optional[Dict[str, np.ndarray]] = None,

@@ -337,6 +337,35 @@ def test_calls_recorded_in_a_cuda_graph_replay_to_the_same_results():
     v.close()
 
 
+@pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
+def test_per_sequence_draft_counts(dtype):
+    """draft_lengths: only the first m_b drafts of a sequence count, the bonus position is row m_b, later
+    rows are never read (they hold NaN here), and the fused form refuses the argument."""
+    cfg = wl.tiny_config(B=14, K=6, V_t=40013, V_d=33001, dtype=dtype, f_mapped=0.6, sigma_d=0.4,
+                         temperatures=(0.0, 0.7, 1.0), seed=85)
+    batch = wl.make_batch(cfg)
+    lengths = np.array([0, 1, 2, 3, 4, 5, 6, 6, 3, 0, 2, 5, 1, 4], np.int32)
+    nan = np.float32(np.nan) if dtype == wl.F32 else np.uint16(0x7fc0)
+    for b, m in enumerate(lengths):
+        batch["target_logits"][b, m + 1:] = nan
+        batch["drafter_logits"][b, m:] = nan
+        batch["draft_ids"][b, m:] = -12345
+    batch["draft_lengths"] = lengths
+    rep = check(batch)
+    gpu = run_gpu(batch)
+    assert (gpu["accepted"] <= lengths).all() and (gpu["row_status"] == 0).all()
+    assert gpu["accepted"].max() >= 2 and ((gpu["accepted"] == lengths) & (lengths > 0)).sum() >= 2   # bonus rows below K were sampled
+    for b, m in enumerate(lengths):
+        assert (gpu["p_draft"][b, m:] == 0).all() and (gpu["q_draft"][b, m:] == 0).all()
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"], fused=True)
+    dev = to_device(batch)
+    with pytest.raises(tli.TLIError) as e:
+        v.verify(dev["target_logits"], dev["drafter_logits"], dev["draft_ids"], dev["temperature"], dev["uniforms"],
+                 draft_lengths=dev["draft_lengths"])
+    assert e.value.code == tli.TLI_ERR_UNSUPPORTED
+    v.close()
+
+
 def test_a_wait_that_nothing_completes_gives_up_and_leaves_the_context_usable():
     """The kernels' waits are bounded: run the same wait code on a barrier nobody will complete."""
     cfg = wl.tiny_config(B=3, K=2, V_t=9000, V_d=7000, dtype=wl.F32, f_mapped=0.5, seed=83)
