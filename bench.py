@@ -246,21 +246,23 @@ class GpuCase:
                                    self.ws, self.status) for i in range(self.copies)]
         self.stream = torch.cuda.current_stream().cuda_stream
         self.calls = 0
+        self.host_args = None
+        if want_host:
+            dt = tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16
+            self.host_buf = torch.empty(tli.tli_verify_host_buffer_bytes(self.ver.ctx, cfg.B, cfg.K, dt),
+                                        dtype=torch.uint8, device=device)
+            h = self.host
+            self.host_args = tli.make_host_args(h["zt"], h["zd"], h["draft"], h["tau"], h["u"],
+                                                h["out"][0], h["out"][1], self.host_buf)
 
     def step(self):
         self.tli.tli_verify(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
         self.calls += 1
 
     def step_e2e(self):
-        """Host buffers in, host results out: H2D of every input, the call, D2H of (accepted, next_token)."""
-        h = self.host
-        self.zt[0].copy_(h["zt"], non_blocking=True)
-        self.zd[0].copy_(h["zd"], non_blocking=True)
-        self.draft.copy_(h["draft"], non_blocking=True)
-        self.tau.copy_(h["tau"], non_blocking=True)
-        self.u.copy_(h["u"], non_blocking=True)
-        self.tli.tli_verify(self.ver.ctx, self.args[0], self.stream)
-        h["out"].copy_(self.out, non_blocking=True)
+        """tli_verify_host(): pinned host buffers in, host results out -- H2D of every input, the kernels,
+        D2H of (accepted, next_token), all inside the one C call."""
+        self.tli.tli_verify_host(self.ver.ctx, self.host_args, self.stream)
 
     def make_graph(self):
         """One CUDA graph holding a tli_verify() call on every input copy; returns (graph, calls in it)."""

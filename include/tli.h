@@ -192,6 +192,35 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 int tli_verify_static(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
 
 typedef struct {
+    int32_t B, K, dtype;            /* as in tli_verify_args */
+    const void *target_logits;      /* [host] [B, K+1, V_t], contiguous */
+    const void *drafter_logits;     /* [host] [B, K, V_d], contiguous */
+    const int32_t *draft_ids;       /* [host] int32[B, K] */
+    const float *temperature;       /* [host] float[B] */
+    const float *uniforms;          /* [host] float[B, K+1] */
+    int32_t *accepted;              /* [host] out int32[B] */
+    int32_t *next_token;            /* [host] out int32[B] */
+    int32_t *row_status;            /* [host] out int32[B]; may be NULL */
+    void *device_buffer;            /* [device] staging for the inputs, the outputs and the scratch of
+                                     * tli_verify(): 256-byte aligned, >= tli_verify_host_buffer_bytes() */
+    size_t device_buffer_bytes;
+} tli_verify_host_args;
+
+/* Bytes of device memory tli_verify_host() needs for (B, K, dtype); 0 on bad arguments. */
+size_t tli_verify_host_buffer_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype);
+
+/*
+ * tli_verify() for inputs and outputs in host memory: copies the five inputs
+ * to the caller's device buffer (cudaMemcpyAsync on the stream), runs the
+ * verification there and copies accepted / next_token / row_status back, all
+ * in stream order.  Allocates nothing and does not synchronise: the outputs
+ * are valid once the caller has synchronised the stream.  With pageable host
+ * memory the copies block the calling thread; pin the buffers to keep the call
+ * asynchronous.  What it computes, and its errors, are tli_verify()'s.
+ */
+int tli_verify_host(tli_ctx *ctx, const tli_verify_host_args *args, void *cuda_stream);
+
+typedef struct {
     int32_t B;      /* sequences, >= 1 */
     int32_t R;      /* rows of drafter logits per sequence, >= 1; B * R <= TLI_MAX_B */
     int32_t dtype;  /* TLI_F32 or TLI_BF16 */

@@ -2744,6 +2744,80 @@ int tli_verify_static(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream)
     return verify_impl(ctx, &b, cuda_stream, nullptr);
 }
 
+namespace {
+struct HostLayout { size_t zt, zd, draft, tau, u, out, status, ws, total; };
+HostLayout host_layout(const tli_ctx *ctx, int B, int K, int dtype) {
+    HostLayout L;
+    const size_t elt = dtype == TLI_F32 ? 4 : 2;
+    size_t off = 0;
+    L.zt = off;     off = align_up(off + elt * static_cast<size_t>(B) * (K + 1) * ctx->V_t, 256);
+    L.zd = off;     off = align_up(off + elt * static_cast<size_t>(B) * K * ctx->V_d, 256);
+    L.draft = off;  off = align_up(off + sizeof(int) * static_cast<size_t>(B) * K, 256);
+    L.tau = off;    off = align_up(off + sizeof(float) * static_cast<size_t>(B), 256);
+    L.u = off;      off = align_up(off + sizeof(float) * static_cast<size_t>(B) * (K + 1), 256);
+    L.out = off;    off = align_up(off + sizeof(int) * 2 * static_cast<size_t>(B), 256);     // accepted, next_token
+    L.status = off; off = align_up(off + sizeof(int) * static_cast<size_t>(B), 256);
+    L.ws = off;     off = align_up(off + make_layout(B, K, ctx->V_t, ctx->V_d, dtype, ctx->num_sms).total, 256);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t tli_verify_host_buffer_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype) {
+    if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    return host_layout(ctx, B, K, dtype).total;
+}
+
+int tli_verify_host(tli_ctx *ctx, const tli_verify_host_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
+    if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->target_logits || !a->drafter_logits || !a->draft_ids || !a->temperature || !a->uniforms ||
+        !a->accepted || !a->next_token)
+        return TLI_ERR_ARG;
+    const HostLayout L = host_layout(ctx, a->B, a->K, a->dtype);
+    if (!a->device_buffer || reinterpret_cast<uintptr_t>(a->device_buffer) % 256 || a->device_buffer_bytes < L.total)
+        return TLI_ERR_WORKSPACE;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    char *d = reinterpret_cast<char *>(a->device_buffer);
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    const size_t B = static_cast<size_t>(a->B), K = static_cast<size_t>(a->K);
+    struct { size_t off; const void *src; size_t bytes; } in[5] = {
+        {L.zt, a->target_logits, elt * B * (K + 1) * ctx->V_t},
+        {L.zd, a->drafter_logits, elt * B * K * ctx->V_d},
+        {L.draft, a->draft_ids, sizeof(int) * B * K},
+        {L.tau, a->temperature, sizeof(float) * B},
+        {L.u, a->uniforms, sizeof(float) * B * (K + 1)},
+    };
+    cudaError_t e;
+    for (int i = 0; i < 5; ++i)
+        if ((e = cudaMemcpyAsync(d + in[i].off, in[i].src, in[i].bytes, cudaMemcpyHostToDevice, stream)) != cudaSuccess)
+            return cuda_fail(e, "cudaMemcpyAsync to the device");
+    tli_verify_args v;
+    memset(&v, 0, sizeof v);
+    v.B = a->B; v.K = a->K; v.dtype = a->dtype;
+    v.target_logits = d + L.zt; v.t_stride_b = static_cast<int64_t>(K + 1) * ctx->V_t; v.t_stride_k = ctx->V_t;
+    v.drafter_logits = d + L.zd; v.d_stride_b = static_cast<int64_t>(K) * ctx->V_d; v.d_stride_k = ctx->V_d;
+    v.draft_ids = reinterpret_cast<const int32_t *>(d + L.draft);
+    v.temperature = reinterpret_cast<const float *>(d + L.tau);
+    v.uniforms = reinterpret_cast<const float *>(d + L.u);
+    v.accepted = reinterpret_cast<int32_t *>(d + L.out);
+    v.next_token = reinterpret_cast<int32_t *>(d + L.out) + B;
+    v.row_status = reinterpret_cast<int32_t *>(d + L.status);
+    v.workspace = d + L.ws; v.workspace_bytes = L.total - L.ws;
+    const int rc = verify_impl(ctx, &v, cuda_stream, nullptr);
+    if (rc != TLI_OK) return rc;
+    if ((e = cudaMemcpyAsync(a->accepted, v.accepted, sizeof(int) * B, cudaMemcpyDeviceToHost, stream)) != cudaSuccess ||
+        (e = cudaMemcpyAsync(a->next_token, v.next_token, sizeof(int) * B, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(e, "cudaMemcpyAsync to the host");
+    if (a->row_status &&
+        (e = cudaMemcpyAsync(a->row_status, v.row_status, sizeof(int) * B, cudaMemcpyDeviceToHost, stream)) != cudaSuccess)
+        return cuda_fail(e, "cudaMemcpyAsync to the host");
+    return TLI_OK;
+}
+
 const char *tli_status_string(int code) {
     switch (code) {
         case TLI_OK: return "ok";

@@ -39,6 +39,7 @@ TLI_STATIC_SCRATCH_BYTES = 4194304
 
 EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
+           "tli_verify_host_buffer_bytes", "tli_verify_host",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -53,6 +54,16 @@ class tli_verify_args(ctypes.Structure):
         ("p_draft", ctypes.c_void_p), ("q_draft", ctypes.c_void_p),
         ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
         ("draft_lengths", ctypes.c_void_p),
+    ]
+
+
+class tli_verify_host_args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("drafter_logits", ctypes.c_void_p), ("draft_ids", ctypes.c_void_p),
+        ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
+        ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
+        ("device_buffer", ctypes.c_void_p), ("device_buffer_bytes", ctypes.c_size_t),
     ]
 
 
@@ -119,6 +130,10 @@ def load() -> ctypes.CDLL:
         lib.tli_slem_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_slem_verify.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_slem_args), ctypes.c_void_p]
         lib.tli_slem_verify.restype = ctypes.c_int
+        lib.tli_verify_host_buffer_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_verify_host_buffer_bytes.restype = ctypes.c_size_t
+        lib.tli_verify_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_host_args), ctypes.c_void_p]
+        lib.tli_verify_host.restype = ctypes.c_int
         lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_fused.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
@@ -215,6 +230,34 @@ def tli_verify_static(ctx: int, args: tli_verify_args, stream: Optional[int] = N
     rc = load().tli_verify_static(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify_static")
+
+
+def tli_verify_host_buffer_bytes(ctx: int, B: int, K: int, dtype: int) -> int:
+    return int(load().tli_verify_host_buffer_bytes(ctx, B, K, dtype))
+
+
+def make_host_args(target_logits: torch.Tensor, drafter_logits: torch.Tensor, draft_ids: torch.Tensor,
+                   temperature: torch.Tensor, uniforms: torch.Tensor, accepted: torch.Tensor, next_token: torch.Tensor,
+                   device_buffer: torch.Tensor, row_status: Optional[torch.Tensor] = None) -> tli_verify_host_args:
+    """Fill a tli_verify_host_args: contiguous CPU tensors (pinned for an asynchronous call) and a device buffer."""
+    B, K1, _ = target_logits.shape
+    for t in (target_logits, drafter_logits, draft_ids, temperature, uniforms, accepted, next_token):
+        if t.is_cuda or not t.is_contiguous():
+            raise ValueError("host tensors must be contiguous CPU tensors")
+    return tli_verify_host_args(B, K1 - 1, _logit_dtype(target_logits), target_logits.data_ptr(), drafter_logits.data_ptr(),
+                                draft_ids.data_ptr(), temperature.data_ptr(), uniforms.data_ptr(),
+                                accepted.data_ptr(), next_token.data_ptr(),
+                                None if row_status is None else row_status.data_ptr(),
+                                device_buffer.data_ptr(), device_buffer.numel() * device_buffer.element_size())
+
+
+def tli_verify_host(ctx: int, args: tli_verify_host_args, stream: Optional[int] = None) -> None:
+    """tli_verify_host() on ``stream``; the outputs are valid after the stream has been synchronised."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_verify_host(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_verify_host")
 
 
 def tli_draft_workspace_bytes(ctx: int, B: int, R: int, dtype: int) -> int:

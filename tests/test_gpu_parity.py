@@ -337,6 +337,33 @@ def test_calls_recorded_in_a_cuda_graph_replay_to_the_same_results():
     v.close()
 
 
+def test_host_buffer_entry_point_gives_the_same_results():
+    """tli_verify_host(): pinned host tensors in and out through a caller's device buffer."""
+    cfg = wl.tiny_config(B=7, K=3, V_t=30011, V_d=20011, dtype=wl.BF16, f_mapped=0.5, temperatures=(0.0, 0.9), seed=86)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    ref = run_gpu(batch, v)
+    pin = lambda a: torch.from_numpy(np.ascontiguousarray(a)).pin_memory()
+    zt, zd = pin(batch["target_logits"]).view(torch.bfloat16), pin(batch["drafter_logits"]).view(torch.bfloat16)
+    acc, nxt, st = (torch.full((7,), -5, dtype=torch.int32).pin_memory() for _ in range(3))
+    need = tli.tli_verify_host_buffer_bytes(v.ctx, 7, 3, tli.TLI_BF16)
+    assert need > zt.numel() * 2 + zd.numel() * 2
+    buf = torch.empty(need, dtype=torch.uint8, device="cuda")
+    args = tli.make_host_args(zt, zd, pin(batch["draft_ids"]), pin(batch["temperature"]), pin(batch["uniforms"]),
+                              acc, nxt, buf, st)
+    tli.tli_verify_host(v.ctx, args)
+    torch.cuda.synchronize()
+    np.testing.assert_array_equal(acc.numpy(), ref["accepted"])
+    np.testing.assert_array_equal(nxt.numpy(), ref["next_token"])
+    np.testing.assert_array_equal(st.numpy(), ref["row_status"])
+    args.device_buffer_bytes = need - 1
+    with pytest.raises(tli.TLIError) as e:
+        tli.tli_verify_host(v.ctx, args)
+    assert e.value.code == tli.TLI_ERR_WORKSPACE
+    assert tli.tli_verify_host_buffer_bytes(v.ctx, 0, 3, tli.TLI_BF16) == 0
+    v.close()
+
+
 @pytest.mark.parametrize("dtype", [wl.F32, wl.BF16])
 def test_per_sequence_draft_counts(dtype):
     """draft_lengths: only the first m_b drafts of a sequence count, the bonus position is row m_b, later
