@@ -2,7 +2,8 @@
 
 ctypes front end of the fp64 CPU oracle in ``tli_oracle.c`` (Algorithms 4 and 5
 of the paper: ``verify`` for the verification half, ``draft`` for drawing the
-draft ids from q') and of Algorithm 2's exact-match verification (``slem``).  Only tests, the smoke check and the benchmark's CPU-baseline
+draft ids from q'), of Algorithm 2's exact-match verification (``slem``) and of
+the paper's expected acceptance rates (``rates``).  Only tests, the smoke check and the benchmark's CPU-baseline
 legs may import this package; the CUDA library never does, and this package
 imports nothing from it.
 """
@@ -72,6 +73,18 @@ class _SlemArgs(ctypes.Structure):
     ]
 
 
+class _RatesArgs(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("V_t", ctypes.c_int32), ("V_d", ctypes.c_int32),
+        ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_k", ctypes.c_int64),
+        ("id_map", ctypes.c_void_p), ("temperature", ctypes.c_void_p),
+        ("mass", ctypes.c_void_p), ("alpha_union", ctypes.c_void_p), ("alpha_tli", ctypes.c_void_p),
+        ("flags", ctypes.c_void_p),
+    ]
+
+
 def build(force: bool = False) -> str:
     """Compile ``tli_oracle.c`` with gcc -O2 into ``liboracle.so`` beside it."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
@@ -97,6 +110,8 @@ def _load():
         lib.oracle_tli_draft.restype = ctypes.c_int
         lib.oracle_slem_verify.argtypes = [ctypes.POINTER(_SlemArgs), ctypes.c_int32, ctypes.c_int32]
         lib.oracle_slem_verify.restype = ctypes.c_int
+        lib.oracle_tli_rates.argtypes = [ctypes.POINTER(_RatesArgs), ctypes.c_int32, ctypes.c_int32]
+        lib.oracle_tli_rates.restype = ctypes.c_int
         _lib = lib
     return _lib
 
@@ -310,6 +325,48 @@ def slem(target_logits, candidates, temperature, uniforms, lengths=None, probe_t
         rc = lib.oracle_slem_verify(ctypes.byref(args), lo_hi[0], lo_hi[1])
         if rc != 0:
             raise RuntimeError("oracle_slem_verify failed with code %d" % rc)
+
+    if threads == 1:
+        run((0, B))
+    else:
+        cuts = [(B * i) // threads for i in range(threads + 1)]
+        with ThreadPoolExecutor(max_workers=threads) as ex:
+            list(ex.map(run, [(cuts[i], cuts[i + 1]) for i in range(threads)]))
+    return out
+
+
+def rates(target_logits, drafter_logits, id_map, temperature, threads: int = 1) -> Dict[str, np.ndarray]:
+    """Expected acceptance rates per draft position: ``mass`` (drafter mass on the intersection),
+    ``alpha_union`` (drafting from q) and ``alpha_tli`` (drafting from q'), float64 [B,K]; ``flags`` int32 [B].
+    ``target_logits`` is [B,>=K,V_t] (rows 0..K-1 are read), ``drafter_logits`` [B,K,V_d]."""
+    lib = _load()
+    zt, zd = np.asarray(target_logits), np.asarray(drafter_logits)
+    if zt.dtype == np.float32 and zd.dtype == np.float32:
+        dtype = F32
+    elif zt.dtype == np.uint16 and zd.dtype == np.uint16:
+        dtype = BF16
+    else:
+        raise TypeError("logits must both be float32 or both be uint16 bfloat16 bit patterns")
+    if zt.ndim != 3 or zd.ndim != 3 or zt.strides[2] != zt.itemsize or zd.strides[2] != zd.itemsize:
+        raise ValueError("logits must be 3-d with a contiguous vocabulary axis")
+    B, K, V_d = zd.shape
+    if zt.shape[0] != B or zt.shape[1] < K:
+        raise ValueError("target logits must be [B,>=K,V_t]")
+    V_t = zt.shape[2]
+    idm = np.ascontiguousarray(id_map, dtype=np.int32)
+    tau = np.ascontiguousarray(temperature, dtype=np.float32).reshape(B)
+    out = {"mass": np.zeros((B, K)), "alpha_union": np.zeros((B, K)), "alpha_tli": np.zeros((B, K)),
+           "flags": np.zeros(B, np.int32)}
+    args = _RatesArgs(B, K, V_t, V_d, dtype, zt.ctypes.data, zt.strides[0] // zt.itemsize, zt.strides[1] // zt.itemsize,
+                      zd.ctypes.data, zd.strides[0] // zd.itemsize, zd.strides[1] // zd.itemsize,
+                      _ptr(idm), _ptr(tau), _ptr(out["mass"]), _ptr(out["alpha_union"]), _ptr(out["alpha_tli"]),
+                      _ptr(out["flags"]))
+    threads = max(1, min(int(threads), B))
+
+    def run(lo_hi):
+        rc = lib.oracle_tli_rates(ctypes.byref(args), lo_hi[0], lo_hi[1])
+        if rc != 0:
+            raise RuntimeError("oracle_tli_rates failed with code %d" % rc)
 
     if threads == 1:
         run((0, B))

@@ -42,7 +42,8 @@
  * The file also holds the drafting side of the same algorithms
  * (oracle_tli_draft): drawing the draft ids from q', and the verification step
  * of Algorithm 2, exact matching against sampled target tokens
- * (oracle_slem_verify); both at the end.
+ * (oracle_slem_verify), and the expected acceptance rates of the paper's table
+ * (oracle_tli_rates); all at the end.
  *
  * Parity status: every function here is pinned by tests that do not use this
  * file's own formulas (worked example, brute-force losslessness on tiny
@@ -607,5 +608,94 @@ int oracle_slem_verify(const oracle_slem_args *a, int32_t row_begin, int32_t row
         if (a->flags) a->flags[b] = flags;
     }
     free(p);
+    return 0;
+}
+
+/*
+ * Expected acceptance rates of one draft position, the paper's table of
+ * expected acceptance rates: for target p and drafter q of position (b, j),
+ *   mass        M       = sum_{x in T cap D} q(x)
+ *   alpha_union         = sum_{x in T cap D} min{p(x), q(x)}          (drafting from q)
+ *   alpha_tli           = sum_{x in T cap D} min{p(x), q(x) / M}      (drafting from q', Algorithm 4)
+ * with p = softmax(target row / tau), q = softmax(drafter row / tau) over all
+ * of D and p(x) read at the target id of x.  tau == 0 is the limit of one-hot
+ * distributions: q sits on the arg-max over D, q' on the arg-max over the
+ * intersection, p on the arg-max over T (lowest id on ties), so each rate is
+ * 0 or 1.  An empty intersection gives 0, 0, 0.  Parity status: pinned by the
+ * worked example, by Theorem 4.1 (alpha_union <= alpha_tli), by numpy's direct
+ * evaluation, by the closed forms for identity and disjoint maps, and by a
+ * Monte-Carlo run of the drafting and verification oracles whose empirical
+ * acceptance frequency must match alpha_tli.
+ */
+typedef struct {
+    int32_t B, K, V_t, V_d, dtype;
+    const void *target_logits;  /* [B, >=K, V_t], strides in elements; rows 0..K-1 are read */
+    int64_t t_stride_b, t_stride_k;
+    const void *drafter_logits; /* [B, K, V_d] */
+    int64_t d_stride_b, d_stride_k;
+    const int32_t *id_map;      /* [V_d] */
+    const float *temperature;   /* [B] */
+    /* outputs, [B, K] */
+    double *mass, *alpha_union, *alpha_tli;
+    int32_t *flags;             /* [B] */
+} oracle_rates_args;
+
+int oracle_tli_rates(const oracle_rates_args *a, int32_t row_begin, int32_t row_end)
+{
+    if (!a || a->B < 1 || a->K < 1 || a->V_t < 1 || a->V_d < 1) return -1;
+    if (a->dtype != ORACLE_F32 && a->dtype != ORACLE_BF16) return -1;
+    if (row_begin < 0 || row_end > a->B || row_begin > row_end) return -1;
+    const int K = a->K, V_t = a->V_t, V_d = a->V_d;
+    double *p = (double *)malloc(sizeof(double) * (size_t)V_t);
+    double *q = (double *)malloc(sizeof(double) * (size_t)V_d);
+    if (!p || !q) { free(p); free(q); return -3; }
+    for (int b = row_begin; b < row_end; ++b) {
+        const double tau = (double)a->temperature[b];
+        int flags = 0;
+        for (int j = 0; j < K; ++j) {
+            const int64_t o = (int64_t)b * K + j;
+            const int64_t t_off = (int64_t)b * a->t_stride_b + (int64_t)j * a->t_stride_k;
+            const int64_t d_off = (int64_t)b * a->d_stride_b + (int64_t)j * a->d_stride_k;
+            double M = 0.0, au = 0.0, at = 0.0;
+            if (!(tau >= 0.0) || isinf(tau)) {
+                flags |= FLAG_BAD_TEMPERATURE;
+            } else if (tau == 0.0) {
+                int finite = 1;
+                for (int t = 0; t < V_t; ++t) if (!isfinite(load_logit(a->target_logits, a->dtype, t_off + t))) finite = 0;
+                for (int x = 0; x < V_d; ++x) if (!isfinite(load_logit(a->drafter_logits, a->dtype, d_off + x))) finite = 0;
+                if (!finite) { flags |= FLAG_NONFINITE; }
+                else {
+                    const int at_id = argmax_row(a->target_logits, a->dtype, t_off, V_t);
+                    const int ad_all = argmax_row(a->drafter_logits, a->dtype, d_off, V_d);
+                    int ad_in = -1; double m = 0.0;
+                    for (int x = 0; x < V_d; ++x) {
+                        double z = load_logit(a->drafter_logits, a->dtype, d_off + x);
+                        if (a->id_map[x] >= 0 && (ad_in < 0 || z > m)) { m = z; ad_in = x; }
+                    }
+                    M = (a->id_map[ad_all] >= 0) ? 1.0 : 0.0;
+                    au = (a->id_map[ad_all] == at_id) ? 1.0 : 0.0;
+                    at = (ad_in >= 0 && a->id_map[ad_in] == at_id) ? 1.0 : 0.0;
+                    if (ad_in < 0) flags |= FLAG_FALLBACK;
+                }
+            } else if (!softmax_row(a->target_logits, a->dtype, t_off, V_t, tau, p) ||
+                       !softmax_row(a->drafter_logits, a->dtype, d_off, V_d, tau, q)) {
+                flags |= FLAG_NONFINITE;
+            } else {
+                int n_in = 0;
+                for (int x = 0; x < V_d; ++x) if (a->id_map[x] >= 0) { M += q[x]; ++n_in; }
+                if (n_in == 0) flags |= FLAG_FALLBACK;
+                for (int x = 0; x < V_d; ++x) {
+                    const int t = a->id_map[x];
+                    if (t < 0) continue;
+                    const double pt = p[t];
+                    au += (pt < q[x]) ? pt : q[x];
+                    if (M > 0.0) { const double qp = q[x] / M; at += (pt < qp) ? pt : qp; }
+                }
+            }
+            a->mass[o] = M; a->alpha_union[o] = au; a->alpha_tli[o] = at;
+        }
+        if (a->flags) a->flags[b] = flags;
+    }
+    free(p); free(q);
     return 0;
 }
