@@ -322,6 +322,43 @@ size_t tli_slem_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t M, int32_
  */
 int tli_slem_verify(tli_ctx *ctx, const tli_slem_args *args, void *cuda_stream);
 
+typedef struct {
+    int32_t B;      /* sequences, >= 1 */
+    int32_t K;      /* draft positions per sequence, 1 .. TLI_MAX_K; 2 * B * K <= TLI_MAX_B */
+    int32_t dtype;  /* TLI_F32 or TLI_BF16, for both logit tensors */
+    const void *target_logits;  /* [device] [B, >= K, V_t], as for tli_verify(); rows 0 .. K-1 are read */
+    int64_t t_stride_b, t_stride_k;
+    const void *drafter_logits; /* [device] [B, K, V_d] */
+    int64_t d_stride_b, d_stride_k;
+    const float *temperature;   /* [device] float[B] */
+    float *mass;                /* [device] out float[B, K]: drafter mass on the intersection, sum_{T cap D} q */
+    float *alpha_union;         /* [device] out float[B, K]: sum_{T cap D} min{p, q} */
+    float *alpha_tli;           /* [device] out float[B, K]: sum_{T cap D} min{p, q / mass} */
+    int32_t *position_status;   /* [device] out int32[B, K] of TLI_ROW_* bits; may be NULL */
+    void *workspace;            /* [device] scratch, 256-byte aligned, >= tli_rates_workspace_bytes() */
+    size_t workspace_bytes;
+} tli_rates_args;
+
+/* Bytes of device scratch tli_acceptance_rates() needs for (B, K, dtype); 0 on bad arguments. */
+size_t tli_rates_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype);
+
+/*
+ * Expected acceptance rates of every draft position, the paper's table of
+ * expected acceptance rates: with p = softmax(target row j / tau) and
+ * q = softmax(drafter row j / tau) over all of D,
+ *     mass        = sum_{x in T cap D} q(x)
+ *     alpha_union = sum_{x in T cap D} min{p(map x), q(x)}          drafting from q
+ *     alpha_tli   = sum_{x in T cap D} min{p(map x), q(x) / mass}   drafting from q' (Algorithm 4)
+ * (alpha_union <= alpha_tli, Theorem 4.1).  tau == 0 gives the one-hot limit:
+ * each value is 0 or 1.  An empty intersection gives zeros and
+ * TLI_ROW_FALLBACK; NaN or +inf in a row gives zeros and TLI_ROW_NONFINITE.
+ * Two passes over the drafter rows and one over the target rows plus one
+ * gathered target logit per id of the intersection.  For choosing a drafter
+ * and watching a deployment, not part of a decoding step.  Asynchronous,
+ * allocates nothing, uses the context's counters.
+ */
+int tli_acceptance_rates(tli_ctx *ctx, const tli_rates_args *args, void *cuda_stream);
+
 /*
  * Measurement hook: the three-kernel form of tli_verify() (see tli_set_fused)
  * with CUDA events recorded on `cuda_stream` around each kernel.  Blocks until

@@ -1591,6 +1591,326 @@ __global__ void __launch_bounds__(128) tli_slem_match_kernel(const SlemParams P)
 }
 
 // ---------------------------------------------------------------------------
+// expected acceptance rates of every draft position (the paper's table of expected acceptance rates)
+// ---------------------------------------------------------------------------
+//
+// Three small steps.  (1) Strip statistics of the K target rows and the K drafter rows of every
+// sequence: reference and sum of 2^(z*s - c), for drafter rows once over all of D and once over the
+// intersection (same reference).  (2) One CTA per row folds its strips.  (3) One CTA per 16 KB tile
+// of a drafter row walks the ids inside the intersection, gathers the target logit at map[x] and
+// adds min{p, q} and min{p, q'}; the last CTA of the pair (atomic ticket) adds the tiles in order.
+
+struct __align__(16) RateStrip {       // per strip of a row
+    double s_all, s_in;                // sums at reference c (temperature 0: best ids, all / inside)
+    float c, c_in;                     // reference (temperature 0: largest logit, all / inside)
+    int flags, pad;
+};
+struct __align__(16) RateRow {         // per row
+    double s_all, s_in;
+    float c, pad0;
+    int idx_all, idx_in, flags, pad1;
+};
+struct RateParams {
+    int B, K, V_t, V_d;
+    const void *zt; long long t_sb, t_sk;
+    const void *zd; long long d_sb, d_sk;
+    const int *map; const uint32_t *maskbits; const float *tau;
+    float *mass, *alpha_union, *alpha_tli; int *status;
+    RateStrip *strips;     // [2*B*K][nstrip_max]
+    RateRow *rows;         // [2*B*K]: target rows first, then drafter rows
+    double2 *tiles;        // [B*K][ntile_d]
+    unsigned *cnt;         // [B*K] tickets, zero between calls
+    int nstrip_t, nstrip_d, nstrip_max, ntile_d;
+};
+
+// grid (tiles of the longer kind of row, 2*B*K): blockIdx.y < B*K target rows, then drafter rows
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 6) tli_rate_stats_kernel(const RateParams P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const int BK = P.B * P.K;
+    const int row = blockIdx.y;
+    const bool drafter = row >= BK;
+    const int pair = drafter ? row - BK : row;
+    const int b = pair / P.K, j = pair - b * P.K;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int strip = blockIdx.x * kStripsPerTile + warp;
+    if (strip >= (drafter ? P.nstrip_d : P.nstrip_t)) return;
+    const float tau = __ldg(P.tau + b);
+    if (!(tau >= 0.f) || isinf(tau)) return;
+    const RowView<DT> rv = drafter
+        ? RowView<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk, P.V_d)
+        : RowView<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk, P.V_t);
+    const int nvec = rv.nvec();
+    float z[kVecPerThread][EPV];
+    uint32_t in_row[kVecPerThread], in_map[kVecPerThread];
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = strip * (32 * kVecPerThread) + k * 32 + lane;
+        in_row[k] = 0u; in_map[k] = 0u;
+        if (v < nvec) {
+            const int e0 = rv.first_elem(v);
+            unpack<DT>(rv.load(v), z[k]);
+            in_row[k] = (1u << EPV) - 1u;
+            if (e0 < 0) in_row[k] &= ~((1u << (-e0)) - 1u);
+            if (e0 + EPV > rv.V) in_row[k] &= (1u << (rv.V - e0)) - 1u;
+            if (drafter) in_map[k] = mask_bits(P.maskbits, e0) & in_row[k];
+        } else {
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) z[k][i] = -INFINITY;
+        }
+    }
+    RateStrip out;
+    out.pad = 0;
+    if (tau == 0.f) {
+        float ba = -INFINITY, bi = -INFINITY; int ia = INT_MAX, ii = INT_MAX; bool bad = false;
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const int e0 = rv.first_elem(strip * (32 * kVecPerThread) + k * 32 + lane);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                if ((in_row[k] >> i) & 1u) {
+                    bad = bad || !(z[k][i] < INFINITY);
+                    if (ia == INT_MAX || z[k][i] > ba) { ba = z[k][i]; ia = e0 + i; }
+                }
+                if ((in_map[k] >> i) & 1u) { if (ii == INT_MAX || z[k][i] > bi) { bi = z[k][i]; ii = e0 + i; } }
+            }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float b2 = __shfl_xor_sync(0xffffffffu, ba, o); int i2 = __shfl_xor_sync(0xffffffffu, ia, o);
+            if (better(b2, i2, ba, ia)) { ba = b2; ia = i2; }
+            b2 = __shfl_xor_sync(0xffffffffu, bi, o); i2 = __shfl_xor_sync(0xffffffffu, ii, o);
+            if (better(b2, i2, bi, ii)) { bi = b2; ii = i2; }
+        }
+        out.s_all = static_cast<double>(ia); out.s_in = static_cast<double>(ii); out.c = ba; out.c_in = bi;
+        out.flags = __any_sync(0xffffffffu, bad) ? static_cast<int>(TLI_ROW_NONFINITE) : 0;
+    } else {
+        const float s = 1.4426950408889634f / tau;
+        float mx = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k)
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) mx = fmaxf(mx, z[k][i]);
+        const float c = reference_for(warp_max(mx) * s);
+        double sa = 0.0, si = 0.0;
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            float wa = 0.f, wi = 0.f;
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                const float w = ex2(__fmaf_rn(z[k][i], s, -c));        // -inf outside the row: 0
+                wa = __fadd_rn(wa, w);
+                wi = __fadd_rn(wi, ((in_map[k] >> i) & 1u) ? w : 0.f);
+            }
+            sa += static_cast<double>(wa); si += static_cast<double>(wi);
+        }
+        out.s_all = warp_sum(sa); out.s_in = warp_sum(si); out.c = c; out.c_in = c; out.flags = 0;
+    }
+    if (lane == 0) {
+        const double2 *src = reinterpret_cast<const double2 *>(&out);
+        double2 *dst = reinterpret_cast<double2 *>(P.strips + static_cast<size_t>(row) * P.nstrip_max + strip);
+        __stcg(dst, src[0]); __stcg(dst + 1, src[1]);
+    }
+}
+
+// one CTA of 128 threads per row: the strips of a row at one reference, in strip order per thread
+__global__ void __launch_bounds__(128) tli_rate_rows_kernel(const RateParams P) {
+    __shared__ float sm_c[4]; __shared__ int sm_i[4], sm_i2[4]; __shared__ float sm_c2[4];
+    __shared__ double sm_a[4], sm_b[4]; __shared__ int sm_flags;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int BK = P.B * P.K;
+    const int row = blockIdx.x;
+    const bool drafter = row >= BK;
+    const int pair = drafter ? row - BK : row;
+    const int b = pair / P.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float tau = __ldg(P.tau + b);
+    if (!(tau >= 0.f) || isinf(tau)) return;
+    const int nstrip = drafter ? P.nstrip_d : P.nstrip_t;
+    const RateStrip *src = P.strips + static_cast<size_t>(row) * P.nstrip_max;
+    if (tid == 0) sm_flags = 0;
+    __syncthreads();
+    RateRow out;
+    out.pad0 = 0.f; out.pad1 = 0; out.idx_all = INT_MAX; out.idx_in = INT_MAX; out.s_all = 0.0; out.s_in = 0.0; out.c = kNegBig;
+    int flags = 0;
+    if (tau == 0.f) {
+        float ba = -INFINITY, bi = -INFINITY; int ia = INT_MAX, ii = INT_MAX;
+        for (int i = tid; i < nstrip; i += 128) {
+            const double2 lo = __ldcg(reinterpret_cast<const double2 *>(src + i));
+            const double2 hi = __ldcg(reinterpret_cast<const double2 *>(src + i) + 1);
+            const float2 cc = *reinterpret_cast<const float2 *>(&hi.x);
+            flags |= reinterpret_cast<const int2 *>(&hi.y)->x;
+            const int a2 = static_cast<int>(lo.x), i2 = static_cast<int>(lo.y);
+            if (better(cc.x, a2, ba, ia)) { ba = cc.x; ia = a2; }
+            if (better(cc.y, i2, bi, ii)) { bi = cc.y; ii = i2; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            float b2 = __shfl_xor_sync(0xffffffffu, ba, o); int i2 = __shfl_xor_sync(0xffffffffu, ia, o);
+            if (better(b2, i2, ba, ia)) { ba = b2; ia = i2; }
+            b2 = __shfl_xor_sync(0xffffffffu, bi, o); i2 = __shfl_xor_sync(0xffffffffu, ii, o);
+            if (better(b2, i2, bi, ii)) { bi = b2; ii = i2; }
+        }
+        if (lane == 0) { sm_c[warp] = ba; sm_i[warp] = ia; sm_c2[warp] = bi; sm_i2[warp] = ii; }
+        if (flags) atomicOr(&sm_flags, flags);
+        __syncthreads();
+        if (tid == 0) {
+            ba = sm_c[0]; ia = sm_i[0]; bi = sm_c2[0]; ii = sm_i2[0];
+            for (int w = 1; w < 4; ++w) {
+                if (better(sm_c[w], sm_i[w], ba, ia)) { ba = sm_c[w]; ia = sm_i[w]; }
+                if (better(sm_c2[w], sm_i2[w], bi, ii)) { bi = sm_c2[w]; ii = sm_i2[w]; }
+            }
+            out.idx_all = ia; out.idx_in = ii; out.flags = sm_flags;
+        }
+    } else {
+        float c = kNegBig;
+        for (int i = tid; i < nstrip; i += 128) {
+            const double2 hi = __ldcg(reinterpret_cast<const double2 *>(src + i) + 1);
+            c = fmaxf(c, reinterpret_cast<const float2 *>(&hi.x)->x);
+        }
+        c = warp_max(c);
+        if (lane == 0) sm_c[warp] = c;
+        __syncthreads();
+        c = fmaxf(fmaxf(sm_c[0], sm_c[1]), fmaxf(sm_c[2], sm_c[3]));
+        double sa = 0.0, si = 0.0;
+        for (int i = tid; i < nstrip; i += 128) {
+            const double2 lo = __ldcg(reinterpret_cast<const double2 *>(src + i));
+            const double2 hi = __ldcg(reinterpret_cast<const double2 *>(src + i) + 1);
+            const double f = pow2_neg_d(reinterpret_cast<const float2 *>(&hi.x)->x - c);
+            sa += lo.x * f; si += lo.y * f;
+        }
+        sa = warp_sum(sa); si = warp_sum(si);
+        if (lane == 0) { sm_a[warp] = sa; sm_b[warp] = si; }
+        __syncthreads();
+        if (tid == 0) {
+            out.s_all = ((sm_a[0] + sm_a[1]) + sm_a[2]) + sm_a[3];
+            out.s_in = ((sm_b[0] + sm_b[1]) + sm_b[2]) + sm_b[3];
+            out.c = c;
+            out.flags = (!isfinite(out.s_all) || !(out.s_all > 0.0)) ? static_cast<int>(TLI_ROW_NONFINITE) : 0;
+        }
+    }
+    if (tid == 0) {
+        const double2 *w = reinterpret_cast<const double2 *>(&out);
+        double2 *dst = reinterpret_cast<double2 *>(P.rows + row);
+        __stcg(dst, w[0]); __stcg(dst + 1, w[1]); __stcg(dst + 2, w[2]);
+    }
+}
+
+__device__ __forceinline__ RateRow load_rate_row(const RateRow *p) {
+    RateRow r;
+    double2 *w = reinterpret_cast<double2 *>(&r);
+    w[0] = __ldcg(reinterpret_cast<const double2 *>(p));
+    w[1] = __ldcg(reinterpret_cast<const double2 *>(p) + 1);
+    w[2] = __ldcg(reinterpret_cast<const double2 *>(p) + 2);
+    return r;
+}
+
+// grid (ntile_d, B*K)
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 6) tli_rate_pairs_kernel(const RateParams P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    __shared__ double sm_u[kWarps], sm_t[kWarps];
+    __shared__ int sm_last;
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    const int pair = blockIdx.y, tile = blockIdx.x;
+    const int b = pair / P.K, j = pair - b * P.K;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const float tau = __ldg(P.tau + b);
+    const int BK = P.B * P.K;
+    if (!(tau >= 0.f) || isinf(tau)) {
+        if (tile == 0 && tid == 0) {
+            P.mass[pair] = 0.f; P.alpha_union[pair] = 0.f; P.alpha_tli[pair] = 0.f;
+            if (P.status) P.status[pair] = TLI_ROW_BAD_TEMPERATURE;
+        }
+        return;
+    }
+    const RateRow rt = load_rate_row(P.rows + pair);
+    const RateRow rd = load_rate_row(P.rows + BK + pair);
+    int status = rt.flags | rd.flags;
+    if (tau == 0.f) {
+        if (tile == 0 && tid == 0) {
+            float M = 0.f, au = 0.f, at = 0.f;
+            if (!(status & TLI_ROW_NONFINITE)) {
+                const int t_all = (rd.idx_all != INT_MAX) ? __ldg(P.map + rd.idx_all) : -1;
+                const int t_in = (rd.idx_in != INT_MAX) ? __ldg(P.map + rd.idx_in) : -1;
+                M = t_all >= 0 ? 1.f : 0.f;
+                au = (t_all >= 0 && t_all == rt.idx_all) ? 1.f : 0.f;
+                at = (t_in >= 0 && t_in == rt.idx_all) ? 1.f : 0.f;
+                if (rd.idx_in == INT_MAX) status |= TLI_ROW_FALLBACK;
+            }
+            P.mass[pair] = M; P.alpha_union[pair] = au; P.alpha_tli[pair] = at;
+            if (P.status) P.status[pair] = status;
+        }
+        return;
+    }
+    if (status & TLI_ROW_NONFINITE) {
+        if (tile == 0 && tid == 0) {
+            P.mass[pair] = 0.f; P.alpha_union[pair] = 0.f; P.alpha_tli[pair] = 0.f;
+            if (P.status) P.status[pair] = TLI_ROW_NONFINITE;
+        }
+        return;
+    }
+    const float s = 1.4426950408889634f / tau;
+    const float rs_t = static_cast<float>(1.0 / rt.s_all);
+    const float rs_a = static_cast<float>(1.0 / rd.s_all);
+    const float rs_i = rd.s_in > 0.0 ? static_cast<float>(1.0 / rd.s_in) : 0.f;     // q' = e / S_in
+    const RowView<DT> rv(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk, P.V_d);
+    const long long t_off = static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk;
+    const int nvec = rv.nvec();
+    double au = 0.0, at = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = tile * kVecPerTile + k * kThreads + tid;
+        if (v >= nvec) continue;
+        const int e0 = rv.first_elem(v);
+        float z[EPV];
+        unpack<DT>(rv.load(v), z);
+        const uint32_t bits = mask_bits(P.maskbits, e0);
+        float su = 0.f, st = 0.f;
+#pragma unroll
+        for (int i = 0; i < EPV; ++i) {
+            const int x = e0 + i;
+            if (((bits >> i) & 1u) && x >= 0 && x < P.V_d) {
+                const int t = __ldg(P.map + x);
+                const float ed = ex2(__fmaf_rn(z[i], s, -rd.c));
+                const float et = ex2(__fmaf_rn(load_elt<DT>(P.zt, t_off + t), s, -rt.c));
+                const float p = __fmul_rn(et, rs_t);
+                su = __fadd_rn(su, fminf(p, __fmul_rn(ed, rs_a)));
+                st = __fadd_rn(st, fminf(p, __fmul_rn(ed, rs_i)));
+            }
+        }
+        au += static_cast<double>(su); at += static_cast<double>(st);
+    }
+    au = warp_sum(au); at = warp_sum(at);
+    if (lane == 0) { sm_u[warp] = au; sm_t[warp] = at; }
+    __syncthreads();
+    if (tid == 0) {
+        double u2 = 0.0, t2 = 0.0;
+#pragma unroll
+        for (int w = 0; w < kWarps; ++w) { u2 += sm_u[w]; t2 += sm_t[w]; }
+        __stcg(P.tiles + static_cast<size_t>(pair) * P.ntile_d + tile, make_double2(u2, t2));
+        __threadfence();
+        const unsigned ticket = atomicAdd(P.cnt + pair, 1u);
+        sm_last = (ticket == static_cast<unsigned>(P.ntile_d) - 1);
+        if (sm_last) P.cnt[pair] = 0;
+    }
+    __syncthreads();
+    if (!sm_last || tid != 0) return;
+    __threadfence();
+    double u2 = 0.0, t2 = 0.0;
+    for (int i = 0; i < P.ntile_d; ++i) {
+        const double2 v = __ldcg(P.tiles + static_cast<size_t>(pair) * P.ntile_d + i);
+        u2 += v.x; t2 += v.y;
+    }
+    const double M = rd.s_in / rd.s_all;
+    if (!(rd.s_in > 0.0)) status |= TLI_ROW_FALLBACK;          // empty intersection, or no mass in it
+    P.mass[pair] = static_cast<float>(M);
+    P.alpha_union[pair] = static_cast<float>(u2);
+    P.alpha_tli[pair] = static_cast<float>(t2);
+    if (P.status) P.status[pair] = status;
+}
+
+// ---------------------------------------------------------------------------
 // the fused kernel: statistics, decisions and sampling in one persistent grid
 // ---------------------------------------------------------------------------
 //
@@ -2742,6 +3062,78 @@ int tli_verify_static(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream)
     b.workspace = scratch;
     b.workspace_bytes = TLI_STATIC_SCRATCH_BYTES;
     return verify_impl(ctx, &b, cuda_stream, nullptr);
+}
+
+namespace {
+struct RateLayout { size_t strips, rows, tiles, total; int nstrip_t, nstrip_d, nstrip_max, ntile_t, ntile_d; };
+RateLayout rate_layout(const tli_ctx *ctx, int B, int K, int dtype) {
+    RateLayout L;
+    L.ntile_t = chunks_per_row(ctx->V_t, dtype, kVecPerTile);
+    L.ntile_d = chunks_per_row(ctx->V_d, dtype, kVecPerTile);
+    L.nstrip_t = L.ntile_t * kStripsPerTile; L.nstrip_d = L.ntile_d * kStripsPerTile;
+    L.nstrip_max = L.nstrip_t > L.nstrip_d ? L.nstrip_t : L.nstrip_d;
+    const size_t bk = static_cast<size_t>(B) * K;
+    size_t off = 0;
+    L.strips = off; off = align_up(off + sizeof(RateStrip) * 2 * bk * L.nstrip_max, 256);
+    L.rows = off;   off = align_up(off + sizeof(RateRow) * 2 * bk, 256);
+    L.tiles = off;  off = align_up(off + sizeof(double2) * bk * L.ntile_d, 256);
+    L.total = off;
+    return L;
+}
+}  // namespace
+
+size_t tli_rates_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype) {
+    if (!ctx || B < 1 || K < 1 || K > TLI_MAX_K || 2ll * B * K > TLI_MAX_B) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    return rate_layout(ctx, B, K, dtype).total;
+}
+
+int tli_acceptance_rates(tli_ctx *ctx, const tli_rates_args *a, void *cuda_stream) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
+    if (a->K > TLI_MAX_K || 2ll * a->B * a->K > TLI_MAX_B) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->target_logits || !a->drafter_logits || !a->temperature || !a->mass || !a->alpha_union || !a->alpha_tli)
+        return TLI_ERR_ARG;
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
+        return TLI_ERR_ARG;
+    if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
+    const RateLayout L = rate_layout(ctx, a->B, a->K, a->dtype);
+    if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
+        return TLI_ERR_WORKSPACE;
+    char *ws = reinterpret_cast<char *>(a->workspace);
+    RateParams P;
+    P.B = a->B; P.K = a->K; P.V_t = ctx->V_t; P.V_d = ctx->V_d;
+    P.zt = a->target_logits; P.t_sb = a->t_stride_b; P.t_sk = a->t_stride_k;
+    P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sk = a->d_stride_k;
+    P.map = ctx->d_map; P.maskbits = ctx->d_mask; P.tau = a->temperature;
+    P.mass = a->mass; P.alpha_union = a->alpha_union; P.alpha_tli = a->alpha_tli; P.status = a->position_status;
+    P.strips = reinterpret_cast<RateStrip *>(ws + L.strips);
+    P.rows = reinterpret_cast<RateRow *>(ws + L.rows);
+    P.tiles = reinterpret_cast<double2 *>(ws + L.tiles);
+    P.cnt = ctx->d_counters + (TLI_MAX_B + 1);
+    P.nstrip_t = L.nstrip_t; P.nstrip_d = L.nstrip_d; P.nstrip_max = L.nstrip_max; P.ntile_d = L.ntile_d;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const int bk = a->B * a->K;
+    const dim3 g1(static_cast<unsigned>(L.ntile_t > L.ntile_d ? L.ntile_t : L.ntile_d), static_cast<unsigned>(2 * bk));
+    if (a->dtype == TLI_F32) tli_rate_stats_kernel<TLI_F32><<<g1, kThreads, 0, stream>>>(P);
+    else tli_rate_stats_kernel<TLI_BF16><<<g1, kThreads, 0, stream>>>(P);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_rate_stats_kernel");
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1; cfg.stream = stream; cfg.dynamicSmemBytes = 0;
+    cfg.gridDim = dim3(static_cast<unsigned>(2 * bk)); cfg.blockDim = dim3(128);
+    if ((e = cudaLaunchKernelEx(&cfg, tli_rate_rows_kernel, P)) != cudaSuccess) return cuda_fail(e, "launch tli_rate_rows_kernel");
+    cfg.gridDim = dim3(static_cast<unsigned>(L.ntile_d), static_cast<unsigned>(bk)); cfg.blockDim = dim3(kThreads);
+    if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_rate_pairs_kernel<TLI_F32>, P);
+    else e = cudaLaunchKernelEx(&cfg, tli_rate_pairs_kernel<TLI_BF16>, P);
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_rate_pairs_kernel");
+    return TLI_OK;
 }
 
 namespace {

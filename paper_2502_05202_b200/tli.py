@@ -39,7 +39,7 @@ TLI_STATIC_SCRATCH_BYTES = 4194304
 
 EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
-           "tli_verify_host_buffer_bytes", "tli_verify_host",
+           "tli_verify_host_buffer_bytes", "tli_verify_host", "tli_rates_workspace_bytes", "tli_acceptance_rates",
            "tli_ctx_info",
            "tli_status_string", "tli_last_cuda_error")
 
@@ -64,6 +64,18 @@ class tli_verify_host_args(ctypes.Structure):
         ("temperature", ctypes.c_void_p), ("uniforms", ctypes.c_void_p),
         ("accepted", ctypes.c_void_p), ("next_token", ctypes.c_void_p), ("row_status", ctypes.c_void_p),
         ("device_buffer", ctypes.c_void_p), ("device_buffer_bytes", ctypes.c_size_t),
+    ]
+
+
+class tli_rates_args(ctypes.Structure):
+    _fields_ = [
+        ("B", ctypes.c_int32), ("K", ctypes.c_int32), ("dtype", ctypes.c_int32),
+        ("target_logits", ctypes.c_void_p), ("t_stride_b", ctypes.c_int64), ("t_stride_k", ctypes.c_int64),
+        ("drafter_logits", ctypes.c_void_p), ("d_stride_b", ctypes.c_int64), ("d_stride_k", ctypes.c_int64),
+        ("temperature", ctypes.c_void_p),
+        ("mass", ctypes.c_void_p), ("alpha_union", ctypes.c_void_p), ("alpha_tli", ctypes.c_void_p),
+        ("position_status", ctypes.c_void_p),
+        ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
     ]
 
 
@@ -134,6 +146,10 @@ def load() -> ctypes.CDLL:
         lib.tli_verify_host_buffer_bytes.restype = ctypes.c_size_t
         lib.tli_verify_host.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_host_args), ctypes.c_void_p]
         lib.tli_verify_host.restype = ctypes.c_int
+        lib.tli_rates_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_rates_workspace_bytes.restype = ctypes.c_size_t
+        lib.tli_acceptance_rates.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_rates_args), ctypes.c_void_p]
+        lib.tli_acceptance_rates.restype = ctypes.c_int
         lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_fused.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
@@ -258,6 +274,41 @@ def tli_verify_host(ctx: int, args: tli_verify_host_args, stream: Optional[int] 
     rc = load().tli_verify_host(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify_host")
+
+
+def tli_rates_workspace_bytes(ctx: int, B: int, K: int, dtype: int) -> int:
+    return int(load().tli_rates_workspace_bytes(ctx, B, K, dtype))
+
+
+def make_rates_args(target_logits: torch.Tensor, drafter_logits: torch.Tensor, temperature: torch.Tensor,
+                    mass: torch.Tensor, alpha_union: torch.Tensor, alpha_tli: torch.Tensor, workspace: torch.Tensor,
+                    position_status: Optional[torch.Tensor] = None) -> tli_rates_args:
+    """Fill a tli_rates_args from device tensors (no copies; the tensors must outlive the call)."""
+    B, K, _ = drafter_logits.shape
+    dt = _logit_dtype(target_logits)
+    if _logit_dtype(drafter_logits) != dt:
+        raise TypeError("both logit tensors must have the same dtype")
+    if target_logits.stride(2) != 1 or drafter_logits.stride(2) != 1:
+        raise ValueError("the vocabulary axis must be contiguous")
+    if target_logits.shape[0] != B or target_logits.shape[1] < K:
+        raise ValueError("target logits must be [B, >=K, V_t]")
+    for name, t in (("mass", mass), ("alpha_union", alpha_union), ("alpha_tli", alpha_tli)):
+        if t.dtype != torch.float32 or tuple(t.shape) != (B, K) or not t.is_contiguous():
+            raise ValueError("%s must be a contiguous float32 tensor of shape %s" % (name, (B, K)))
+    return tli_rates_args(B, K, dt, target_logits.data_ptr(), target_logits.stride(0), target_logits.stride(1),
+                          drafter_logits.data_ptr(), drafter_logits.stride(0), drafter_logits.stride(1),
+                          temperature.data_ptr(), mass.data_ptr(), alpha_union.data_ptr(), alpha_tli.data_ptr(),
+                          None if position_status is None else position_status.data_ptr(),
+                          workspace.data_ptr(), workspace.numel() * workspace.element_size())
+
+
+def tli_acceptance_rates(ctx: int, args: tli_rates_args, stream: Optional[int] = None) -> None:
+    """tli_acceptance_rates() on ``stream`` (a cudaStream_t as int; default: torch's current stream)."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_acceptance_rates(ctx, ctypes.byref(args), ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_acceptance_rates")
 
 
 def tli_draft_workspace_bytes(ctx: int, B: int, R: int, dtype: int) -> int:
@@ -403,6 +454,22 @@ class Verifier:
         args = make_draft_args(drafter_logits, temperature, uniforms, out["draft_ids"], self._ws,
                                out["q_draft"], out["draft_status"])
         tli_draft_sample(self.ctx, args)
+        return out
+
+    def rates(self, target_logits, drafter_logits, temperature) -> Dict[str, torch.Tensor]:
+        """Expected acceptance rates per draft position (mass, alpha_union, alpha_tli); device tensors."""
+        B, K, _ = drafter_logits.shape
+        dev = self.device
+        out = {k: torch.empty(B, K, dtype=torch.float32, device=dev) for k in ("mass", "alpha_union", "alpha_tli")}
+        out["position_status"] = torch.empty(B, K, dtype=torch.int32, device=dev)
+        need = tli_rates_workspace_bytes(self.ctx, B, K, _logit_dtype(target_logits))
+        if need == 0:
+            raise TLIError(TLI_ERR_UNSUPPORTED, "tli_rates_workspace_bytes")
+        if self._ws is None or self._ws.numel() < need:
+            self._ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        args = make_rates_args(target_logits, drafter_logits, temperature, out["mass"], out["alpha_union"],
+                               out["alpha_tli"], self._ws, out["position_status"])
+        tli_acceptance_rates(self.ctx, args)
         return out
 
     def slem(self, target_logits, candidates, temperature, uniforms, lengths=None) -> Dict[str, torch.Tensor]:
