@@ -337,6 +337,35 @@ class GpuCase:
                 "rows_per_call": cfg.B * (cfg.K + 1), "bytes_per_call": nbytes,
                 "mean_accepted": float(acc.float().mean().item())}
 
+    def rates_timing(self, steps):
+        """tli_acceptance_rates() on this workload (K positions per sequence): ms per call."""
+        torch, tli, cfg = self.torch, self.tli, self.cfg
+        dev = self.zt[0].device
+        dt = tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16
+        need = tli.tli_rates_workspace_bytes(self.ver.ctx, cfg.B, cfg.K, dt)
+        if need == 0:
+            return None
+        outs = [torch.empty(cfg.B, cfg.K, dtype=torch.float32, device=dev) for _ in range(3)]
+        st = torch.empty(cfg.B, cfg.K, dtype=torch.int32, device=dev)
+        ws = torch.empty(need, dtype=torch.uint8, device=dev)
+        args = [tli.make_rates_args(zt, zd, self.tau, *outs, ws, st) for zt, zd in zip(self.zt, self.zd)]
+        n = [0]
+
+        def step():
+            tli.tli_acceptance_rates(self.ver.ctx, args[n[0] % len(args)], self.stream)
+            n[0] += 1
+        for _ in range(3 + len(args)):
+            step()
+        ms = timed(torch, None, steps, step, 1) / steps
+        assert int(st.abs().sum()) == 0, "position_status not clean on benchmark inputs"
+        greedy = int((self.tau == 0).sum())
+        # target rows once, drafter rows twice (statistics, then the pair pass); the gathers are not counted
+        nbytes = cfg.elt * cfg.B * cfg.K * (cfg.V_t + 2 * cfg.V_d)
+        return {"ms_per_call": ms, "positions_per_s": cfg.B * cfg.K / (ms * 1e-3), "gbs": nbytes / (ms * 1e-3) / 1e9,
+                "bytes_per_call": nbytes, "greedy_sequences": greedy,
+                "mean_alpha_tli": float(outs[2].mean().item()), "mean_alpha_union": float(outs[1].mean().item()),
+                "mean_mass": float(outs[0].mean().item())}
+
     def e2e_bytes(self):
         h = self.host
         h2d = sum(h[k].numel() * h[k].element_size() for k in ("zt", "zd", "draft", "tau", "u"))
@@ -432,6 +461,7 @@ def gpu_arm(args):
     calls = call_timings(case, torch, args.steps)
     draft = case.draft_timing(max(args.steps, 20)) if world == 1 else None
     slem = case.slem_timing(max(args.steps, 20)) if world == 1 else None
+    rates = case.rates_timing(max(args.steps, 20)) if world == 1 else None
     clocks = sampler.stop() if rank == 0 else None
     case.check()
     # end to end: host buffers in, host results out
@@ -460,6 +490,7 @@ def gpu_arm(args):
         "per_call": calls,
         "draft_sample": draft,
         "slem_verify": slem,
+        "acceptance_rates": rates,
         "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
                      "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
                      "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
@@ -479,7 +510,7 @@ def gpu_arm(args):
                 per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
                             "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
                             "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls,
-                            "draft_sample": draft, "slem_verify": slem})
+                            "draft_sample": draft, "slem_verify": slem, "acceptance_rates": rates})
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
@@ -491,6 +522,7 @@ def gpu_arm(args):
             kc = call_timings(k, torch, steps)
             kc["draft_sample"] = k.draft_timing(steps)
             kc["slem_verify"] = k.slem_timing(steps)
+            kc["acceptance_rates"] = k.rates_timing(steps)
             k.check()
             per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
                         "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
