@@ -20,6 +20,11 @@
 //   tli_select_kernel  large batches only: those inversions as a kernel of their own.
 //   tli_fused_kernel   all of the above in one persistent grid (tli_set_fused; not the default).
 //
+// Beside the verification call: tli_draft_kernel / tli_draft_select_kernel draw one id per row of
+// logits by inverse CDF (the drafts from q' for tli_draft_sample; with no mask, the target tokens
+// of Algorithm 2 for tli_slem_verify, compared by tli_slem_match_kernel), and tli_rate_*_kernel
+// form the paper's expected acceptance rates per draft position (tli_acceptance_rates).
+//
 // Softmax terms are formed as ex2(fma(z, s, -c)) with an integer-valued reference c in log2
 // units: the only per-term rounding is the one in the fma, and every change or combination of
 // references is an exact power of two.
