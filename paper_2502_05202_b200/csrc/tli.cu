@@ -1648,6 +1648,17 @@ __global__ void __launch_bounds__(kThreads, 6) tli_rate_stats_kernel(const RateP
     const int nvec = rv.nvec();
     float z[kVecPerThread][EPV];
     uint32_t in_row[kVecPerThread], in_map[kVecPerThread];
+    const int v0 = strip * (32 * kVecPerThread);
+    const bool interior = rv.first_elem(v0) >= 0 && rv.first_elem(v0 + 32 * kVecPerThread - 1) + EPV <= rv.V;
+    if (interior) {                                   // the whole strip inside the row: no per-vector tests
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const int v = v0 + k * 32 + lane;
+            unpack<DT>(__ldg(rv.vec0 + v), z[k]);
+            in_row[k] = (1u << EPV) - 1u;
+            in_map[k] = drafter ? (mask_bits(P.maskbits, rv.first_elem(v)) & in_row[k]) : 0u;
+        }
+    } else
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
         const int v = strip * (32 * kVecPerThread) + k * 32 + lane;
@@ -1863,20 +1874,33 @@ __global__ void __launch_bounds__(kThreads, 6) tli_rate_pairs_kernel(const RateP
     const long long t_off = static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk;
     const int nvec = rv.nvec();
     double au = 0.0, at = 0.0;
+    const int v_first = tile * kVecPerTile;
+    const bool lean = (rv.head & 3) == 0 && rv.first_elem(v_first) >= 0 &&
+                      rv.first_elem(v_first + kVecPerTile - 1) + EPV <= rv.V;     // the same for the whole CTA
 #pragma unroll
     for (int k = 0; k < kVecPerThread; ++k) {
-        const int v = tile * kVecPerTile + k * kThreads + tid;
-        if (v >= nvec) continue;
+        const int v = v_first + k * kThreads + tid;
+        if (!lean && v >= nvec) continue;
         const int e0 = rv.first_elem(v);
         float z[EPV];
-        unpack<DT>(rv.load(v), z);
-        const uint32_t bits = mask_bits(P.maskbits, e0);
+        int tmap[EPV];
+        if (lean) {                                   // whole tile inside an aligned row: vector loads, no range tests
+            unpack<DT>(__ldg(rv.vec0 + v), z);
+#pragma unroll
+            for (int i = 0; i < EPV; i += 4) {
+                const int4 q = __ldg(reinterpret_cast<const int4 *>(P.map + e0 + i));
+                tmap[i] = q.x; tmap[i + 1] = q.y; tmap[i + 2] = q.z; tmap[i + 3] = q.w;
+            }
+        } else {
+            unpack<DT>(rv.load(v), z);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) tmap[i] = (e0 + i >= 0 && e0 + i < P.V_d) ? __ldg(P.map + e0 + i) : -1;
+        }
         float su = 0.f, st = 0.f;
 #pragma unroll
         for (int i = 0; i < EPV; ++i) {
-            const int x = e0 + i;
-            if (((bits >> i) & 1u) && x >= 0 && x < P.V_d) {
-                const int t = __ldg(P.map + x);
+            if (tmap[i] >= 0) {
+                const int t = tmap[i];
                 const float ed = ex2(__fmaf_rn(z[i], s, -rd.c));
                 const float et = ex2(__fmaf_rn(load_elt<DT>(P.zt, t_off + t), s, -rt.c));
                 const float p = __fmul_rn(et, rs_t);
