@@ -220,3 +220,17 @@ def test_argument_errors_are_reported_not_launched():
     assert tli.tli_draft_workspace_bytes(v.ctx, 70000, 1, tli.TLI_F32) == 0
     torch.cuda.synchronize()
     v.close()
+
+
+def test_largest_vocabulary_and_most_rows():
+    """V_d at the library's limit (fp32: 257 tiles, 2056 strips per row) and B * R at its limit."""
+    V_d = 1 << 20
+    z, id_map, tau, u, V_t = make(1, 2, V_d, wl.F32, 0.3, seed=180, taus=(0.9,), V_t=V_d)
+    gpu = run_gpu(z, id_map, [0.9], u, V_t)
+    compare(z, id_map, [0.9], u, gpu)
+    gpu0 = run_gpu(z, id_map, [0.0], u, V_t)
+    compare(z, id_map, [0.0], u, gpu0)
+    B = 65535
+    z, id_map, tau, u, V_t = make(B, 1, 40, wl.BF16, 0.5, seed=181)
+    many = run_gpu(z, id_map, tau, u, V_t)
+    compare(z, id_map, tau, u, many)

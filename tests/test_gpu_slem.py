@@ -188,3 +188,14 @@ def test_argument_errors_are_reported_not_launched():
     assert tli.tli_slem_workspace_bytes(v.ctx, 0, 1, tli.TLI_F32) == 0
     torch.cuda.synchronize()
     v.close()
+
+
+def test_largest_vocabulary_and_most_rows():
+    """V_t at the library's limit (fp32: 257 tiles, 2056 strips per row) and B * (M+1) at its limit."""
+    z, cand, tau, u = make(1, 1, 1 << 20, wl.F32, seed=280, taus=(0.0, 0.9))
+    for t in ([0.9], [0.0]):
+        gpu = run_gpu(z, cand, t, u)
+        compare(z, cand, t, u, gpu)
+    z, cand, tau, u = make(21845, 2, 50, wl.BF16, seed=281)
+    gpu = run_gpu(z, cand, tau, u)
+    compare(z, cand, tau, u, gpu)
