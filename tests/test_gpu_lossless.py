@@ -83,3 +83,45 @@ def test_exact_matching_is_lossless_on_the_gpu(dtype):
         assert reached.sum() > 300
         chi2_ok(tok, softmax(zt_h[j], tau), "position %d" % j)
     v.close()
+
+
+def test_a_whole_speculation_step_replays_from_a_cuda_graph():
+    """Draft from q', verify, exact-match and acceptance rates recorded into one graph: every call only
+    launches kernels, so the replay must reproduce the eager results bit for bit."""
+    from paper_2502_05202_b200 import workload as wl
+    cfg = wl.tiny_config(B=10, K=3, V_t=50021, V_d=30011, dtype=wl.BF16, f_mapped=0.6, sigma_d=0.5,
+                         temperatures=(0.0, 0.8, 1.0), seed=91)
+    b = wl.make_batch(cfg)
+    dev = lambda a: torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    zt, zd = dev(b["target_logits"]).view(torch.bfloat16), dev(b["drafter_logits"]).view(torch.bfloat16)
+    tau, u = dev(b["temperature"]), dev(b["uniforms"])
+    ud = u[:, :cfg.K].contiguous()
+    idmap = dev(b["id_map"])
+    v = tli.Verifier(cfg.V_t, cfg.V_d, b["id_map"])
+    v._ws = torch.empty(64 << 20, dtype=torch.uint8, device="cuda")          # one scratch for all four calls
+
+    def step():
+        d = v.draft(zd, tau, ud)
+        out = v.verify(zt, zd, d["draft_ids"], tau, u)
+        cand = idmap[d["draft_ids"].long()].contiguous()
+        s = v.slem(zt, cand, tau, u)
+        r = v.rates(zt, zd, tau)
+        return [d["draft_ids"], out["accepted"], out["next_token"], s["accepted"], s["next_token"], r["alpha_tli"]]
+
+    eager = [t.clone() for t in step()]
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g, stream=side):
+        outs = step()
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(3):
+        for t in outs:
+            t.zero_()
+        g.replay()
+        torch.cuda.synchronize()
+        for a, e in zip(outs, eager):
+            assert torch.equal(a, e)
+    del g
+    v.close()
