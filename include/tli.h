@@ -17,6 +17,8 @@
  *     be recorded into a CUDA graph by stream capture and replayed; calls on
  *     one context must not overlap in time (they share the context's
  *     counters), so replays of such a graph are serialised by the caller.
+ *     The same holds for tli_draft_sample(), tli_slem_verify() and
+ *     tli_acceptance_rates(); tli_verify_host() adds only stream-ordered copies.
  *   - Functions return TLI_OK or a negative tli error code.  Errors in the
  *     data (a draft id outside the vocabulary, a NaN logit, a negative
  *     temperature) never fault: they set bits in row_status.
