@@ -184,3 +184,28 @@ def test_bf16_strides_threads_and_probe():
     np.testing.assert_allclose(pr["probe_lo"][sampled], a["cdf_lo"][sampled], atol=1e-15)
     np.testing.assert_allclose(pr["probe_hi"][sampled], a["cdf_hi"][sampled], atol=1e-15)
     np.testing.assert_allclose(pr["probe_w"][sampled], a["q_draft"][sampled], rtol=1e-12)
+
+
+def test_the_chi_square_pin_catches_a_drafter_that_forgets_the_intersection():
+    """Sensitivity of the pin above: ids drawn from q (no renormalisation onto the intersection) fail it."""
+    rng = np.random.default_rng(21)
+    V_d, N, tau = 12, 400_000, 1.0
+    z = rng.normal(0, 1.5, V_d).astype(np.float32)
+    mapped = np.zeros(V_d, bool)
+    mapped[rng.choice(V_d, 7, replace=False)] = True
+    want = masked_softmax(z, mapped, tau)
+    q = np.exp((z.astype(np.float64) - z.max()) / tau)
+    q /= q.sum()
+    wrong = rng.choice(V_d, N, p=q)                                   # a sampler that ignores the mask
+    kept = wrong[mapped[wrong]]                                       # even after dropping the ids outside it ...
+    counts = np.bincount(kept, minlength=V_d)
+    n = len(kept)
+    chi2 = ((counts[mapped] - n * want[mapped]) ** 2 / (n * want[mapped])).sum()
+    assert stats.chi2.sf(chi2, mapped.sum() - 1) > 1e-4                # ... the conditional law is q' (rejection sampling),
+    assert (~mapped[wrong]).mean() > 0.05                             # but a share of the draws lies outside T: the pin's
+    # first assertion (every id inside the intersection) is what such a drafter fails.
+    off_by_one = np.searchsorted(np.cumsum(want), rng.random(N), side="left") + 1      # a CDF walk shifted by one id
+    counts = np.bincount(np.clip(off_by_one, 0, V_d - 1), minlength=V_d)
+    keep = want > 0
+    chi2 = ((counts[keep] - N * want[keep]) ** 2 / (N * want[keep])).sum()
+    assert stats.chi2.sf(chi2, keep.sum() - 1) < 1e-4                  # the chi-square rejects it
