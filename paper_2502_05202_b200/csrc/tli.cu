@@ -987,7 +987,11 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
 // The CDF inversion for one sequence by one CTA, tile -> vector -> element, from the tile sums in
 // the workspace.  Either the last CTA of the sampling kernel to finish a tile of the sequence runs
 // it, or (large batches) the selection kernel does, one CTA per sequence.
-template <int DT>
+// KEEP: each thread forms the weights of four consecutive vectors of the chosen tile and keeps them
+// in registers, so that the final walk needs no second trip to memory (the selection kernel, which
+// has the registers); otherwise the vector the target falls into is formed again (inside the
+// sampling kernel, whose 32 registers per thread would spill them).
+template <int DT, bool KEEP = false>
 __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowView<DT> &rt, const void *zd_row) {
     constexpr int EPV = Elt<DT>::kPerVec;
     __shared__ double sm_red[kWarps];
@@ -1046,26 +1050,43 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
     const int T = sm_tile;
     const double rem = sm_rem;
     const int nvec = rt.nvec();
-    // vector sums of tile T in address order
-#pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) {
-        const int g = k * kThreads + tid;
-        const int v = T * kVecPerTile + g;
-        float sseg = 0.f;
-        if (v < nvec) {
-            float w[EPV];
-            vector_weights<DT>(P, sel, rt, zd_row, v, w);
-            sseg = ordered_sum(w);
-        }
-        sm_seg[g] = sseg;
-    }
-    if (tid == 0) { sm_found = INT_MAX; sm_lastpos = -1; }
-    __syncthreads();
-    // thread i owns vectors 4i .. 4i+3: block-wide exclusive prefix in fp64
+    // vector sums of tile T; thread i owns vectors 4i .. 4i+3 in the block-wide exclusive prefix (fp64)
+    float wv[KEEP ? kVecPerThread : 1][EPV];
     double loc[kVecPerThread];
     double mine = 0.0;
+    if constexpr (KEEP) {
 #pragma unroll
-    for (int k = 0; k < kVecPerThread; ++k) { loc[k] = static_cast<double>(sm_seg[tid * kVecPerThread + k]); mine += loc[k]; }
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const int v = T * kVecPerTile + tid * kVecPerThread + k;
+            float sseg = 0.f;
+            if (v < nvec) {
+                vector_weights<DT>(P, sel, rt, zd_row, v, wv[k]);
+                sseg = ordered_sum(wv[k]);
+            } else {
+#pragma unroll
+                for (int i = 0; i < EPV; ++i) wv[k][i] = 0.f;
+            }
+            loc[k] = static_cast<double>(sseg); mine += loc[k];
+        }
+        if (tid == 0) { sm_found = INT_MAX; sm_lastpos = -1; }
+    } else {
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) {
+            const int g = k * kThreads + tid;
+            const int v = T * kVecPerTile + g;
+            float sseg = 0.f;
+            if (v < nvec) {
+                float w[EPV];
+                vector_weights<DT>(P, sel, rt, zd_row, v, w);
+                sseg = ordered_sum(w);
+            }
+            sm_seg[g] = sseg;
+        }
+        if (tid == 0) { sm_found = INT_MAX; sm_lastpos = -1; }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < kVecPerThread; ++k) { loc[k] = static_cast<double>(sm_seg[tid * kVecPerThread + k]); mine += loc[k]; }
+    }
     double incl = mine;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
@@ -1106,7 +1127,16 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
         const double rem2 = (found != INT_MAX) ? (rem - before) : INFINITY;
         float w[EPV];
         const int v = T * kVecPerTile + G;
-        vector_weights<DT>(P, sel, rt, zd_row, v, w);
+        if constexpr (KEEP) {
+#pragma unroll
+            for (int k = 0; k < kVecPerThread; ++k)
+                if (k == G - tid * kVecPerThread) {
+#pragma unroll
+                    for (int i = 0; i < EPV; ++i) w[i] = wv[k][i];
+                }
+        } else {
+            vector_weights<DT>(P, sel, rt, zd_row, v, w);
+        }
         float runf = 0.f;
         int pick = -1, lastw = 0;
 #pragma unroll
@@ -1167,7 +1197,7 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
     RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
     const void *zd_row = reinterpret_cast<const char *>(P.zd) +
         (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
-    select_sequence<DT>(P, b, sel, rt, zd_row);
+    select_sequence<DT, true>(P, b, sel, rt, zd_row);
 }
 
 // ---------------------------------------------------------------------------
