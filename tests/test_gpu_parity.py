@@ -226,6 +226,24 @@ def test_extreme_batch_and_draft_counts(B, K):
     check(wl.make_batch(cfg))
 
 
+def test_most_sequences_in_one_call():
+    """B at the library's limit (65535 sequences of a small vocabulary)."""
+    rng = np.random.default_rng(61)
+    B, K, V_t, V_d = tli.TLI_MAX_B, 2, 96, 80
+    zt = rng.normal(0, 2, (B, K + 1, V_t)).astype(np.float32)
+    id_map = np.full(V_d, -1, np.int32)
+    inside = rng.choice(V_d, 56, replace=False)
+    id_map[inside] = rng.permutation(V_t)[:56]
+    zd = rng.normal(-2, 1, (B, K, V_d)).astype(np.float32)
+    zd[:, :, inside] = zt[:, :K, id_map[inside]] + rng.normal(0, 0.3, (B, K, 56)).astype(np.float32)
+    batch = {"target_logits": zt, "drafter_logits": zd, "id_map": id_map,
+             "draft_ids": inside[rng.integers(0, 56, (B, K))].astype(np.int32),
+             "temperature": rng.choice(np.array([0.0, 0.7, 1.0], np.float32), B),
+             "uniforms": rng.integers(0, 1 << 24, (B, K + 1)).astype(np.float32) / np.float32(1 << 24)}
+    rep = check(batch, threads=16)
+    assert rep.rows == B and rep.exact >= B - 50
+
+
 def test_large_vocabulary_near_the_limit():
     cfg = wl.tiny_config(B=2, K=1, V_t=tli.TLI_MAX_V, V_d=tli.TLI_MAX_V - 7, dtype=wl.F32, f_mapped=0.5, seed=60)
     check(wl.make_batch(cfg))
