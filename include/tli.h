@@ -132,8 +132,7 @@ typedef struct {
                                  * sequence b count; its later drafter rows and its target rows beyond
                                  * row draft_lengths[b] are not read, and when all counted drafts are
                                  * accepted the extra token is drawn from target row draft_lengths[b].
-                                 * The extra token still uses uniforms[b, K].  NULL = K for all.
-                                 * Not available in the fused form (TLI_ERR_UNSUPPORTED) */
+                                 * The extra token still uses uniforms[b, K].  NULL = K for all */
 } tli_verify_args;
 
 /*
@@ -362,26 +361,28 @@ size_t tli_rates_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32
 int tli_acceptance_rates(tli_ctx *ctx, const tli_rates_args *args, void *cuda_stream);
 
 /*
- * Measurement hook: the three-kernel form of tli_verify() (see tli_set_fused)
- * with CUDA events recorded on `cuda_stream` around each kernel.  Blocks until
- * the call has finished and writes three durations in milliseconds to [host]
- * ms[3]: ms[0] the statistics pass over all logits, ms[1] the per-sequence
- * decision, ms[2] the sampling pass over one row per sequence.  Creates and
- * destroys four events per call; not meant for the serving path.
+ * Measurement hook: tli_verify() with CUDA events recorded on `cuda_stream`
+ * around each kernel.  Blocks until the call has finished and writes three
+ * durations in milliseconds to [host] ms[3]: ms[0] the statistics pass over
+ * all logits, ms[1] the per-sequence decision kernel (0 when the cluster kernel
+ * decides and samples in one launch, see tli_set_tiled), ms[2] the sampling
+ * pass over one row per sequence.  Creates and destroys four events per call;
+ * not meant for the serving path.
  */
 int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream, float *ms);
 
 /*
- * How tli_verify() and tli_verify_static() run on this context.  enabled = 0
- * (default): three kernels one after the other (statistics, decision,
- * sampling).  enabled = 1: one persistent kernel that streams the statistics,
- * decides each sequence as soon as its last statistic has arrived and draws its
- * extra token while later sequences are still streaming.  Results are identical
- * bit for bit.  The fused form is the slower one today (its sampling chunks
- * stall the streaming warps on their gathers) and is kept as the basis for
- * further work.
+ * How tli_verify() and tli_verify_static() draw the extra token of Algorithm 5
+ * (the residual or bonus sample) on this context.  enabled = 0 (default): by
+ * size -- one kernel of one thread-block cluster per sequence (decision and
+ * sample together) when a target row fits the shared memory of a cluster and
+ * the batch is moderate, the tile kernels (decision, tile sums, inversion)
+ * otherwise.  enabled = 1: always the tile kernels.  Both forms compute the
+ * same weights element by element; they add them in different orders, so their
+ * tokens can differ where uniforms[b,K] * total lies within rounding of a CDF
+ * boundary.  For tests and measurements.
  */
-int tli_set_fused(tli_ctx *ctx, int enabled);
+int tli_set_tiled(tli_ctx *ctx, int enabled);
 
 /*
  * Self-test of the kernels' bounded waits.  Every wait inside the kernels (on a

@@ -82,14 +82,16 @@ struct Params {
     unsigned *cnt_stats; unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
     unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
-    unsigned *samp_counter;             // fused kernel: next sampling item; zero between calls
-    int *seq_state;                     // fused kernel: SEQ_* per sequence; zero between calls
-    double *stripsum;                   // fused kernel: [B][nct][kSWarps] weight sums in target-id order
     int nct, ncd;        // statistics-kernel chunks per target / drafter row
     int ntile;           // 16 KB tiles per target row (sampling pass)
     int split_select;    // 1: the CDF inversions run as a kernel of their own
     int cps;             // chunks per segment
     int nst, nsd;        // segments per target / drafter row
+    int B_big;           // sequences [0, B_big) use the segments above; the rest, handed out last, finer ones
+    int cps_f, nst_f, nsd_f;   // ... of cps_f chunks: nst_f / nsd_f segments per row
+    int pst_t, pst_d;    // partials reserved per target / drafter row (the larger of the two counts)
+    int fin_slice;       // cluster kernel: 16-byte vectors of the sampled target row per CTA
+    int fin_dvec;        // cluster kernel: 16-byte vectors reserved for the staged drafter row
 };
 
 // ---------------------------------------------------------------------------
@@ -272,9 +274,6 @@ __device__ __forceinline__ float2 ld_shared_pair(const float2 *p) {     // a pai
     asm volatile("ld.volatile.shared.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "r"(smem_addr(p)) : "memory");
     return v;
 }
-__device__ __forceinline__ void consumer_sync() {            // the consumer warps only
-    asm volatile("bar.sync 1, %0;" ::"n"(kSThreads) : "memory");
-}
 
 // ---- the schedule both the producer and the consumers walk ----
 
@@ -285,29 +284,57 @@ struct Segment {
     int seg;          // index of the segment within its row
     bool skip;        // nothing to read (bad temperature, or drafter row at temperature 0)
     float tau;
+    int m;            // drafts of the sequence that count
 };
 
+// Segments are numbered sequence-major.  The sequences from B_big on are cut into finer segments:
+// they are handed out last, when the CTAs are about to run dry, so that no CTA is left with a long
+// segment while the others have finished.
+__device__ __forceinline__ long long segment_count(const Params &P) {
+    return static_cast<long long>(P.B_big) * ((P.K + 1) * P.nst + P.K * P.nsd) +
+           static_cast<long long>(P.B - P.B_big) * ((P.K + 1) * P.nst_f + P.K * P.nsd_f);
+}
+
+// The index arithmetic of a segment, and the loads of its sequence's temperature and draft count:
+// issued here, used by finish_segment(), so that their latency passes while the producer is still
+// streaming the segment before.
 __device__ __forceinline__ Segment decode_segment(const Params &P, long long id) {
     Segment g;
     const int per_b = (P.K + 1) * P.nst + P.K * P.nsd;
-    g.b = static_cast<int>(id / per_b);
-    int item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
-    g.tau = __ldg(P.tau + g.b);
-    const bool bad = !(g.tau >= 0.f) || isinf(g.tau);
-    const int m = P.draft_len ? min(max(__ldg(P.draft_len + g.b), 0), P.K) : P.K;    // drafts of this sequence
-    int nchunk;
-    if (item < (P.K + 1) * P.nst) {
-        g.row = item / P.nst; g.seg = item - g.row * P.nst; nchunk = P.nct;
-        g.skip = bad || g.row > m;               // target rows 0..m: m drafts and the bonus position
+    const long long n_big = static_cast<long long>(P.B_big) * per_b;
+    int nst = P.nst, nsd = P.nsd, cps = P.cps;
+    int item;
+    if (id < n_big) {
+        g.b = static_cast<int>(id / per_b);
+        item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
     } else {
-        item -= (P.K + 1) * P.nst;
-        const int j = item / P.nsd;
-        g.row = P.K + 1 + j; g.seg = item - j * P.nsd; nchunk = P.ncd;
-        g.skip = bad || g.tau == 0.f || j >= m;
+        nst = P.nst_f; nsd = P.nsd_f; cps = P.cps_f;
+        const int per_f = (P.K + 1) * nst + P.K * nsd;
+        const long long id2 = id - n_big;
+        const int bf = static_cast<int>(id2 / per_f);
+        g.b = P.B_big + bf;
+        item = static_cast<int>(id2 - static_cast<long long>(bf) * per_f);
     }
-    g.chunk0 = g.seg * P.cps;
-    g.chunk1 = min(g.chunk0 + P.cps, nchunk);
+    g.tau = __ldg(P.tau + g.b);
+    g.m = P.draft_len ? __ldg(P.draft_len + g.b) : P.K;
+    int nchunk;
+    if (item < (P.K + 1) * nst) {
+        g.row = item / nst; g.seg = item - g.row * nst; nchunk = P.nct;
+    } else {
+        item -= (P.K + 1) * nst;
+        const int j = item / nsd;
+        g.row = P.K + 1 + j; g.seg = item - j * nsd; nchunk = P.ncd;
+    }
+    g.chunk0 = g.seg * cps;
+    g.chunk1 = min(g.chunk0 + cps, nchunk);
+    g.skip = false;
     return g;
+}
+__device__ __forceinline__ void finish_segment(const Params &P, Segment &g) {
+    const bool bad = !(g.tau >= 0.f) || isinf(g.tau);
+    const int m = min(max(g.m, 0), P.K);
+    if (g.row <= P.K) g.skip = bad || g.row > m;                   // target rows 0..m: m drafts and the bonus position
+    else g.skip = bad || g.tau == 0.f || g.row - P.K - 1 >= m;
 }
 
 template <int DT> __device__ __forceinline__ RowView<DT> segment_row(const Params &P, const Segment &g) {
@@ -524,7 +551,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const long long nseg_total = static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
+    const long long nseg_total = segment_count(P);
 
     if (threadIdx.x < 32) {
         // ---------------- producer ----------------
@@ -534,15 +561,22 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             bool ok = true;
             // every CTA starts on the segment of its own number (so that a small batch spreads over all
             // CTAs however unevenly they start); the rest come from the counter
-            long long next = blockIdx.x;
+            // two segments ahead: the number of the one after next is being fetched, the next one's
+            // temperature is being loaded, the current one is streamed
+            long long id = blockIdx.x;
+            Segment g = decode_segment(P, id);
+            long long id_next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);
             while (ok) {
-                const long long id = next;
                 if (id >= nseg_total) break;
-                next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);     // used one segment later
-                const Segment g = decode_segment(P, id);
-                if (g.skip) continue;                    // bad temperature, or drafter row at temperature 0
-                const RowView<DT> rv = segment_row<DT>(P, g);
-                for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk) {
+                Segment g_next = g;
+                if (id_next < nseg_total) g_next = decode_segment(P, id_next);
+                const long long id_after = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);
+                finish_segment(P, g);
+                const Segment gc = g;
+                g = g_next; id = id_next; id_next = id_after;
+                if (gc.skip) continue;                   // bad temperature, or drafter row at temperature 0
+                const RowView<DT> rv = segment_row<DT>(P, gc);
+                for (int chunk = gc.chunk0; chunk < gc.chunk1; ++chunk) {
                     ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
                     if (!ok) break;
                     int v0, v1;
@@ -550,9 +584,9 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
                     StatsMeta mt;
                     mt.chunk = chunk;
-                    mt.flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
+                    mt.flags = (chunk == gc.chunk0 ? META_FIRST : 0) | (chunk == gc.chunk1 - 1 ? META_LAST : 0) |
                                (interior ? META_INTERIOR : 0);
-                    mt.b = g.b; mt.row = g.row; mt.seg = g.seg; mt.tau = g.tau; mt.pad[0] = mt.pad[1] = 0;
+                    mt.b = gc.b; mt.row = gc.row; mt.seg = gc.seg; mt.tau = gc.tau; mt.pad[0] = mt.pad[1] = 0;
                     sm.meta[st] = mt;
                     const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
                     mbar_arrive_expect_tx(&sm.full[st], bytes);
@@ -563,6 +597,9 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     if (++st == NST) { st = 0; par ^= 1u; }
                 }
             }
+            // nothing more to start: the next kernel of the stream may be made resident as CTAs of this
+            // one leave (it still waits for all of this grid before it reads the partials)
+            asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             if (ok) {                                    // tell the consumers there is nothing more
                 if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
                     StatsMeta mt;
@@ -586,7 +623,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         // ---------------- consumers ----------------
         const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
         Segment g;
-        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f;
+        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f; g.m = 0;
         RowView<DT> rv(P.zt, 0, P.V_t);
         bool greedy = false, masked = false;
         float s = 0.f;
@@ -692,8 +729,8 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 }
                 if (lane == 0) {
                     float2 *dst = (g.row <= P.K)
-                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
-                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
+                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.pst_t + g.seg
+                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.pst_d + g.seg;
                     __stcg(dst, pr);
                 }
             }
@@ -708,46 +745,53 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
 }
 
 // ---------------------------------------------------------------------------
-// decision: one CTA per sequence
+// decision: Algorithm 5's acceptance tests and count, once per sequence
 // ---------------------------------------------------------------------------
 //
 // fp64 combination of the segment partials of every row of the sequence, Algorithm 5's
 // acceptance tests (thresholds in fp64 from two gathered logits each) and count of accepted
-// drafts, hand-over to the sampling pass.  The gathers do not depend on the statistics, so they
-// are issued first and complete while the partials are being combined.
-template <int DT>
-__global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
-    const int b = blockIdx.x;
+// drafts, and what the sampling pass needs.  The gathers do not depend on the statistics, so they
+// are issued before the wait for the statistics kernel and complete while the partials are being
+// combined.  Run by all NT threads of a CTA; every thread returns the same `sel` and `flags`.
+// `writer`: this CTA stores accepted / row_status / p_draft / q_draft (and next_token when the
+// sequence is finished here: invalid temperature, temperature 0, non-finite logits).
+// Returns true when the extra token is still to be drawn (sel.mode is MODE_RESIDUAL or
+// MODE_TARGET_ONLY).
+template <int DT, int NT>
+__device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool writer, RowSel &sel, int &flags) {
     const int tid = threadIdx.x;
     // loads that depend on nothing go out together: temperature, this thread's uniform, (below) its draft id
     const float tau = __ldg(P.tau + b);
     const float u_mine = (tid <= P.K) ? __ldg(P.u + static_cast<size_t>(b) * (P.K + 1) + tid) : 0.f;
-    __shared__ float sm_u_last;
     __shared__ float sm_c[2 * TLI_MAX_K + 1];      // reference (or max value for temperature 0)
     __shared__ double sm_s[2 * TLI_MAX_K + 1];     // sum (or arg-max index)
     __shared__ int sm_accept[TLI_MAX_K];
     __shared__ int sm_flags;
+    __shared__ RowSel sm_sel;
     const int K = P.K;
     const int Kb = P.draft_len ? min(max(__ldg(P.draft_len + b), 0), K) : K;     // drafts of this sequence that count
+    sel.n = 0; sel.mode = MODE_SKIP; sel.s = 0.f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f; sel.v = 0.f;
     if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
-        if (tid == 0) {
-            P.accepted[b] = 0; P.next_token[b] = 0;
-            if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
-            RowSel sel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-            P.sel[b] = sel;
+        flags = TLI_ROW_BAD_TEMPERATURE;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (writer) {
+            if (tid == 0) {
+                P.accepted[b] = 0; P.next_token[b] = 0;
+                if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
+            }
+            if (tid < K) {
+                if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
+                if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
+            }
         }
-        if (tid < K) {
-            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
-            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
-        }
-        return;
+        return false;
     }
     const bool greedy = (tau == 0.f);
     // the drafted token's two logits and its target id: loads in flight while the rows are combined
     int g_x = -1, g_t = -1, g_fl = 0;
     float g_zt = 0.f, g_zd = 0.f;
     if (tid < Kb) {
-        g_x = P.draft[static_cast<size_t>(b) * K + tid];
+        g_x = __ldg(P.draft + static_cast<size_t>(b) * K + tid);
         if (g_x < 0 || g_x >= P.V_d) g_fl |= TLI_ROW_DRAFT_RANGE;
         else { g_t = __ldg(P.map + g_x); if (g_t < 0) g_fl |= TLI_ROW_DRAFT_UNMAPPED; }
         if (g_t >= 0 && !greedy) {
@@ -756,26 +800,28 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         }
     }
     const int nrows = greedy ? (K + 1) : (2 * K + 1);      // rows beyond the sequence's own drafts have no partials
-    if (tid == K) sm_u_last = u_mine;
+    if (tid == K) sm_sel.v = u_mine;
+
+    // everything below reads what the statistics kernel wrote (its partials, its time-out word)
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) {
         int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
         if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
         sm_flags = fl;
     }
-
-    asm volatile("griddepcontrol.wait;" ::: "memory");
     // Eight lanes per row, one pass: every lane folds its share of the row's partials into a running
     // pair (changes of reference are exact powers of two), then the eight lanes are folded together.
     // (the loop bound is the same for all lanes of a warp: lanes beyond the last row run along with
     // zero partials, because the shuffles below need the whole warp)
-    for (int r0 = 0; r0 < nrows; r0 += kThreads / 8) {
+    for (int r0 = 0; r0 < nrows; r0 += NT / 8) {
         const int r = r0 + (tid >> 3);
         const int sub = tid & 7;
         const bool is_t = r <= K;
         const bool mine = r < nrows && (is_t ? r <= Kb : r - K - 1 < Kb);
-        const int nseg = !mine ? 0 : (is_t ? P.nst : P.nsd);
-        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
-                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
+        const bool fine = b >= P.B_big;
+        const int nseg = !mine ? 0 : (is_t ? (fine ? P.nst_f : P.nst) : (fine ? P.nsd_f : P.nsd));
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.pst_t
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.pst_d;
         if (greedy) {
             float best = -INFINITY; int idx = INT_MAX;
             for (int i = sub; i < nseg; i += 8) {
@@ -838,48 +884,69 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
         }
         sm_accept[j] = ok;
         if (fl) atomicOr(&sm_flags, fl);
-        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
-        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
-    } else if (tid < K) {
+        if (writer) {
+            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
+            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+        }
+    } else if (tid < K && writer) {
         if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
         if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
-    }
-    // the bonus row's sum must be usable too
-    if (tid == Kb && !greedy) {
-        const double S_t = sm_s[Kb];
-        if (!(S_t > 0.0) || !isfinite(S_t)) atomicOr(&sm_flags, TLI_ROW_NONFINITE);
     }
     __syncthreads();
     if (tid == 0) {
         int n = Kb;
         for (int j = 0; j < Kb; ++j) if (!sm_accept[j]) { n = j; break; }
         int fl = sm_flags;
-        RowSel sel;
-        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
-        sel.v = sm_u_last;
+        // the row the extra token is drawn from must have a usable sum too
+        if (!greedy) {
+            const double S_n = sm_s[n];
+            if (!(S_n > 0.0) || !isfinite(S_n)) fl |= TLI_ROW_NONFINITE;
+        }
+        RowSel rs;
+        rs.n = n; rs.mode = MODE_SKIP; rs.s = s_f; rs.c_t = 0.f; rs.rs_t = 0.f; rs.c_d = 0.f; rs.rs_d = 0.f;
+        rs.v = sm_sel.v;
+        int token = -1;                            // -1: the sampling pass supplies it
         if (greedy) {
-            P.next_token[b] = static_cast<int>(sm_s[n]);
+            token = static_cast<int>(sm_s[n]);
         } else if (fl & TLI_ROW_NONFINITE) {
             n = 0;
-            P.next_token[b] = 0;
+            token = 0;
         } else {
-            sel.c_t = sm_c[n];
-            sel.rs_t = static_cast<float>(1.0 / sm_s[n]);
+            rs.c_t = sm_c[n];
+            rs.rs_t = static_cast<float>(1.0 / sm_s[n]);
             if (n < Kb) {
                 const double S_d = sm_s[K + 1 + n];
-                sel.mode = MODE_RESIDUAL;
-                sel.c_d = sm_c[K + 1 + n];
-                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
+                rs.mode = MODE_RESIDUAL;
+                rs.c_d = sm_c[K + 1 + n];
+                rs.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
             } else {
-                sel.mode = MODE_TARGET_ONLY;
+                rs.mode = MODE_TARGET_ONLY;
             }
         }
-        sel.n = n;
-        P.accepted[b] = n;
-        if (P.status) P.status[b] = fl;
-        P.sel[b] = sel;
+        rs.n = n;
+        if (writer) {
+            P.accepted[b] = n;
+            if (token >= 0) P.next_token[b] = token;
+            if (P.status) P.status[b] = fl;
+        }
+        sm_sel = rs;
+        sm_flags = fl;
     }
-    }
+    __syncthreads();
+    sel = sm_sel;
+    flags = sm_flags;
+    return sel.mode != MODE_SKIP;
+}
+
+// The decision as a kernel of its own, one CTA per sequence (the form for vocabularies too large
+// for the cluster kernel below): leaves a RowSel per sequence for the tile kernel.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
+    RowSel sel;
+    int flags;
+    decide_sequence<DT, kThreads>(P, blockIdx.x, true, sel, flags);
+    if (threadIdx.x == 0) P.sel[blockIdx.x] = sel;
+}
 
 // ---------------------------------------------------------------------------
 // pass 2: the extra token
@@ -891,7 +958,20 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
 // LEAN: the caller knows that the vector lies wholly inside the row and that its first id is a
 // multiple of four (true for every vector of a tile that is not at an end of an aligned row), which
 // takes the checks and the element-wise loads out of the code.
-template <int DT, bool LEAN = false>
+// SMEM: zd_row is the shared-memory address (as ld.shared takes it) of element 0 of a staged copy of
+// the drafter row, not a global pointer.
+template <int DT> __device__ __forceinline__ float load_elt_shared(uint32_t row_addr, int i) {
+    if (DT == TLI_F32) {
+        float v;
+        asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(row_addr + static_cast<uint32_t>(i) * 4u));
+        return v;
+    }
+    unsigned short h;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(row_addr + static_cast<uint32_t>(i) * 2u));
+    return __uint_as_float(static_cast<uint32_t>(h) << 16);
+}
+
+template <int DT, bool LEAN = false, bool SMEM = false>
 __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
                                                     const void *zd_row, float (&w)[Elt<DT>::kPerVec]) {
     constexpr int EPV = Elt<DT>::kPerVec;
@@ -921,7 +1001,8 @@ __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSe
         const float et = ex2(__fmaf_rn(z[i], sel.s, nct));
         float q = 0.f;
         if (x[i] >= 0) {
-            const float zdv = load_elt<DT>(zd_row, x[i]);
+            const float zdv = SMEM ? load_elt_shared<DT>(static_cast<uint32_t>(reinterpret_cast<uintptr_t>(zd_row)), x[i])
+                                   : load_elt<DT>(zd_row, x[i]);
             q = __fmul_rn(ex2(__fmaf_rn(zdv, sel.s, ncd)), sel.rs_d);
         }
         // p and q' are each rounded before the subtraction, so that equal distributions leave exactly 0
@@ -929,11 +1010,11 @@ __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSe
     }
 }
 
-template <int DT, bool LEAN = false>
+template <int DT, bool LEAN = false, bool SMEM = false>
 __device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
                                                const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
     const uint4 raw = LEAN ? __ldg(rt.vec0 + v) : rt.load(v);
-    vector_weights_from<DT, LEAN>(P, sel, raw, rt.first_elem(v), zd_row, w);
+    vector_weights_from<DT, LEAN, SMEM>(P, sel, raw, rt.first_elem(v), zd_row, w);
 }
 
 template <int N> __device__ __forceinline__ float ordered_sum(const float (&w)[N]) {
@@ -1198,6 +1279,222 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
     const void *zd_row = reinterpret_cast<const char *>(P.zd) +
         (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
     select_sequence<DT, true>(P, b, sel, rt, zd_row);
+}
+
+// ---------------------------------------------------------------------------
+// decision and extra token in one launch: one thread-block cluster per sequence
+// ---------------------------------------------------------------------------
+//
+// The form for vocabularies whose drafter row fits one CTA's shared memory (every bf16 vocabulary
+// of today's models) and for moderate batches.  Each CTA of the cluster repeats the (cheap)
+// decision, then owns one slice of target row n:
+//   staging   one bulk copy brings drafter row n into the CTA's shared memory while the first
+//             loads of the target slice and of the inverse map are already on their way: the
+//             gather q'(inv[t]) then costs a shared-memory access instead of a second trip to L2;
+//   weights   max(0, p - q'_T) (or p) per element with vector_weights_from, one fp32 sum per
+//             16-byte vector kept in shared memory;
+//   inversion block-wide fp64 prefix over the vector sums, the CTA totals exchanged through
+//             distributed shared memory, and the CTA holding v * total walks vector -> element.
+// Two cluster barriers and two trips to memory after the statistics are in, against three kernel
+// boundaries and about ten dependent trips of the tile form.  Every CTA of a cluster takes the
+// same branches (they decide from the same data), so the barriers always meet.
+
+constexpr int kFinThreads = 512;
+constexpr int kFinWarps = kFinThreads / 32;
+constexpr int kFinMaxCluster = 8;
+
+__device__ __forceinline__ unsigned cluster_cta_rank() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ unsigned cluster_cta_count() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_barrier() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, unsigned rank) {      // the same offset in CTA `rank`
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
+    asm volatile("st.shared::cluster.f64 [%0], %1;" ::"r"(addr), "d"(v) : "memory");
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params P) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    extern __shared__ __align__(16) unsigned char fin_smem[];
+    __shared__ double sm_warp_tot[kFinWarps];
+    __shared__ double sm_cta_tot[2][kFinMaxCluster];       // one set per attempt
+    __shared__ int sm_found, sm_lastpos, sm_error;
+    __shared__ uint64_t sm_bar;
+    const int b = blockIdx.y;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned rank = cluster_cta_rank(), C = cluster_cta_count();
+    const int slice = P.fin_slice;                           // vectors of the target row per CTA
+    uint4 *drow = reinterpret_cast<uint4 *>(fin_smem);       // drafter row n on its 16-byte vector grid
+    float *vsum = reinterpret_cast<float *>(fin_smem + static_cast<size_t>(P.fin_dvec) * 16);
+
+    if (tid == 0) {
+        mbar_init(&sm_bar, 1);
+        sm_error = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    cluster_barrier();            // every CTA of the cluster is running before anybody stores into a neighbour
+
+    RowSel sel;
+    int flags;
+    if (!decide_sequence<DT, kFinThreads>(P, b, rank == 0, sel, flags)) return;
+
+    const RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const int nvec = rt.nvec();
+    const int v_begin = static_cast<int>(rank) * slice;
+    const int count = max(0, min(slice, nvec - v_begin));    // this CTA's vectors: v_begin .. v_begin + count
+    uint32_t zd_smem = 0;                                    // shared-memory address of element 0 of the staged row
+
+    if (sel.mode == MODE_RESIDUAL && count > 0) {
+        const RowView<DT> rd(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n) * P.d_sk, P.V_d);
+        int v0, v1;
+        full_vectors<DT>(rd, 0, INT_MAX / 2, v0, v1);          // the vectors wholly inside the row: [v0, v1)
+        if (tid == 0) {
+            const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
+            mbar_arrive_expect_tx(&sm_bar, bytes);
+            if (bytes) bulk_load(drow + v0, rd.vec0 + v0, bytes, &sm_bar);
+        }
+        // the at most two ragged vectors of the row, element by element
+        const int nvec_d = rd.nvec();
+        if (tid == 32 && v0 > 0) drow[0] = rd.load(0);
+        if (tid == 64 && v1 < nvec_d) drow[nvec_d - 1] = rd.load(nvec_d - 1);
+        zd_smem = smem_addr(drow) + static_cast<uint32_t>(rd.head) * Elt<DT>::kBytes;
+    }
+    // the first vectors of the slice and their inverse-map entries travel while the row is staged
+    const bool lean = (rt.head & 3) == 0 && count > 0 && rt.first_elem(v_begin) >= 0 &&
+                      rt.first_elem(v_begin + count - 1) + EPV <= rt.V;                  // the same for the whole CTA
+    if (sel.mode == MODE_RESIDUAL && count > 0) {
+        mbar_wait(&sm_bar, 0u, &sm_error, P.error);
+        __syncthreads();                                     // the ragged vectors too
+    }
+
+    const double v_target = static_cast<double>(sel.v);
+    const void *zd_arg = reinterpret_cast<const void *>(static_cast<uintptr_t>(zd_smem));
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        // ---- weights of this CTA's slice, one fp32 sum per vector ----
+        if (lean) {
+#pragma unroll 2
+            for (int i = tid; i < count; i += kFinThreads) {
+                float w[EPV];
+                vector_weights<DT, true, true>(P, sel, rt, zd_arg, v_begin + i, w);
+                vsum[i] = ordered_sum(w);
+            }
+        } else {
+            for (int i = tid; i < count; i += kFinThreads) {
+                float w[EPV];
+                vector_weights<DT, false, true>(P, sel, rt, zd_arg, v_begin + i, w);
+                vsum[i] = ordered_sum(w);
+            }
+        }
+        __syncthreads();
+        // ---- fp64 prefix: thread i owns the run of vectors [i * len, (i + 1) * len) ----
+        const int len = (slice + kFinThreads - 1) / kFinThreads;
+        const int r0 = min(tid * len, count), r1 = min(r0 + len, count);
+        double mine = 0.0;
+        for (int i = r0; i < r1; ++i) mine += static_cast<double>(vsum[i]);
+        double incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const double up = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += up;
+        }
+        if (lane == 31) sm_warp_tot[warp] = incl;
+        if (tid == 0) { sm_found = INT_MAX; sm_lastpos = -1; }
+        __syncthreads();
+        double base = 0.0, cta_total = 0.0;
+#pragma unroll
+        for (int i = 0; i < kFinWarps; ++i) {
+            if (i == warp) base = cta_total;
+            cta_total += sm_warp_tot[i];
+        }
+        if (tid < static_cast<int>(C))                       // this CTA's total to every CTA of the cluster
+            st_cluster_f64(cluster_addr(smem_addr(&sm_cta_tot[attempt][rank]), static_cast<unsigned>(tid)), cta_total);
+        cluster_barrier();
+        // ---- which CTA holds v * R (the same arithmetic in every CTA) ----
+        double R = 0.0;
+        for (unsigned r = 0; r < C; ++r) R += sm_cta_tot[attempt][r];
+        if (!(R > 0.0) || !isfinite(R)) {
+            if (attempt == 1 || sel.mode == MODE_TARGET_ONLY) {          // no usable mass even from p: give up on the row
+                if (rank == 0 && tid == 0) {
+                    P.next_token[b] = 0;
+                    if (P.status) P.status[b] = flags | TLI_ROW_NONFINITE;
+                }
+                return;
+            }
+            // zero residual mass: sample from p of the same position instead
+            sel.mode = MODE_TARGET_ONLY;
+            flags |= TLI_ROW_FALLBACK;
+            if (rank == 0 && tid == 0 && P.status) P.status[b] = flags;
+            continue;
+        }
+        const double target = v_target * R;
+        int owner = -1, lastpos_cta = 0;
+        double before = 0.0, run_c = 0.0;
+        for (unsigned r = 0; r < C; ++r) {
+            const double tr = sm_cta_tot[attempt][r];
+            const double nx = run_c + tr;
+            if (tr > 0.0) lastpos_cta = static_cast<int>(r);
+            if (owner < 0 && nx > target) { owner = static_cast<int>(r); before = run_c; }
+            run_c = nx;
+        }
+        if (owner < 0) { owner = lastpos_cta; before = R - sm_cta_tot[attempt][lastpos_cta]; }
+        if (static_cast<int>(rank) != owner) return;
+        // ---- this CTA: vector, then element ----
+        if (sm_error && tid == 0 && P.status) P.status[b] = flags | TLI_ROW_TIMEOUT;      // the staging wait ran out
+        const double rem = target - before;
+        double run = base + incl - mine;                 // mass before this thread's first vector
+        int cand = INT_MAX, lastpos = -1;
+        double cand_before = 0.0;
+        for (int i = r0; i < r1; ++i) {
+            const double wv = static_cast<double>(vsum[i]);
+            const double nx = run + wv;
+            if (wv > 0.0) lastpos = i;
+            if (cand == INT_MAX && nx > rem) { cand = i; cand_before = run; }
+            run = nx;
+        }
+        if (cand != INT_MAX) atomicMin(&sm_found, cand);
+        if (lastpos >= 0) atomicMax(&sm_lastpos, lastpos);
+        __syncthreads();
+        const int found = sm_found;
+        const int G = (found != INT_MAX) ? found : sm_lastpos;
+        if (G < 0) {                                     // cannot happen when the slice has positive mass
+            if (tid == 0) P.next_token[b] = 0;
+            return;
+        }
+        if ((found != INT_MAX) ? (cand == found) : (tid == 0)) {
+            // walk the elements of vector G with the same running fp32 sum that formed its total;
+            // when rounding left no vector above the target, take the last positive element instead
+            const double rem2 = (found != INT_MAX) ? (rem - cand_before) : INFINITY;
+            float w[EPV];
+            if (lean) vector_weights<DT, true, true>(P, sel, rt, zd_arg, v_begin + G, w);
+            else vector_weights<DT, false, true>(P, sel, rt, zd_arg, v_begin + G, w);
+            float runf = 0.f;
+            int pick = -1, lastw = 0;
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) {
+                runf = (i == 0) ? w[0] : __fadd_rn(runf, w[i]);
+                if (w[i] > 0.f) lastw = i;
+                if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
+            }
+            if (pick < 0) pick = lastw;
+            int token = rt.first_elem(v_begin + G) + pick;
+            token = min(max(token, 0), P.V_t - 1);
+            P.next_token[b] = token;
+        }
+        return;
+    }
 }
 
 // ---------------------------------------------------------------------------
@@ -1969,670 +2266,6 @@ __global__ void __launch_bounds__(kThreads, 6) tli_rate_pairs_kernel(const RateP
     if (P.status) P.status[pair] = status;
 }
 
-// ---------------------------------------------------------------------------
-// the fused kernel: statistics, decisions and sampling in one persistent grid
-// ---------------------------------------------------------------------------
-//
-// The statistics kernel's machinery with two additions.  (1) Once a sequence is decided, the
-// segments of the one target row its extra token is drawn from become work items of the same
-// ring: a producer takes them (in sequence order, by compare-and-swap on one counter, as soon as
-// the sequence is marked decided) ahead of further statistics segments, so the row is still in L2.
-// Consumers turn such a chunk into weights and store one sum per warp-sized strip, in target-id
-// order.  (2) The two short serial jobs per sequence -- the decision when its last statistic
-// arrives, the CDF inversion when its last strip sum arrives -- go to a seventeenth "epilogue"
-// warp through a mailbox in shared memory, so the streaming warps never stop for them.
-// Nothing waits without bound: producers that run out of work poll for the last decisions with a
-// limit, consumers and the epilogue warp wait only on their own CTA.
-
-enum : int { META_SAMPLE = 32 };
-enum : int { SEQ_PENDING = 0, SEQ_SAMPLE = 1, SEQ_NO_SAMPLE = 2 };
-constexpr int kMailbox = 32;
-constexpr unsigned kIdleLimit = 1u << 20;
-
-struct FusedSmem {
-    uint64_t full[kMaxStages];
-    uint64_t empty[kMaxStages];
-    StageMeta meta[kMaxStages];
-    RowSel sel[kMaxStages];            // with META_SAMPLE | META_FIRST: the sequence's RowSel
-    float2 pairs[2][kSWarps];
-    int error;
-    // consumers -> epilogue warp: entry = (sequence << 1) | job, job 0 = decide, 1 = invert the CDF
-    int mail[kMailbox];
-    unsigned mail_tail, mail_head;
-    int consumers_done;
-    float ep_c[2 * TLI_MAX_K + 1];     // epilogue warp: reference (or max value) per row
-    double ep_s[2 * TLI_MAX_K + 1];    //                sum (or arg-max index) per row
-};
-
-constexpr int kFusedSmemBytes = kRingBytes + static_cast<int>(sizeof(FusedSmem));
-constexpr int kFThreads = kSThreads + 64;          // producer warp + consumers + epilogue warp
-
-__device__ __forceinline__ int ld_volatile(const int *p) { return *reinterpret_cast<const volatile int *>(p); }
-__device__ __forceinline__ unsigned ld_volatile(const unsigned *p) { return *reinterpret_cast<const volatile unsigned *>(p); }
-__device__ __forceinline__ void st_volatile(int *p, int v) { *reinterpret_cast<volatile int *>(p) = v; }
-
-// Hand a job to the epilogue warp (called by one consumer thread only).
-__device__ __forceinline__ void mail_push(FusedSmem &sm, int entry, unsigned *g_error) {
-    volatile unsigned *head = &sm.mail_head;
-    volatile unsigned *tail = &sm.mail_tail;
-    unsigned t = *tail;
-    for (unsigned i = 0; t - *head >= kMailbox; ++i) {          // full: the epilogue warp is behind
-        if (i > kIdleLimit) { atomicOr(g_error, 4u); return; }
-        __nanosleep(128);
-    }
-    reinterpret_cast<volatile int *>(sm.mail)[t % kMailbox] = entry;
-    __threadfence_block();
-    *tail = t + 1;
-}
-
-// A RowSel written by another CTA, read past L1.
-__device__ __forceinline__ RowSel load_sel(const RowSel *p) {
-    const uint4 a = __ldcg(reinterpret_cast<const uint4 *>(p));
-    const uint4 b = __ldcg(reinterpret_cast<const uint4 *>(p) + 1);
-    RowSel r;
-    r.n = static_cast<int>(a.x); r.mode = static_cast<int>(a.y);
-    r.s = __uint_as_float(a.z); r.c_t = __uint_as_float(a.w);
-    r.rs_t = __uint_as_float(b.x); r.c_d = __uint_as_float(b.y);
-    r.rs_d = __uint_as_float(b.z); r.v = __uint_as_float(b.w);
-    return r;
-}
-
-// The decision for one sequence by one warp: lanes over rows, then lanes over drafts.
-template <int DT>
-__device__ void warp_decide(const Params &P, FusedSmem &sm, int b, int lane) {
-    const int K = P.K;
-    const float tau = __ldg(P.tau + b);
-    const bool greedy = (tau == 0.f);
-    const float s_f = 1.4426950408889634f / tau;
-    // loads that depend on nothing first: uniforms, draft ids -> map -> the two logits
-    float u_j[2]; int g_t[2]; int g_fl[2]; float g_zt[2], g_zd[2];
-    const float u_last = __ldg(P.u + static_cast<size_t>(b) * (K + 1) + K);
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const int j = lane + 32 * r;
-        u_j[r] = 0.f; g_t[r] = -1; g_fl[r] = 0; g_zt[r] = 0.f; g_zd[r] = 0.f;
-        if (j < K) {
-            u_j[r] = __ldg(P.u + static_cast<size_t>(b) * (K + 1) + j);
-            const int x = P.draft[static_cast<size_t>(b) * K + j];
-            if (x < 0 || x >= P.V_d) g_fl[r] = TLI_ROW_DRAFT_RANGE;
-            else { g_t[r] = __ldg(P.map + x); if (g_t[r] < 0) g_fl[r] = TLI_ROW_DRAFT_UNMAPPED; }
-            if (g_t[r] >= 0 && !greedy) {
-                g_zt[r] = load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(j) * P.t_sk + g_t[r]);
-                g_zd[r] = load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(j) * P.d_sk + x);
-            }
-        }
-    }
-    // every row's partials into one (reference, sum) or (max, index), a row per lane
-    const int nrows = greedy ? (K + 1) : (2 * K + 1);
-    for (int r = lane; r < nrows; r += 32) {
-        const bool is_t = r <= K;
-        const int nseg = is_t ? P.nst : P.nsd;
-        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
-                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
-        if (greedy) {
-            float best = -INFINITY; int idx = INT_MAX;
-            for (int i = 0; i < nseg; ++i) {
-                const float2 pr = __ldcg(part + i);
-                const int i2 = __float_as_int(pr.y);
-                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
-            }
-            sm.ep_c[r] = best; sm.ep_s[r] = (idx == INT_MAX) ? 0.0 : static_cast<double>(idx);
-        } else {
-            float c = kNegBig;
-            for (int i = 0; i < nseg; ++i) c = fmaxf(c, __ldcg(part + i).x);
-            double sum = 0.0;
-            for (int i = 0; i < nseg; ++i) {
-                const float2 pr = __ldcg(part + i);
-                sum += static_cast<double>(pr.y) * pow2_neg_d(pr.x - c);
-            }
-            sm.ep_c[r] = c; sm.ep_s[r] = sum;
-        }
-    }
-    __syncwarp();
-    int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
-    if (ld_volatile(P.error)) fl |= TLI_ROW_TIMEOUT;
-    int n = K;
-#pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const int j = lane + 32 * r;
-        int ok = 1;                       // lanes beyond K do not reject
-        float pv = 0.f, qv = 0.f;
-        if (j < K) {
-            ok = 0;
-            fl |= g_fl[r];
-            const int t = g_t[r];
-            if (greedy) {
-                ok = (t >= 0 && t == static_cast<int>(sm.ep_s[j]));
-            } else {
-                const double S_t = sm.ep_s[j], S_d = sm.ep_s[K + 1 + j];
-                if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
-                else if (t >= 0) {
-                    const double sd = static_cast<double>(s_f);
-                    const double p = exp2(static_cast<double>(g_zt[r]) * sd - static_cast<double>(sm.ep_c[j])) / S_t;
-                    const double q = (S_d > 0.0) ? exp2(static_cast<double>(g_zd[r]) * sd - static_cast<double>(sm.ep_c[K + 1 + j])) / S_d : 0.0;
-                    double thr;
-                    if (q > 0.0) thr = fmin(1.0, p / q);
-                    else thr = (p > 0.0) ? 1.0 : 0.0;
-                    ok = static_cast<double>(u_j[r]) < thr;
-                    pv = static_cast<float>(p); qv = static_cast<float>(q);
-                }
-            }
-            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
-            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
-        }
-        const unsigned rejected = __ballot_sync(0xffffffffu, !ok);
-        if (rejected && n == K) n = 32 * r + (__ffs(rejected) - 1);
-    }
-    if (!greedy) {                        // the bonus row's sum must be usable too
-        const double S_k = sm.ep_s[K];
-        if (!(S_k > 0.0) || !isfinite(S_k)) fl |= TLI_ROW_NONFINITE;
-    }
-    fl = __reduce_or_sync(0xffffffffu, fl);
-    if (lane == 0) {
-        RowSel sel;
-        sel.n = n; sel.mode = MODE_SKIP; sel.s = s_f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f;
-        sel.v = u_last;
-        if (greedy) {
-            P.next_token[b] = static_cast<int>(sm.ep_s[n]);
-        } else if (fl & TLI_ROW_NONFINITE) {
-            n = 0;
-            P.next_token[b] = 0;
-        } else {
-            sel.c_t = sm.ep_c[n];
-            sel.rs_t = static_cast<float>(1.0 / sm.ep_s[n]);
-            if (n < K) {
-                const double S_d = sm.ep_s[K + 1 + n];
-                sel.mode = MODE_RESIDUAL;
-                sel.c_d = sm.ep_c[K + 1 + n];
-                sel.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
-            } else {
-                sel.mode = MODE_TARGET_ONLY;
-            }
-        }
-        sel.n = n;
-        P.accepted[b] = n;
-        if (P.status) P.status[b] = fl;
-        P.sel[b] = sel;
-        __threadfence();                  // the RowSel before the mark that lets producers take the sequence
-        st_volatile(P.seq_state + b, sel.mode == MODE_SKIP ? SEQ_NO_SAMPLE : SEQ_SAMPLE);
-    }
-    __syncwarp();
-}
-
-// Strip (chunk, warp) of the sampled row: vectors chunk*CVEC + warp*32*CV + q*32 + lane, q < CV.
-// Sum of one lane's CV vectors of the strip, the vectors' own sums in vs[].
-template <int DT, int CV>
-__device__ __forceinline__ double strip_lane_sum(const Params &P, const RowSel &sel, const RowView<DT> &rt,
-                                                 const void *zd_row, int chunk, int w, int lane, float (&vs)[CV]) {
-    constexpr int EPV = Elt<DT>::kPerVec;
-    const int nvec = rt.nvec();
-    double acc = 0.0;
-#pragma unroll
-    for (int q = 0; q < CV; ++q) {
-        const int v = chunk * (kSThreads * CV) + w * (32 * CV) + q * 32 + lane;
-        vs[q] = 0.f;
-        if (v < nvec) {
-            float wt[EPV];
-            vector_weights<DT>(P, sel, rt, zd_row, v, wt);
-            vs[q] = ordered_sum(wt);
-        }
-        acc += static_cast<double>(vs[q]);
-    }
-    return acc;
-}
-
-// CDF inversion for one sequence by one warp: strip sums -> strip -> vector -> element.
-template <int DT, int CV>
-__device__ void warp_select(const Params &P, int b, int lane) {
-    constexpr int EPV = Elt<DT>::kPerVec;
-    RowSel sel = load_sel(P.sel + b);
-    const int ntot = P.nct * kSWarps;
-    double *base = P.stripsum + static_cast<size_t>(b) * ntot;
-    RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
-    const void *zd_row = reinterpret_cast<const char *>(P.zd) +
-        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n < P.K ? sel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
-    const int per = (ntot + 31) / 32;
-    const int i0 = min(lane * per, ntot), i1 = min(i0 + per, ntot);
-    int token = 0;
-    bool done = false;
-    for (int attempt = 0; attempt < 2 && !done; ++attempt) {
-        double mine = 0.0;
-        for (int i = i0; i < i1; ++i) mine += __ldcg(base + i);
-        double incl = mine;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const double up = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += up;
-        }
-        const double R = __shfl_sync(0xffffffffu, incl, 31);
-        if (!(R > 0.0) || !isfinite(R)) {
-            if (attempt == 1) {                    // no usable mass even from p: give up on the row
-                if (lane == 0 && P.status) P.status[b] |= TLI_ROW_NONFINITE;
-                token = 0; done = true;
-                break;
-            }
-            // zero residual mass: sample from p of the same position instead
-            sel.mode = MODE_TARGET_ONLY;
-            if (lane == 0 && P.status) P.status[b] |= TLI_ROW_FALLBACK;
-            for (int e = 0; e < ntot; ++e) {
-                float vs[CV];
-                const double t2 = warp_sum(strip_lane_sum<DT, CV>(P, sel, rt, zd_row, e / kSWarps, e % kSWarps, lane, vs));
-                if (lane == 0) base[e] = t2;
-            }
-            __threadfence();
-            __syncwarp();
-            continue;
-        }
-        const double target = static_cast<double>(sel.v) * R;
-        // the lane whose block holds the target, else the last lane with any mass
-        const unsigned over = __ballot_sync(0xffffffffu, incl > target);
-        const unsigned some = __ballot_sync(0xffffffffu, mine > 0.0);
-        const bool clamped = (over == 0u);
-        const int L = clamped ? (31 - __clz(some)) : (__ffs(over) - 1);
-        const double before_L = __shfl_sync(0xffffffffu, incl - mine, L);
-        int found = -1;
-        double rem = 0.0;
-        if (lane == L) {
-            const double want = clamped ? INFINITY : (target - before_L);
-            double run = 0.0;
-            int lastpos = i0;
-            for (int i = i0; i < i1; ++i) {
-                const double x = __ldcg(base + i);
-                if (x > 0.0) lastpos = i;
-                if (found < 0 && run + x > want) { found = i; rem = want - run; }
-                run += x;
-            }
-            if (found < 0) { found = lastpos; rem = INFINITY; }
-        }
-        found = __shfl_sync(0xffffffffu, found, L);
-        rem = __shfl_sync(0xffffffffu, rem, L);
-        // the strip's vectors again, in order: q-major, then lane
-        const int chunk = found / kSWarps, w = found % kSWarps;
-        float vs[CV];
-        strip_lane_sum<DT, CV>(P, sel, rt, zd_row, chunk, w, lane, vs);
-        double run = 0.0;
-        int pick_q = -1, pick_lane = -1;
-        double pick_before = 0.0;
-        int last_q = -1, last_lane = -1;
-#pragma unroll
-        for (int q = 0; q < CV; ++q) {
-            const double x = static_cast<double>(vs[q]);
-            double inc = x;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const double up = __shfl_up_sync(0xffffffffu, inc, o);
-                if (lane >= o) inc += up;
-            }
-            const unsigned ov = __ballot_sync(0xffffffffu, run + inc > rem);
-            const unsigned pos = __ballot_sync(0xffffffffu, x > 0.0);
-            if (pos) { last_q = q; last_lane = 31 - __clz(pos); }
-            if (pick_q < 0 && ov) {
-                pick_q = q; pick_lane = __ffs(ov) - 1;
-                pick_before = run + __shfl_sync(0xffffffffu, inc - x, pick_lane);
-            }
-            run += __shfl_sync(0xffffffffu, inc, 31);
-        }
-        double rem2 = rem - pick_before;
-        if (pick_q < 0) { pick_q = last_q; pick_lane = last_lane; rem2 = INFINITY; }
-        if (pick_q < 0) { token = 0; done = true; break; }       // cannot happen when the strip has mass
-        if (lane == pick_lane) {
-            // walk the elements of that vector with the same running fp32 sum that formed its total
-            const int v = chunk * (kSThreads * CV) + w * (32 * CV) + pick_q * 32 + lane;
-            float wt[EPV];
-            vector_weights<DT>(P, sel, rt, zd_row, v, wt);
-            float runf = 0.f;
-            int pick = -1, lastw = 0;
-#pragma unroll
-            for (int i = 0; i < EPV; ++i) {
-                runf = (i == 0) ? wt[0] : __fadd_rn(runf, wt[i]);
-                if (wt[i] > 0.f) lastw = i;
-                if (pick < 0 && static_cast<double>(runf) > rem2) pick = i;
-            }
-            if (pick < 0) pick = lastw;
-            token = min(max(rt.first_elem(v) + pick, 0), P.V_t - 1);
-        }
-        token = __shfl_sync(0xffffffffu, token, pick_lane);
-        done = true;
-    }
-    if (lane == 0) {
-        P.next_token[b] = token;
-        st_volatile(P.seq_state + b, SEQ_PENDING);       // ready for the next call
-    }
-    __syncwarp();
-}
-
-template <int DT, int CV>
-__global__ void __launch_bounds__(kFThreads, kCtasPerSm) tli_fused_kernel(const Params P) {
-    constexpr int CVEC = kSThreads * CV;                       // vectors per chunk
-    constexpr int NST = kRingBytes / (CVEC * 16);              // stages
-    constexpr int EPV = Elt<DT>::kPerVec;
-    static_assert(NST >= 2 && NST <= kMaxStages, "stage count");
-    extern __shared__ __align__(128) unsigned char smem_raw[];
-    uint4 *stage_base = reinterpret_cast<uint4 *>(smem_raw);
-    FusedSmem &sm = *reinterpret_cast<FusedSmem *>(smem_raw + kRingBytes);
-    if (threadIdx.x == 0) {
-#pragma unroll
-        for (int i = 0; i < NST; ++i) { mbar_init(&sm.full[i], 1); mbar_init(&sm.empty[i], kSWarps); }
-        sm.error = 0; sm.mail_tail = 0; sm.mail_head = 0; sm.consumers_done = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    const long long nseg_total = static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
-    const long long nsamp_total = static_cast<long long>(P.B) * P.nst;
-
-    if (threadIdx.x < 32) {
-        // ---------------- producer ----------------
-        if (threadIdx.x == 0) {
-            unsigned st = 0, par = 1;                     // stage and the parity of its "empty" phase to wait for
-            unsigned issued = 0, idle = 0;
-            bool ok = true;
-            long long next = blockIdx.x;                  // own number first, then from the counter
-            while (ok) {
-                // sampling items first: their rows are still in L2
-                const long long k = ld_volatile(P.samp_counter);
-                if (k < nsamp_total) {
-                    const int b = static_cast<int>(k / P.nst);
-                    const int state = ld_volatile(P.seq_state + b);
-                    if (state != SEQ_PENDING) {
-                        if (atomicCAS(P.samp_counter, static_cast<unsigned>(k), static_cast<unsigned>(k) + 1u) == static_cast<unsigned>(k)) {
-                            idle = 0;
-                            const int seg = static_cast<int>(k - static_cast<long long>(b) * P.nst);
-                            if (state == SEQ_NO_SAMPLE) {
-                                if (seg == P.nst - 1) st_volatile(P.seq_state + b, SEQ_PENDING);   // last item: ready for the next call
-                            } else {
-                                __threadfence();
-                                const RowSel sel = load_sel(P.sel + b);
-                                const RowView<DT> rv(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
-                                const int c0 = seg * P.cps, c1 = min(c0 + P.cps, P.nct);
-                                for (int chunk = c0; chunk < c1; ++chunk) {
-                                    ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
-                                    if (!ok) break;
-                                    int v0, v1;
-                                    full_vectors<DT>(rv, chunk, CVEC, v0, v1);
-                                    const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
-                                    sm.meta[st].id = k; sm.meta[st].chunk = chunk;
-                                    sm.meta[st].flags = META_SAMPLE | (chunk == c0 ? META_FIRST : 0) | (chunk == c1 - 1 ? META_LAST : 0) |
-                                                        (interior ? META_INTERIOR : 0);
-                                    if (chunk == c0) sm.sel[st] = sel;
-                                    const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
-                                    mbar_arrive_expect_tx(&sm.full[st], bytes);
-                                    if (bytes)
-                                        bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
-                                                  rv.vec0 + v0, bytes, &sm.full[st]);
-                                    ++issued;
-                                    if (++st == NST) { st = 0; par ^= 1u; }
-                                }
-                            }
-                        }
-                        continue;
-                    }
-                }
-                if (next < nseg_total) {
-                    idle = 0;
-                    const long long id = next;
-                    next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);     // used one segment later
-                    const Segment g = decode_segment(P, id);
-                    if (g.skip) {                            // bad temperature, or drafter row at temperature 0
-                        // a sequence with a bad temperature has no statistics: it is answered here, once
-                        if (g.row == 0 && g.seg == 0) {
-                            P.accepted[g.b] = 0; P.next_token[g.b] = 0;
-                            if (P.status) P.status[g.b] = TLI_ROW_BAD_TEMPERATURE;
-                            for (int j = 0; j < P.K; ++j) {
-                                if (P.p_out) P.p_out[static_cast<size_t>(g.b) * P.K + j] = 0.f;
-                                if (P.q_out) P.q_out[static_cast<size_t>(g.b) * P.K + j] = 0.f;
-                            }
-                            __threadfence();
-                            st_volatile(P.seq_state + g.b, SEQ_NO_SAMPLE);
-                        }
-                        continue;
-                    }
-                    const RowView<DT> rv = segment_row<DT>(P, g);
-                    for (int chunk = g.chunk0; chunk < g.chunk1; ++chunk) {
-                        ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
-                        if (!ok) break;
-                        int v0, v1;
-                        full_vectors<DT>(rv, chunk, CVEC, v0, v1);
-                        const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
-                        sm.meta[st].id = id; sm.meta[st].chunk = chunk;
-                        sm.meta[st].flags = (chunk == g.chunk0 ? META_FIRST : 0) | (chunk == g.chunk1 - 1 ? META_LAST : 0) |
-                                            (interior ? META_INTERIOR : 0);
-                        const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
-                        mbar_arrive_expect_tx(&sm.full[st], bytes);
-                        if (bytes)
-                            bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
-                                      rv.vec0 + v0, bytes, &sm.full[st]);
-                        ++issued;
-                        if (++st == NST) { st = 0; par ^= 1u; }
-                    }
-                    continue;
-                }
-                if (k >= nsamp_total) break;                 // all work handed out
-                // every statistic is handed out; the last sequences are still being decided
-                if (++idle > kIdleLimit) { sm.error = 1; atomicOr(P.error, 8u); ok = false; break; }
-                __nanosleep(256);
-            }
-            if (ok) {                                    // tell the consumers there is nothing more
-                if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
-                    sm.meta[st].id = -1; sm.meta[st].chunk = 0; sm.meta[st].flags = META_END;
-                    mbar_arrive(&sm.full[st]);
-                }
-            }
-            // After a timeout nobody may be waiting for the copies still in flight: let them land
-            // (bounded) before this CTA's shared memory goes away.
-            if (*reinterpret_cast<volatile int *>(&sm.error)) {
-                const unsigned n = issued < static_cast<unsigned>(NST) ? issued : static_cast<unsigned>(NST);
-                for (unsigned j = 0; j < n; ++j) {
-                    const unsigned sidx = (st + NST - 1 - j) % NST;           // the last n stages issued
-                    const unsigned use = (issued - 1 - j) / NST;               // how often that stage had been used before
-                    for (unsigned i = 0; i < kWaitLimit && !mbar_test(&sm.full[sidx], use & 1u); ++i) __nanosleep(64);
-                }
-            }
-        }
-    } else if (threadIdx.x >= 32 + kSThreads) {
-        // ---------------- epilogue warp ----------------
-        const int lane = threadIdx.x & 31;
-        unsigned head = 0;
-        for (unsigned spins = 0;;) {
-            const unsigned tail = *reinterpret_cast<volatile unsigned *>(&sm.mail_tail);
-            if (head == tail) {
-                if (*reinterpret_cast<volatile int *>(&sm.consumers_done) &&
-                    head == *reinterpret_cast<volatile unsigned *>(&sm.mail_tail)) break;
-                if (++spins > (1u << 24)) { if (lane == 0) atomicOr(P.error, 16u); break; }
-                __nanosleep(200);
-                continue;
-            }
-            spins = 0;
-            const int entry = reinterpret_cast<volatile int *>(sm.mail)[head % kMailbox];
-            ++head;
-            __syncwarp();
-            if (lane == 0) *reinterpret_cast<volatile unsigned *>(&sm.mail_head) = head;
-            __threadfence();
-            if (entry & 1) warp_select<DT, CV>(P, entry >> 1, lane);
-            else warp_decide<DT>(P, sm, entry >> 1, lane);
-        }
-    } else {
-        // ---------------- consumers ----------------
-        const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
-        Segment g;
-        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f;
-        RowView<DT> rv(P.zt, 0, P.V_t);
-        bool greedy = false, masked = false;
-        float s = 0.f;
-        float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
-        float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
-        RowSel ssel = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};   // sampling items
-        const void *zd_row = P.zd;
-        int sb = 0;
-        bool clean_exit = false;
-        unsigned seg_parity = 0;
-        unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
-        for (;;) {
-            if (!mbar_wait(&sm.full[st], par, &sm.error, P.error)) break;
-            const StageMeta meta = sm.meta[st];
-            const uint4 *stage = stage_base + static_cast<size_t>(st) * CVEC;
-            uint64_t *empty_bar = &sm.empty[st];
-            const unsigned st_now = st;
-            if (++st == NST) { st = 0; par ^= 1u; }
-            if (meta.flags & META_END) { clean_exit = true; break; }
-            const int chunk = meta.chunk;
-
-            if (meta.flags & META_SAMPLE) {
-                // ---- a chunk of the row the extra token is drawn from: weights, one sum per warp strip ----
-                if (meta.flags & META_FIRST) {
-                    sb = static_cast<int>(meta.id / P.nst);
-                    ssel = sm.sel[st_now];
-                    rv = RowView<DT>(P.zt, static_cast<long long>(sb) * P.t_sb + static_cast<long long>(ssel.n) * P.t_sk, P.V_t);
-                    zd_row = reinterpret_cast<const char *>(P.zd) +
-                        (static_cast<long long>(sb) * P.d_sb + static_cast<long long>(ssel.n < P.K ? ssel.n : 0) * P.d_sk) * Elt<DT>::kBytes;
-                }
-                uint4 raw[CV];
-                int vidx[CV];
-                {
-                    int v0 = 0, v1 = 0;
-                    const bool interior = (meta.flags & META_INTERIOR) != 0;
-                    if (!interior) full_vectors<DT>(rv, chunk, CVEC, v0, v1);
-                    const int nvec = rv.nvec();
-#pragma unroll
-                    for (int q = 0; q < CV; ++q) {
-                        const int g_in = warp * (32 * CV) + q * 32 + lane;        // strips are contiguous in target-id order
-                        const int v = chunk * CVEC + g_in;
-                        vidx[q] = v;
-                        if (interior || (v >= v0 && v < v1)) raw[q] = stage[g_in];
-                        else if (v < nvec) raw[q] = rv.load(v);
-                        else { raw[q] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord); vidx[q] = -1; }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) mbar_arrive(empty_bar);
-                double wsum = 0.0;
-#pragma unroll
-                for (int q = 0; q < CV; ++q) {
-                    float vsum = 0.f;
-                    if (vidx[q] >= 0) {
-                        float wt[EPV];
-                        vector_weights_from<DT>(P, ssel, raw[q], rv.first_elem(vidx[q]), zd_row, wt);
-                        vsum = ordered_sum(wt);
-                    }
-                    wsum += static_cast<double>(vsum);
-                }
-                wsum = warp_sum(wsum);
-                if (lane == 0) __stcg(P.stripsum + (static_cast<size_t>(sb) * P.nct + chunk) * kSWarps + warp, wsum);
-                if (!(meta.flags & META_LAST)) continue;
-                if (lane == 0) __threadfence();
-                consumer_sync();
-                if (tid == 0) {
-                    if (atomicAdd(P.cnt_sample + sb, 1u) == static_cast<unsigned>(P.nst) - 1u) {
-                        P.cnt_sample[sb] = 0;
-                        mail_push(sm, (sb << 1) | 1, P.error);
-                    }
-                }
-                continue;
-            }
-
-            if (meta.flags & META_FIRST) {
-                g = decode_segment(P, meta.id);
-                rv = segment_row<DT>(P, g);
-                greedy = (g.tau == 0.f);
-                masked = g.row > P.K;
-                s = 1.4426950408889634f / g.tau;
-                c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
-            }
-            uint4 raw[CV];
-            load_chunk<DT, CV>(rv, chunk, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_bar);                            // stage may be refilled now
-            if (greedy) {
-                argmax_chunk<DT, CV>(raw, rv, chunk, tid, best, best_idx);
-            } else if (masked) {
-                uint32_t bits[CV];
-                const int nvec = rv.nvec();
-#pragma unroll
-                for (int q = 0; q < CV; ++q) {
-                    const int v = chunk * CVEC + q * kSThreads + tid;
-                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
-                }
-                if constexpr (DT == TLI_BF16) {               // mask the packed words, then as a target row
-#pragma unroll
-                    for (int q = 0; q < CV; ++q) mask_bf16_vector(raw[q], bits[q]);
-                    softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
-                } else {
-                    softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
-                }
-            } else {
-                const uint32_t bits[CV] = {};
-                softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
-            }
-            if (!(meta.flags & META_LAST)) continue;
-
-            // ---- segment done: one (reference, sum) or (max, index) pair per warp, then per CTA ----
-            float px, py;
-            if (greedy) {
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) {
-                    float b2 = __shfl_xor_sync(0xffffffffu, best, o);
-                    int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
-                    if (b2 > best || (b2 == best && i2 < best_idx)) { best = b2; best_idx = i2; }
-                }
-                px = best; py = __int_as_float(best_idx);
-            } else {
-                const float c_w = warp_max(c_run);
-                float a_w = acc * pow2_neg(c_run - c_w);
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) a_w += __shfl_xor_sync(0xffffffffu, a_w, o);
-                px = c_w; py = a_w;
-            }
-            float2 *pairs = sm.pairs[seg_parity];
-            seg_parity ^= 1u;
-            if (lane == 0) pairs[warp] = make_float2(px, py);
-            consumer_sync();
-            if (warp == 0) {
-                float2 pr;
-                if (greedy) {
-                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(-INFINITY, __int_as_float(INT_MAX));
-                    float bb = pr.x; int ii = __float_as_int(pr.y);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) {
-                        float b2 = __shfl_xor_sync(0xffffffffu, bb, o);
-                        int i2 = __shfl_xor_sync(0xffffffffu, ii, o);
-                        if (b2 > bb || (b2 == bb && i2 < ii)) { bb = b2; ii = i2; }
-                    }
-                    pr = make_float2(bb, __int_as_float(ii));
-                } else {
-                    pr = (lane < kSWarps) ? pairs[lane] : make_float2(kNegBig, 0.f);
-                    const float c_all = warp_max(pr.x);
-                    float a_all = pr.y * pow2_neg(pr.x - c_all);
-#pragma unroll
-                    for (int o = 16; o > 0; o >>= 1) a_all += __shfl_xor_sync(0xffffffffu, a_all, o);
-                    pr = make_float2(c_all, a_all);
-                }
-                if (lane == 0) {
-                    float2 *dst = (g.row <= P.K)
-                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
-                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
-                    __stcg(dst, pr);
-                    // the last partial of a sequence: its decision goes to the epilogue warp
-                    __threadfence();
-                    const unsigned total = greedy ? (P.K + 1) * P.nst : (P.K + 1) * P.nst + P.K * P.nsd;
-                    if (atomicAdd(P.cnt_stats + g.b, 1u) == total - 1u) {
-                        P.cnt_stats[g.b] = 0;
-                        mail_push(sm, g.b << 1, P.error);
-                    }
-                }
-            }
-        }
-        if (tid == 0) {
-            __threadfence_block();
-            *reinterpret_cast<volatile int *>(&sm.consumers_done) = 1;
-            // the last CTA to leave puts the schedulers' counters back for the next call
-            if (clean_exit) {
-                __threadfence();
-                const unsigned t = atomicAdd(P.cta_done, 1u);
-                if (t == gridDim.x - 1) { *P.seg_counter = 0u; *P.samp_counter = 0u; *P.cta_done = 0u; __threadfence(); }
-            }
-        }
-    }
-}
-
 // Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete,
 // with a caller-chosen poll limit, and reports how the wait ended.  The kernel returns normally.
 __global__ void tli_bounded_wait_kernel(unsigned limit, int *result, unsigned *scratch_error) {
@@ -2667,11 +2300,46 @@ int chunks_per_row(int V, int dtype, int vec_per_chunk) {
 }
 
 struct Layout {
-    size_t part_t, part_d, sel, tilesum, stripsum, total;
+    size_t part_t, part_d, sel, tilesum, total;
     int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
     int nct, ncd, cps, nst, nsd, ntile;
+    int B_big, cps_f, nst_f, nsd_f, pst_t, pst_d;
     unsigned grid;
+    int fin_cluster;     // CTAs per sequence of the cluster kernel; 0: the tile kernels draw the extra token
+    int fin_slice;       // vectors of the target row per CTA of the cluster
+    int fin_dvec;        // vectors reserved for the staged drafter row
+    size_t fin_smem;     // its dynamic shared memory
 };
+
+// The cluster kernel keeps the whole drafter row and four bytes per 16-byte vector of its slice of
+// the target row in shared memory.  It is used when that fits twice into an SM, or once while the
+// whole batch is resident at one CTA per SM; larger vocabularies and batches go to the tile
+// kernels, which are built for throughput.  Small batches get the widest cluster, so that more SMs
+// share the one row.
+constexpr size_t kFinSmemTwoPerSm = 100 * 1024;
+constexpr size_t kFinSmemOnePerSm = 200 * 1024;
+constexpr size_t kFinMaxSmemBytes = kFinSmemOnePerSm;
+void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms) {
+    L.fin_cluster = 0; L.fin_slice = 0; L.fin_dvec = 0; L.fin_smem = 0;
+    const int nvec = chunks_per_row(V_t, dtype, 1);                 // vectors of a row, whatever its alignment
+    const int dvec = chunks_per_row(V_d, dtype, 1);
+    auto need = [&](int c) { return static_cast<size_t>(dvec) * 16 + static_cast<size_t>((nvec + c - 1) / c) * 4; };
+    int C = 0;
+    for (int c = 1; c <= kFinMaxCluster; c *= 2)
+        if (need(c) <= kFinSmemTwoPerSm) { C = c; break; }
+    if (C) {
+        while (C < kFinMaxCluster && static_cast<long long>(B) * C * 2 <= 2LL * num_sms) C *= 2;
+        if (static_cast<long long>(B) * C > 8LL * num_sms) return;
+    } else {
+        for (int c = kFinMaxCluster; c >= 1; c /= 2)
+            if (need(c) <= kFinSmemOnePerSm && static_cast<long long>(B) * c <= num_sms) { C = c; break; }
+        if (C == 0) return;
+    }
+    L.fin_cluster = C;
+    L.fin_slice = (nvec + C - 1) / C;
+    L.fin_dvec = dvec;
+    L.fin_smem = need(C);
+}
 
 // Chunk size: as large as leaves every CTA of the persistent grid (two per SM) about one chunk
 // (measured: the per-chunk bookkeeping costs more than a few idle CTAs do).
@@ -2695,16 +2363,25 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.cps = static_cast<int>(cps < 1 ? 1 : (cps > cap ? cap : cps));
     L.nst = (L.nct + L.cps - 1) / L.cps;
     L.nsd = (L.ncd + L.cps - 1) / L.cps;
-    const long long nseg = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nst + static_cast<long long>(K) * L.nsd);
+    // the last eighth of a batch that keeps the CTAs busy for many segments goes out in single chunks
+    L.B_big = B; L.cps_f = L.cps; L.nst_f = L.nst; L.nsd_f = L.nsd;
+    if (L.cps > 1 && B >= 8 && chunks > ctas * 16) {
+        L.B_big = B - (B + 7) / 8;
+        L.cps_f = 1; L.nst_f = L.nct; L.nsd_f = L.ncd;
+    }
+    L.pst_t = L.nst > L.nst_f ? L.nst : L.nst_f;
+    L.pst_d = L.nsd > L.nsd_f ? L.nsd : L.nsd_f;
+    const long long nseg = static_cast<long long>(L.B_big) * (static_cast<long long>(K + 1) * L.nst + static_cast<long long>(K) * L.nsd) +
+                           static_cast<long long>(B - L.B_big) * (static_cast<long long>(K + 1) * L.nst_f + static_cast<long long>(K) * L.nsd_f);
     const long long grid = nseg < ctas ? nseg : ctas;
     L.grid = static_cast<unsigned>(grid);
     size_t off = 0;
-    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nst, 256);
-    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.nsd, 256);
+    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.pst_t, 256);
+    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.pst_d, 256);
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
     L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.ntile, 256);
-    L.stripsum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.nct * kSWarps, 256);
     L.total = off;
+    plan_finish(L, B, V_t, V_d, dtype, num_sms);
     return L;
 }
 
@@ -2716,7 +2393,7 @@ struct tli_ctx {
     int *d_map;
     int *d_inv;
     uint32_t *d_mask;
-    int fused;                  // option: one fused kernel (default) or three kernels
+    int tiled;                  // option: the extra token always by the tile kernels (default 0: by size)
     unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
@@ -2753,7 +2430,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
-    c->fused = 0;
+    c->tiled = 0;
     int rc = TLI_OK;
     do {
         if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }
@@ -2763,10 +2440,8 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
         TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
 #undef TLI_SET_SMEM
-#define TLI_SET_SMEM(DT, CV) if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_fused_kernel<DT, CV>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFusedSmemBytes)
-        TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
-        TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
-#undef TLI_SET_SMEM
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinMaxSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinMaxSmemBytes);
         if (e != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
@@ -2825,8 +2500,8 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
         return TLI_ERR_ARG;
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
-    if (a->draft_lengths && ctx->fused) return TLI_ERR_UNSUPPORTED;     // the fused form takes whole batches only
-    const Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
+    Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
+    if (ctx->tiled) L.fin_cluster = 0;
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
         return TLI_ERR_WORKSPACE;
 
@@ -2844,31 +2519,18 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.part_d = reinterpret_cast<float2 *>(ws + L.part_d);
     P.sel = reinterpret_cast<RowSel *>(ws + L.sel);
     P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
-    P.stripsum = reinterpret_cast<double *>(ws + L.stripsum);
     P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
-    P.seq_state = reinterpret_cast<int *>(ctx->d_counters + 2 * (TLI_MAX_B + 1));
     P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
-    P.seg_counter = P.error + 1; P.cta_done = P.error + 2; P.samp_counter = P.error + 3;
+    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
     // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
     P.split_select = (static_cast<long long>(a->B) * L.ntile >= 4096) ? 1 : 0;
     P.nct = L.nct; P.ncd = L.ncd; P.ntile = L.ntile; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
+    P.fin_slice = L.fin_slice; P.fin_dvec = L.fin_dvec;
+    P.B_big = L.B_big; P.cps_f = L.cps_f; P.nst_f = L.nst_f; P.nsd_f = L.nsd_f; P.pst_t = L.pst_t; P.pst_d = L.pst_d;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
-    if (ctx->fused && !ev) {
-        const dim3 g1(L.grid), b1(kFThreads);
-#define TLI_LAUNCH_FUSED(DT, CV) tli_fused_kernel<DT, CV><<<g1, b1, kFusedSmemBytes, stream>>>(P)
-        if (a->dtype == TLI_F32) {
-            if (L.cv == 4) TLI_LAUNCH_FUSED(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_FUSED(TLI_F32, 2); else TLI_LAUNCH_FUSED(TLI_F32, 1);
-        } else {
-            if (L.cv == 4) TLI_LAUNCH_FUSED(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_FUSED(TLI_BF16, 2); else TLI_LAUNCH_FUSED(TLI_BF16, 1);
-        }
-#undef TLI_LAUNCH_FUSED
-        const cudaError_t ef = cudaGetLastError();
-        if (ef != cudaSuccess) return cuda_fail(ef, "launch tli_fused_kernel");
-        return TLI_OK;
-    }
     const dim3 grid2(static_cast<unsigned>(L.ntile), static_cast<unsigned>(a->B));
     {
         const dim3 g1(L.grid), b1(kSThreads + 32);
@@ -2884,15 +2546,31 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
 
-    // The three small kernels are launched as programmatic dependents: none of their predecessors
-    // triggers early, so they still start only when the predecessor is done, but their launch is
-    // set up while it runs (4-6 us per call).  Each begins with griddepcontrol.wait.
+    // The kernels after the first are launched as programmatic dependents: no predecessor triggers
+    // early, so they still start only when it is done, but their launch is set up while it runs
+    // (4-6 us per call).  Each begins with griddepcontrol.wait.
     cudaLaunchConfig_t cfg;
     memset(&cfg, 0, sizeof cfg);
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[0].val.programmaticStreamSerializationAllowed = 1;
-    cfg.attrs = attr; cfg.numAttrs = 1; cfg.stream = stream; cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0;
+    cfg.attrs = attr; cfg.numAttrs = 1; cfg.stream = stream;
+    if (L.fin_cluster) {
+        // decision and extra token by one cluster per sequence
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = static_cast<unsigned>(L.fin_cluster);
+        attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+        cfg.blockDim = dim3(kFinThreads); cfg.dynamicSmemBytes = L.fin_smem;
+        cfg.gridDim = dim3(static_cast<unsigned>(L.fin_cluster), static_cast<unsigned>(a->B));
+        if (ev) cudaEventRecord(ev[2], stream);
+        if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_finish_kernel<TLI_F32>, P);
+        else e = cudaLaunchKernelEx(&cfg, tli_finish_kernel<TLI_BF16>, P);
+        if (e != cudaSuccess) return cuda_fail(e, "launch tli_finish_kernel");
+        if (ev) cudaEventRecord(ev[3], stream);
+        return TLI_OK;
+    }
+    cfg.blockDim = dim3(kThreads); cfg.dynamicSmemBytes = 0;
     cfg.gridDim = dim3(static_cast<unsigned>(a->B));
     if (a->dtype == TLI_F32) e = cudaLaunchKernelEx(&cfg, tli_decide_kernel<TLI_F32>, P);
     else e = cudaLaunchKernelEx(&cfg, tli_decide_kernel<TLI_BF16>, P);
@@ -3052,9 +2730,9 @@ int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, i
     return TLI_OK;
 }
 
-int tli_set_fused(tli_ctx *ctx, int enabled) {
+int tli_set_tiled(tli_ctx *ctx, int enabled) {
     if (!ctx) return TLI_ERR_ARG;
-    ctx->fused = enabled ? 1 : 0;
+    ctx->tiled = enabled ? 1 : 0;
     return TLI_OK;
 }
 

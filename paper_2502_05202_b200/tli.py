@@ -37,7 +37,7 @@ TLI_MAX_K = 64
 TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_fused", "tli_selftest_bounded_wait",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
            "tli_verify_host_buffer_bytes", "tli_verify_host", "tli_rates_workspace_bytes", "tli_acceptance_rates",
            "tli_ctx_info",
@@ -150,8 +150,8 @@ def load() -> ctypes.CDLL:
         lib.tli_rates_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_acceptance_rates.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_rates_args), ctypes.c_void_p]
         lib.tli_acceptance_rates.restype = ctypes.c_int
-        lib.tli_set_fused.argtypes = [ctypes.c_void_p, ctypes.c_int]
-        lib.tli_set_fused.restype = ctypes.c_int
+        lib.tli_set_tiled.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        lib.tli_set_tiled.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
         lib.tli_selftest_bounded_wait.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -381,7 +381,7 @@ def tli_slem_verify(ctx: int, args: tli_slem_args, stream: Optional[int] = None)
 
 
 def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = None):
-    """tli_verify_profile(): blocks; returns ms of (statistics kernel, decision kernel, sampling kernel)."""
+    """tli_verify_profile(): blocks; returns ms of (statistics kernel, decision kernel or 0, sampling kernel)."""
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
     ms = (ctypes.c_float * 3)()
@@ -391,11 +391,11 @@ def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = 
     return ms[0], ms[1], ms[2]
 
 
-def tli_set_fused(ctx: int, enabled: bool) -> None:
-    """tli_set_fused(): three kernels per call (default) or one fused kernel."""
-    rc = load().tli_set_fused(ctx, 1 if enabled else 0)
+def tli_set_tiled(ctx: int, enabled: bool) -> None:
+    """tli_set_tiled(): the extra token by size (default) or always by the tile kernels."""
+    rc = load().tli_set_tiled(ctx, 1 if enabled else 0)
     if rc != TLI_OK:
-        raise TLIError(rc, "tli_set_fused")
+        raise TLIError(rc, "tli_set_tiled")
 
 
 def tli_selftest_bounded_wait(ctx: int, polls: int = 2000, stream: Optional[int] = None) -> bool:
@@ -412,12 +412,12 @@ def tli_selftest_bounded_wait(ctx: int, polls: int = 2000, stream: Optional[int]
 class Verifier:
     """Convenience owner of one context plus its scratch and output tensors."""
 
-    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0, fused: bool = False):
+    def __init__(self, V_t: int, V_d: int, id_map, device: int = 0, tiled: bool = False):
         self.device = torch.device("cuda", device)
         self.V_t, self.V_d = int(V_t), int(V_d)
         self.ctx = tli_create(device, V_t, V_d, id_map)
-        if fused:
-            tli_set_fused(self.ctx, True)
+        if tiled:
+            tli_set_tiled(self.ctx, True)
         self._ws: Optional[torch.Tensor] = None
 
     def close(self) -> None:

@@ -44,9 +44,10 @@ def to_device(batch: Dict[str, np.ndarray], device="cuda") -> Dict[str, torch.Te
 
 
 def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = None,
-            dev: Optional[Dict[str, torch.Tensor]] = None) -> Dict[str, np.ndarray]:
-    """One tli_verify() call.  Without a verifier of the caller's, both forms of the call are run
-    (the fused kernel and the three-kernel sequence) and must agree bit for bit."""
+            dev: Optional[Dict[str, torch.Tensor]] = None, tiled: bool = False) -> Dict[str, np.ndarray]:
+    """One tli_verify() call.  Without a verifier of the caller's a context is made for the call
+    (`tiled`: the extra token by the tile kernels whatever the size) and the call is repeated on it:
+    the second call must give the same results bit for bit."""
     if dev is None:
         dev = to_device(batch)
 
@@ -60,20 +61,13 @@ def run_gpu(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = Non
         return once(verifier)
     V_t = batch["target_logits"].shape[2]
     V_d = batch["drafter_logits"].shape[2]
-    res = None
-    forms = (False,) if batch.get("draft_lengths") is not None else (False, True)   # ragged counts: three kernels only
-    for fused in forms:
-        v = tli.Verifier(V_t, V_d, batch["id_map"], fused=fused)
-        r = once(v)
-        r2 = once(v)                                  # a second call on the same context: counters came back to zero
-        v.close()
-        for k in r:
-            np.testing.assert_array_equal(r[k], r2[k], err_msg="repeat call differs (%s, fused=%s)" % (k, fused))
-        if res is not None:
-            for k in r:
-                np.testing.assert_array_equal(res[k], r[k], err_msg="fused and three-kernel results differ: " + k)
-        res = r
-    return res
+    v = tli.Verifier(V_t, V_d, batch["id_map"], tiled=tiled)
+    r = once(v)
+    r2 = once(v)                                  # a second call on the same context: counters came back to zero
+    v.close()
+    for k in r:
+        np.testing.assert_array_equal(r[k], r2[k], err_msg="repeat call differs (%s, tiled=%s)" % (k, tiled))
+    return r
 
 
 def run_oracle(batch: Dict[str, np.ndarray], threads: int = 8, **kw) -> Dict[str, np.ndarray]:
@@ -200,7 +194,16 @@ def compare(batch: Dict[str, np.ndarray], gpu: Dict[str, np.ndarray], orc: Optio
 
 
 def check(batch: Dict[str, np.ndarray], verifier: Optional[tli.Verifier] = None, threads: int = 8) -> Report:
-    gpu = run_gpu(batch, verifier)
-    rep = compare(batch, gpu, threads=threads)
+    """The GPU against the oracle.  Without a verifier of the caller's both forms of the call are
+    checked (extra token by size rule, and by the tile kernels); the report is the default form's."""
+    if verifier is not None:
+        rep = compare(batch, run_gpu(batch, verifier), threads=threads)
+        assert rep.ok(), str(rep)
+        return rep
+    orc = run_oracle(batch, threads=threads)
+    dev = to_device(batch)
+    rep = compare(batch, run_gpu(batch, dev=dev), orc=orc, threads=threads)
     assert rep.ok(), str(rep)
+    rep_tiled = compare(batch, run_gpu(batch, dev=dev, tiled=True), orc=orc, threads=threads)
+    assert rep_tiled.ok(), "tile kernels: " + str(rep_tiled)
     return rep
