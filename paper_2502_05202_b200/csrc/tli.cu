@@ -82,14 +82,10 @@ struct Params {
     unsigned *cnt_stats; unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
     unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
-    int nct, ncd;        // statistics-kernel chunks per target / drafter row
     int ntile;           // 16 KB tiles per target row (sampling pass)
     int split_select;    // 1: the CDF inversions run as a kernel of their own
-    int cps;             // chunks per segment
-    int nst, nsd;        // segments per target / drafter row
-    int B_big;           // sequences [0, B_big) use the segments above; the rest, handed out last, finer ones
-    int cps_f, nst_f, nsd_f;   // ... of cps_f chunks: nst_f / nsd_f segments per row
-    int pst_t, pst_d;    // partials reserved per target / drafter row (the larger of the two counts)
+    int seg_vec;         // statistics kernel: 16-byte vectors per segment
+    int nst, nsd;        // ... and segments per target / drafter row
     int fin_slice;       // cluster kernel: 16-byte vectors of the sampled target row per CTA
     int fin_dvec;        // cluster kernel: 16-byte vectors reserved for the staged drafter row
 };
@@ -276,23 +272,26 @@ __device__ __forceinline__ float2 ld_shared_pair(const float2 *p) {     // a pai
 }
 
 // ---- the schedule both the producer and the consumers walk ----
+//
+// A row is seen as 16-byte vectors on the aligned address grid (RowView).  A segment is a run of
+// consecutive vectors of one row and leaves one partial result; a stage of the ring holds up to
+// 512*CV vectors of it.  Segments are numbered sequence-major and handed out in that order.
+// (Shorter segments for the sequences handed out last, so that the CTAs run dry together, were
+// measured and dropped: what a CTA still holds when the queue runs dry is its ring of stages and
+// the two segments it works ahead, whatever the length of the segments.)
 
 struct Segment {
     int b;            // sequence
     int row;          // 0..K target rows, K+1..2K drafter rows
-    int chunk0, chunk1;
+    int v0, v1;       // vectors [v0, v1) of the row's grid (clipped to the row by the producer)
     int seg;          // index of the segment within its row
     bool skip;        // nothing to read (bad temperature, or drafter row at temperature 0)
     float tau;
     int m;            // drafts of the sequence that count
 };
 
-// Segments are numbered sequence-major.  The sequences from B_big on are cut into finer segments:
-// they are handed out last, when the CTAs are about to run dry, so that no CTA is left with a long
-// segment while the others have finished.
 __device__ __forceinline__ long long segment_count(const Params &P) {
-    return static_cast<long long>(P.B_big) * ((P.K + 1) * P.nst + P.K * P.nsd) +
-           static_cast<long long>(P.B - P.B_big) * ((P.K + 1) * P.nst_f + P.K * P.nsd_f);
+    return static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
 }
 
 // The index arithmetic of a segment, and the loads of its sequence's temperature and draft count:
@@ -301,32 +300,19 @@ __device__ __forceinline__ long long segment_count(const Params &P) {
 __device__ __forceinline__ Segment decode_segment(const Params &P, long long id) {
     Segment g;
     const int per_b = (P.K + 1) * P.nst + P.K * P.nsd;
-    const long long n_big = static_cast<long long>(P.B_big) * per_b;
-    int nst = P.nst, nsd = P.nsd, cps = P.cps;
-    int item;
-    if (id < n_big) {
-        g.b = static_cast<int>(id / per_b);
-        item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
-    } else {
-        nst = P.nst_f; nsd = P.nsd_f; cps = P.cps_f;
-        const int per_f = (P.K + 1) * nst + P.K * nsd;
-        const long long id2 = id - n_big;
-        const int bf = static_cast<int>(id2 / per_f);
-        g.b = P.B_big + bf;
-        item = static_cast<int>(id2 - static_cast<long long>(bf) * per_f);
-    }
+    g.b = static_cast<int>(id / per_b);
+    int item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
     g.tau = __ldg(P.tau + g.b);
     g.m = P.draft_len ? __ldg(P.draft_len + g.b) : P.K;
-    int nchunk;
-    if (item < (P.K + 1) * nst) {
-        g.row = item / nst; g.seg = item - g.row * nst; nchunk = P.nct;
+    if (item < (P.K + 1) * P.nst) {
+        g.row = item / P.nst; g.seg = item - g.row * P.nst;
     } else {
-        item -= (P.K + 1) * nst;
-        const int j = item / nsd;
-        g.row = P.K + 1 + j; g.seg = item - j * nsd; nchunk = P.ncd;
+        item -= (P.K + 1) * P.nst;
+        const int j = item / P.nsd;
+        g.row = P.K + 1 + j; g.seg = item - j * P.nsd;
     }
-    g.chunk0 = g.seg * cps;
-    g.chunk1 = min(g.chunk0 + cps, nchunk);
+    g.v0 = g.seg * P.seg_vec;
+    g.v1 = g.v0 + P.seg_vec;
     g.skip = false;
     return g;
 }
@@ -343,37 +329,33 @@ template <int DT> __device__ __forceinline__ RowView<DT> segment_row(const Param
     return RowView<DT>(P.zd, static_cast<long long>(g.b) * P.d_sb + static_cast<long long>(g.row - P.K - 1) * P.d_sk, P.V_d);
 }
 
-// Vectors of chunk `chunk` that lie wholly inside the row: [v0, v1).  Only these are bulk-copied;
+// Vectors [v0, v1) of the range [a, b) that lie wholly inside the row.  Only these are bulk-copied;
 // the (at most two) ragged vectors of a row are read element by element by the consumers.
-template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT> &rv, int chunk, int cvec, int &v0, int &v1) {
+template <int DT> __device__ __forceinline__ void full_vectors(const RowView<DT> &rv, int a, int b, int &v0, int &v1) {
     constexpr int EPV = Elt<DT>::kPerVec;
     const int first_full = rv.head ? 1 : 0;
     const int end_full = (rv.V + rv.head) / EPV;               // vectors [first_full, end_full) are whole
-    v0 = max(chunk * cvec, first_full);
-    v1 = min((chunk + 1) * cvec, end_full);
+    v0 = max(a, first_full);
+    v1 = min(b, end_full);
     if (v1 < v0) v1 = v0;
 }
 
-// What the producer tells the consumers about the chunk it put into a stage.
-struct StageMeta {
-    long long id;     // segment
-    int chunk;        // chunk of the segment's row held by this stage
-    int flags;        // META_*
-};
 enum : int { META_FIRST = 1, META_LAST = 2, META_END = 4, META_INTERIOR = 16 };
 
-// The statistics kernel's label also carries the decoded segment, so that only the producer
-// thread divides segment numbers and reads temperatures.
+// What the producer tells the consumers about the vectors it put into a stage: the stage holds
+// vectors [v0, v0 + nv) of the row, vector v0 + i at position i.  The label also carries the
+// decoded segment, so that only the producer thread divides segment numbers and reads temperatures.
 struct __align__(16) StatsMeta {
-    int chunk, flags;
+    int v0, nv;
+    int flags;
     int b, row;       // as in Segment
     int seg;
     float tau;
-    int pad[2];
+    int pad;
 };
 
 // Per-warp results of a segment wait in one of kMaxStages + 1 slots (slot = the CTA's segment
-// count modulo that): a warp can be at most a ring of chunks, hence at most kMaxStages segment
+// count modulo that): a warp can be at most a ring of stages, hence at most kMaxStages segment
 // ends, ahead of the warp that is still combining a slot, so no slot is rewritten while in use.
 constexpr int kPairSlots = kMaxStages + 1;
 struct StatsSmem {
@@ -387,25 +369,32 @@ struct StatsSmem {
 
 constexpr int kStatsSmemBytes = kRingBytes + static_cast<int>(sizeof(StatsSmem));
 
-// This thread's CV vectors of one chunk.  Chunks that lie wholly inside the row (all but the first
-// and last of a row) come straight from the stage; the others check every vector.
+// This thread's vectors of one stage: vector q*kSThreads + tid of the stage for q < nq.  A full
+// stage that lies wholly inside the row comes straight from shared memory; a short one checks its
+// length; one that touches an end of the row checks every vector.
 template <int DT, int CV>
-__device__ __forceinline__ void load_chunk(const RowView<DT> &rv, int chunk, bool interior, const uint4 *stage, int tid,
+__device__ __forceinline__ void load_stage(const RowView<DT> &rv, int v0, int nv, bool interior, const uint4 *stage, int tid,
                                            uint4 (&raw)[CV]) {
-    if (interior) {
+    const uint4 ninf = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+    if (interior && nv == kSThreads * CV) {
 #pragma unroll
         for (int q = 0; q < CV; ++q) raw[q] = stage[q * kSThreads + tid];
-    } else {
-        int v0, v1;
-        full_vectors<DT>(rv, chunk, kSThreads * CV, v0, v1);
-        const int nvec = rv.nvec();
+    } else if (interior) {
 #pragma unroll
         for (int q = 0; q < CV; ++q) {
-            const int g_in = q * kSThreads + tid;
-            const int v = chunk * (kSThreads * CV) + g_in;
-            if (v >= v0 && v < v1) raw[q] = stage[g_in];
-            else if (v < nvec) raw[q] = rv.load(v);                      // ragged end of the row
-            else raw[q] = make_uint4(Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord);
+            const int i = q * kSThreads + tid;
+            raw[q] = (i < nv) ? stage[i] : ninf;
+        }
+    } else {
+        int f0, f1;
+        full_vectors<DT>(rv, v0, v0 + nv, f0, f1);
+#pragma unroll
+        for (int q = 0; q < CV; ++q) {
+            const int i = q * kSThreads + tid;
+            const int v = v0 + i;
+            if (i >= nv) raw[q] = ninf;
+            else if (v >= f0 && v < f1) raw[q] = stage[i];
+            else raw[q] = rv.load(v);                                   // ragged end of the row
         }
     }
 }
@@ -436,6 +425,9 @@ __device__ __forceinline__ uint32_t bf16x2_max(uint32_t a, uint32_t b) {
     asm("max.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
 }
+__device__ __forceinline__ uint32_t bf16x2_max(const uint4 &r) {
+    return bf16x2_max(bf16x2_max(r.x, r.y), bf16x2_max(r.z, r.w));
+}
 
 // bf16 vectors of a drafter row: the elements whose mask bit is 0 become -inf, two at a time.
 // The low eight bits of `bits` go to the top bits of eight bytes (a multiplication by four
@@ -457,23 +449,25 @@ __device__ __forceinline__ void mask_bf16_vector(uint4 &r, uint32_t bits) {
     r.w = keep_or_neg_inf(r.w, prmt_sign(hi, 0xbbaau));
 }
 
-// One chunk of a softmax row into this thread's running (reference, sum).
-template <int DT, int CV, bool MASKED>
-__device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint32_t (&bits)[CV], float s,
+// The first nq of a thread's vectors of a stage into its running (reference, sum).  nq is the
+// same for the whole CTA; FULL: the caller knows that nq == CV (no tests in the unrolled loops).
+template <int DT, int CV, bool MASKED, bool FULL>
+__device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint32_t (&bits)[CV], int nq, float s,
                                               float &c_run, float &acc) {
     constexpr int EPV = Elt<DT>::kPerVec;
-    // largest value of the chunk (over ids inside the intersection for a drafter row)
+    // largest value of the vectors (over ids inside the intersection for a drafter row)
     float m;
     if (DT == TLI_BF16 && !MASKED) {
-        uint32_t mm = bf16x2_max(bf16x2_max(raw[0].x, raw[0].y), bf16x2_max(raw[0].z, raw[0].w));
+        uint32_t mm = bf16x2_max(raw[0]);
 #pragma unroll
         for (int q = 1; q < CV; ++q)
-            mm = bf16x2_max(mm, bf16x2_max(bf16x2_max(raw[q].x, raw[q].y), bf16x2_max(raw[q].z, raw[q].w)));
+            if (FULL || q < nq) mm = bf16x2_max(mm, bf16x2_max(raw[q]));
         m = fmaxf(bf16_lo(mm), bf16_hi(mm));
     } else {
         m = -INFINITY;
 #pragma unroll
         for (int q = 0; q < CV; ++q) {
+            if (!FULL && q >= nq) continue;
             float z[EPV];
             unpack<DT>(raw[q], z);
 #pragma unroll
@@ -483,7 +477,7 @@ __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint
             }
         }
     }
-    // raise the reference if this chunk tops it; the sum follows by an exact power of two
+    // raise the reference if these vectors top it; the sum follows by an exact power of two
     const float ms = m * s;
     if (ms > c_run) {
         const float c_new = reference_for(ms);
@@ -495,6 +489,7 @@ __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint
     uint64_t a2[2] = {pack2(0.f, 0.f), pack2(0.f, 0.f)};
 #pragma unroll
     for (int q = 0; q < CV; ++q) {
+        if (!FULL && q >= nq) continue;
         float z[EPV];
         unpack<DT>(raw[q], z);
 #pragma unroll
@@ -514,30 +509,39 @@ __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint
     acc += (a0 + a1) + (a3 + a4);
 }
 
-template <int DT, int CV>
-__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], const RowView<DT> &rv, int chunk, int tid,
-                                             float &best, int &best_idx) {
+// Temperature-0 rows: (largest value, lowest index attaining it) over the first nq vectors.
+// bf16: a running pair of packed maxima (even and odd positions) tells in five instructions
+// whether a vector can raise the maximum at all; only then are its eight elements compared.
+template <int DT, int CV, bool FULL>
+__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], int nq, const RowView<DT> &rv, int v_first,
+                                             uint32_t &mm, float &best, int &best_idx) {
     constexpr int EPV = Elt<DT>::kPerVec;
 #pragma unroll
     for (int q = 0; q < CV; ++q) {                        // increasing index order, strict > keeps the lowest
+        if (!FULL && q >= nq) continue;
+        if constexpr (DT == TLI_BF16) {
+            const uint32_t nm = bf16x2_max(mm, bf16x2_max(raw[q]));
+            if (nm == mm) continue;
+            mm = nm;
+        }
         float z[EPV];
         unpack<DT>(raw[q], z);
-        const int e0 = rv.first_elem(chunk * (kSThreads * CV) + q * kSThreads + tid);
+        const int e0 = rv.first_elem(v_first + q * kSThreads);
 #pragma unroll
         for (int i = 0; i < EPV; ++i)
             if (z[i] > best) { best = z[i]; best_idx = e0 + i; }
     }
 }
 
-// Segments are handed out by an atomic counter: a CTA that is busy closing a sequence simply takes
-// fewer of them.  The producer thread fetches the next segment number while it is still loading the
-// current one, streams the chunks through the stage ring and labels every stage for the consumers.
-// CV = 16-byte vectors per consumer thread per chunk: the chunk is kSThreads*CV*16 bytes and the
-// ring holds kRingBytes / that many stages.  Large batches use large chunks (less bookkeeping per
-// byte), small ones small chunks (more parallelism across CTAs).
+// Segments are handed out by an atomic counter: a CTA that is slow simply takes fewer of them.
+// The producer thread works two segments ahead (see above), streams the vectors through the stage
+// ring and labels every stage for the consumers.
+// CV = 16-byte vectors per consumer thread per stage: a stage is kSThreads*CV*16 bytes and the
+// ring holds kRingBytes / that many stages.  Large batches use large stages (less bookkeeping per
+// byte), small ones small stages (more parallelism across CTAs).
 template <int DT, int CV>
 __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(const Params P) {
-    constexpr int CVEC = kSThreads * CV;                       // vectors per chunk
+    constexpr int CVEC = kSThreads * CV;                       // vectors per stage
     constexpr int NST = kRingBytes / (CVEC * 16);              // stages
     static_assert(NST >= 2 && NST <= kMaxStages, "stage count");
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -561,8 +565,6 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             bool ok = true;
             // every CTA starts on the segment of its own number (so that a small batch spreads over all
             // CTAs however unevenly they start); the rest come from the counter
-            // two segments ahead: the number of the one after next is being fetched, the next one's
-            // temperature is being loaded, the current one is streamed
             long long id = blockIdx.x;
             Segment g = decode_segment(P, id);
             long long id_next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);
@@ -576,34 +578,39 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 g = g_next; id = id_next; id_next = id_after;
                 if (gc.skip) continue;                   // bad temperature, or drafter row at temperature 0
                 const RowView<DT> rv = segment_row<DT>(P, gc);
-                for (int chunk = gc.chunk0; chunk < gc.chunk1; ++chunk) {
+                const int v_end = min(gc.v1, rv.nvec());
+                int v0 = gc.v0;
+                do {                                     // an empty segment still sends one (empty) stage
+                    const int nv = max(0, min(CVEC, v_end - v0));
                     ok = mbar_wait(&sm.empty[st], par, &sm.error, P.error);
                     if (!ok) break;
-                    int v0, v1;
-                    full_vectors<DT>(rv, chunk, CVEC, v0, v1);
-                    const bool interior = (v0 == chunk * CVEC && v1 == (chunk + 1) * CVEC);
+                    int f0, f1;
+                    full_vectors<DT>(rv, v0, v0 + nv, f0, f1);
+                    const bool interior = (f0 == v0 && f1 == v0 + nv);
                     StatsMeta mt;
-                    mt.chunk = chunk;
-                    mt.flags = (chunk == gc.chunk0 ? META_FIRST : 0) | (chunk == gc.chunk1 - 1 ? META_LAST : 0) |
+                    mt.v0 = v0; mt.nv = nv;
+                    mt.flags = (v0 == gc.v0 ? META_FIRST : 0) | (v0 + CVEC >= v_end ? META_LAST : 0) |
                                (interior ? META_INTERIOR : 0);
-                    mt.b = gc.b; mt.row = gc.row; mt.seg = gc.seg; mt.tau = gc.tau; mt.pad[0] = mt.pad[1] = 0;
+                    mt.b = gc.b; mt.row = gc.row; mt.seg = gc.seg; mt.tau = gc.tau; mt.pad = 0;
                     sm.meta[st] = mt;
-                    const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
+                    const unsigned bytes = static_cast<unsigned>(f1 - f0) * 16u;
                     mbar_arrive_expect_tx(&sm.full[st], bytes);
                     if (bytes)
-                        bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (v0 - chunk * CVEC),
-                                  rv.vec0 + v0, bytes, &sm.full[st]);
+                        bulk_load(stage_base + static_cast<size_t>(st) * CVEC + (f0 - v0), rv.vec0 + f0, bytes, &sm.full[st]);
                     ++issued;
                     if (++st == NST) { st = 0; par ^= 1u; }
-                }
+                    v0 += CVEC;
+                } while (v0 < v_end);
             }
             // nothing more to start: the next kernel of the stream may be made resident as CTAs of this
-            // one leave (it still waits for all of this grid before it reads the partials)
+            // one leave (it still waits for all of this grid before it reads the partials).  Triggering
+            // earlier, when the queue runs dry, was measured: the early residents slow the last segments
+            // down by as much as their prologue saves.
             asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
             if (ok) {                                    // tell the consumers there is nothing more
                 if (mbar_wait(&sm.empty[st], par, &sm.error, P.error)) {
                     StatsMeta mt;
-                    mt.chunk = 0; mt.flags = META_END; mt.b = 0; mt.row = 0; mt.seg = 0; mt.tau = 1.f; mt.pad[0] = mt.pad[1] = 0;
+                    mt.v0 = 0; mt.nv = 0; mt.flags = META_END; mt.b = 0; mt.row = 0; mt.seg = 0; mt.tau = 1.f; mt.pad = 0;
                     sm.meta[st] = mt;
                     mbar_arrive(&sm.full[st]);
                 }
@@ -623,12 +630,13 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         // ---------------- consumers ----------------
         const int tid = threadIdx.x - 32, lane = tid & 31, warp = tid >> 5;
         Segment g;
-        g.b = 0; g.row = 0; g.chunk0 = g.chunk1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f; g.m = 0;
+        g.b = 0; g.row = 0; g.v0 = g.v1 = 0; g.seg = 0; g.skip = false; g.tau = 1.f; g.m = 0;
         RowView<DT> rv(P.zt, 0, P.V_t);
         bool greedy = false, masked = false;
         float s = 0.f;
         float c_run = kNegBig, acc = 0.f;                  // softmax rows: reference, sum
         float best = -INFINITY; int best_idx = INT_MAX;    // temperature-0 rows: max, lowest index
+        uint32_t best_mm = Elt<TLI_BF16>::kNegInfWord;     // ... and the packed maxima of bf16 rows
         bool clean_exit = false;
         unsigned slot = 0;                                 // where this segment's per-warp results meet
         unsigned st = 0, par = 0;                          // stage and the parity of its "full" phase to wait for
@@ -645,34 +653,37 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 greedy = (g.tau == 0.f);
                 masked = g.row > P.K;
                 s = 1.4426950408889634f / g.tau;
-                c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX;
+                c_run = kNegBig; acc = 0.f; best = -INFINITY; best_idx = INT_MAX; best_mm = Elt<TLI_BF16>::kNegInfWord;
             }
-            const int chunk = meta.chunk;
+            const int v0 = meta.v0, nv = meta.nv;
+            const int nq = (nv + kSThreads - 1) / kSThreads;                  // the same for the whole CTA
             uint32_t bits[CV] = {};
             if (masked) {                                  // the mask words travel while the stage is read
-                const int nvec = rv.nvec();
 #pragma unroll
                 for (int q = 0; q < CV; ++q) {
-                    const int v = chunk * CVEC + q * kSThreads + tid;
-                    bits[q] = (v < nvec) ? mask_bits(P.maskbits, rv.first_elem(v)) : 0u;
+                    const int i = q * kSThreads + tid;
+                    bits[q] = (i < nv) ? mask_bits(P.maskbits, rv.first_elem(v0 + i)) : 0u;
                 }
             }
             uint4 raw[CV];
-            load_chunk<DT, CV>(rv, chunk, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
+            load_stage<DT, CV>(rv, v0, nv, (meta.flags & META_INTERIOR) != 0, stage, tid, raw);
             __syncwarp();
             if (lane == 0) mbar_arrive(empty_bar);                            // stage may be refilled now
-            if (greedy) {
-                argmax_chunk<DT, CV>(raw, rv, chunk, tid, best, best_idx);
-            } else if (masked) {
-                if constexpr (DT == TLI_BF16) {               // mask the packed words, then as a target row
+            if (masked && !greedy) {
+                if constexpr (DT == TLI_BF16) {                   // mask the packed words, then as a target row
 #pragma unroll
                     for (int q = 0; q < CV; ++q) mask_bf16_vector(raw[q], bits[q]);
-                    softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
-                } else {
-                    softmax_chunk<DT, CV, true>(raw, bits, s, c_run, acc);
                 }
-            } else {
-                softmax_chunk<DT, CV, false>(raw, bits, s, c_run, acc);
+            }
+            constexpr bool kMaskInSum = (DT != TLI_BF16);          // fp32 drafter rows apply the mask element by element
+            if (nq == CV) {
+                if (greedy) argmax_chunk<DT, CV, true>(raw, nq, rv, v0 + tid, best_mm, best, best_idx);
+                else if (masked && kMaskInSum) softmax_chunk<DT, CV, true, true>(raw, bits, nq, s, c_run, acc);
+                else softmax_chunk<DT, CV, false, true>(raw, bits, nq, s, c_run, acc);
+            } else if (nq > 0) {
+                if (greedy) argmax_chunk<DT, CV, false>(raw, nq, rv, v0 + tid, best_mm, best, best_idx);
+                else if (masked && kMaskInSum) softmax_chunk<DT, CV, true, false>(raw, bits, nq, s, c_run, acc);
+                else softmax_chunk<DT, CV, false, false>(raw, bits, nq, s, c_run, acc);
             }
             if (!(meta.flags & META_LAST)) continue;
 
@@ -729,8 +740,8 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                 }
                 if (lane == 0) {
                     float2 *dst = (g.row <= P.K)
-                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.pst_t + g.seg
-                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.pst_d + g.seg;
+                        ? P.part_t + (static_cast<size_t>(g.b) * (P.K + 1) + g.row) * P.nst + g.seg
+                        : P.part_d + (static_cast<size_t>(g.b) * P.K + (g.row - P.K - 1)) * P.nsd + g.seg;
                     __stcg(dst, pr);
                 }
             }
@@ -818,10 +829,9 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
         const int sub = tid & 7;
         const bool is_t = r <= K;
         const bool mine = r < nrows && (is_t ? r <= Kb : r - K - 1 < Kb);
-        const bool fine = b >= P.B_big;
-        const int nseg = !mine ? 0 : (is_t ? (fine ? P.nst_f : P.nst) : (fine ? P.nsd_f : P.nsd));
-        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.pst_t
-                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.pst_d;
+        const int nseg = !mine ? 0 : (is_t ? P.nst : P.nsd);
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
         if (greedy) {
             float best = -INFINITY; int idx = INT_MAX;
             for (int i = sub; i < nseg; i += 8) {
@@ -1299,7 +1309,7 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
 // boundaries and about ten dependent trips of the tile form.  Every CTA of a cluster takes the
 // same branches (they decide from the same data), so the barriers always meet.
 
-constexpr int kFinThreads = 512;
+constexpr int kFinThreads = 512;                   // 1024 threads where one CTA has an SM to itself: measured slower (64 registers)
 constexpr int kFinWarps = kFinThreads / 32;
 constexpr int kFinMaxCluster = 8;
 
@@ -1360,7 +1370,7 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
     if (sel.mode == MODE_RESIDUAL && count > 0) {
         const RowView<DT> rd(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n) * P.d_sk, P.V_d);
         int v0, v1;
-        full_vectors<DT>(rd, 0, INT_MAX / 2, v0, v1);          // the vectors wholly inside the row: [v0, v1)
+        full_vectors<DT>(rd, 0, rd.nvec(), v0, v1);            // the vectors wholly inside the row: [v0, v1)
         if (tid == 0) {
             const unsigned bytes = static_cast<unsigned>(v1 - v0) * 16u;
             mbar_arrive_expect_tx(&sm_bar, bytes);
@@ -2302,8 +2312,8 @@ int chunks_per_row(int V, int dtype, int vec_per_chunk) {
 struct Layout {
     size_t part_t, part_d, sel, tilesum, total;
     int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
-    int nct, ncd, cps, nst, nsd, ntile;
-    int B_big, cps_f, nst_f, nsd_f, pst_t, pst_d;
+    int ntile;
+    int seg_vec, nst, nsd;      // segments of the statistics kernel, see Params
     unsigned grid;
     int fin_cluster;     // CTAs per sequence of the cluster kernel; 0: the tile kernels draw the extra token
     int fin_slice;       // vectors of the target row per CTA of the cluster
@@ -2318,7 +2328,6 @@ struct Layout {
 // share the one row.
 constexpr size_t kFinSmemTwoPerSm = 100 * 1024;
 constexpr size_t kFinSmemOnePerSm = 200 * 1024;
-constexpr size_t kFinMaxSmemBytes = kFinSmemOnePerSm;
 void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms) {
     L.fin_cluster = 0; L.fin_slice = 0; L.fin_dvec = 0; L.fin_smem = 0;
     const int nvec = chunks_per_row(V_t, dtype, 1);                 // vectors of a row, whatever its alignment
@@ -2341,10 +2350,12 @@ void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms) {
     L.fin_smem = need(C);
 }
 
-// Chunk size: as large as leaves every CTA of the persistent grid (two per SM) about one chunk
-// (measured: the per-chunk bookkeeping costs more than a few idle CTAs do).
-// Segment size: about four segments per CTA (they are handed out dynamically, so that is enough to
-// balance the tail), long enough to amortise the per-segment reduction, at most 128 KB.
+// Stage size: as large as leaves every CTA of the persistent grid (two per SM) about one stage
+// (measured: the per-stage bookkeeping costs more than a few idle CTAs do).
+// Segment size: a batch that gives every CTA many stages is cut into segments of up to 128 KB,
+// about four per CTA (long enough to amortise the per-segment reduction; longer ones interleave the
+// rows of a large batch worse).  A small batch is cut into the shortest segments that still number
+// no more than the CTAs.
 Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     Layout L;
     const long long elt = dtype == TLI_F32 ? 4 : 2;
@@ -2353,31 +2364,32 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.cv = 1;
     if (bytes >= ctas * (kSThreads * 2 * 16)) L.cv = 2;
     if (bytes >= ctas * (kSThreads * 4 * 16)) L.cv = 4;
-    L.nct = chunks_per_row(V_t, dtype, kSThreads * L.cv);
-    L.ncd = chunks_per_row(V_d, dtype, kSThreads * L.cv);
+    const int cvec = kSThreads * L.cv;                               // vectors per stage
+    const int nvec_t = chunks_per_row(V_t, dtype, 1), nvec_d = chunks_per_row(V_d, dtype, 1);
     L.ntile = chunks_per_row(V_t, dtype, kVecPerTile);
-    const long long chunks = static_cast<long long>(B) * (static_cast<long long>(K + 1) * L.nct + static_cast<long long>(K) * L.ncd);
-    long long cps = chunks / (ctas * 4);
-    if (chunks <= ctas * 16) cps = (chunks + ctas - 1) / ctas;      // small batch: about one segment per CTA
-    const long long cap = 16 / L.cv;                                 // 128 KB: longer segments interleave rows worse
-    L.cps = static_cast<int>(cps < 1 ? 1 : (cps > cap ? cap : cps));
-    L.nst = (L.nct + L.cps - 1) / L.cps;
-    L.nsd = (L.ncd + L.cps - 1) / L.cps;
-    // the last eighth of a batch that keeps the CTAs busy for many segments goes out in single chunks
-    L.B_big = B; L.cps_f = L.cps; L.nst_f = L.nst; L.nsd_f = L.nsd;
-    if (L.cps > 1 && B >= 8 && chunks > ctas * 16) {
-        L.B_big = B - (B + 7) / 8;
-        L.cps_f = 1; L.nst_f = L.nct; L.nsd_f = L.ncd;
+    auto per_row = [](int nvec, int sv) { return (nvec + sv - 1) / sv; };
+    auto count = [&](int sv) {
+        return static_cast<long long>(B) * (static_cast<long long>(K + 1) * per_row(nvec_t, sv) + static_cast<long long>(K) * per_row(nvec_d, sv));
+    };
+    const long long stages = count(cvec);
+    const int sv_cap = 16 * kSThreads;                               // 128 KB
+    if (stages <= ctas * 16) {
+        L.seg_vec = kSThreads;
+        while (L.seg_vec < sv_cap && count(L.seg_vec) > ctas) L.seg_vec += kSThreads;
+    } else {
+        long long cps = stages / (ctas * 4);
+        const long long cap = sv_cap / cvec;
+        cps = cps < 1 ? 1 : (cps > cap ? cap : cps);
+        L.seg_vec = static_cast<int>(cps) * cvec;
     }
-    L.pst_t = L.nst > L.nst_f ? L.nst : L.nst_f;
-    L.pst_d = L.nsd > L.nsd_f ? L.nsd : L.nsd_f;
-    const long long nseg = static_cast<long long>(L.B_big) * (static_cast<long long>(K + 1) * L.nst + static_cast<long long>(K) * L.nsd) +
-                           static_cast<long long>(B - L.B_big) * (static_cast<long long>(K + 1) * L.nst_f + static_cast<long long>(K) * L.nsd_f);
+    L.nst = per_row(nvec_t, L.seg_vec);
+    L.nsd = per_row(nvec_d, L.seg_vec);
+    const long long nseg = count(L.seg_vec);
     const long long grid = nseg < ctas ? nseg : ctas;
     L.grid = static_cast<unsigned>(grid);
     size_t off = 0;
-    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.pst_t, 256);
-    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.pst_d, 256);
+    L.part_t = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * (K + 1) * L.nst, 256);
+    L.part_d = off; off = align_up(off + sizeof(float2) * static_cast<size_t>(B) * K * L.nsd, 256);
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
     L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.ntile, 256);
     L.total = off;
@@ -2440,8 +2452,8 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         TLI_SET_SMEM(TLI_F32, 1); TLI_SET_SMEM(TLI_F32, 2); TLI_SET_SMEM(TLI_F32, 4);
         TLI_SET_SMEM(TLI_BF16, 1); TLI_SET_SMEM(TLI_BF16, 2); TLI_SET_SMEM(TLI_BF16, 4);
 #undef TLI_SET_SMEM
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinMaxSmemBytes);
-        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinMaxSmemBytes);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemOnePerSm);
+        if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemOnePerSm);
         if (e != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
@@ -2525,9 +2537,9 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
     // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
     P.split_select = (static_cast<long long>(a->B) * L.ntile >= 4096) ? 1 : 0;
-    P.nct = L.nct; P.ncd = L.ncd; P.ntile = L.ntile; P.cps = L.cps; P.nst = L.nst; P.nsd = L.nsd;
+    P.ntile = L.ntile;
     P.fin_slice = L.fin_slice; P.fin_dvec = L.fin_dvec;
-    P.B_big = L.B_big; P.cps_f = L.cps_f; P.nst_f = L.nst_f; P.nsd_f = L.nsd_f; P.pst_t = L.pst_t; P.pst_d = L.pst_d;
+    P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
