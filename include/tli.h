@@ -55,7 +55,8 @@ enum {
     TLI_ROW_DRAFT_UNMAPPED = 2,   /* a draft id outside the intersection: rejected (q' = 0 there) */
     TLI_ROW_NONFINITE = 4,        /* NaN or +inf logit seen: accepted = 0, next_token = 0 */
     TLI_ROW_FALLBACK = 8,         /* empty intersection or zero residual mass: sampled from p instead */
-    TLI_ROW_TIMEOUT = 16,         /* a bounded wait inside a kernel ran out (sticky for the context): results not to be trusted */
+    TLI_ROW_TIMEOUT = 16,         /* a bounded wait inside a kernel ran out: results not to be trusted.  Sticky: every
+                                   * later call on the context reports it too, until tli_reset() */
     TLI_ROW_BAD_TEMPERATURE = 32  /* temperature negative or not finite: accepted = 0, next_token = 0 */
 };
 
@@ -152,7 +153,15 @@ typedef struct {
  *
  * All arithmetic on the vocabulary rows is fp32 with fp64 combination of
  * partial sums; temperature-0 rows are exact comparisons on the stored values.
- * A logit of -inf is a token of probability zero; NaN or +inf flags the row.
+ * A logit of -inf is a token of probability zero.  NaN or +inf flags the
+ * sequence (TLI_ROW_NONFINITE, accepted = 0, next_token = 0) when it lies in a
+ * row of one of the drafts that count (target and drafter rows 0 .. m-1, m = K
+ * or draft_lengths[b]) or, when all of them are accepted, in the bonus row m;
+ * in a drafter row only at an id inside the intersection: drafter logits
+ * outside the intersection do not enter q' and are not examined.  In a
+ * temperature-0 sequence a NaN never compares greater than anything, so it is
+ * never the arg-max; which id wins in a row that holds a NaN before its largest
+ * value is unspecified.
  *
  * Returns TLI_ERR_ARG / TLI_ERR_WORKSPACE / TLI_ERR_UNSUPPORTED for
  * host-detectable argument errors (nothing is launched) and TLI_ERR_CUDA if a
@@ -395,6 +404,17 @@ int tli_set_tiled(tli_ctx *ctx, int enabled);
  * not touch the context's sticky error word; the context stays usable.
  */
 int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up);
+
+/*
+ * Put the context's device-side counters back to their initial state (a
+ * stream-ordered memset): the completion tickets, the segment scheduler and the
+ * sticky time-out word.  Needed only after a call reported TLI_ROW_TIMEOUT: the
+ * kernels of that call gave up in mid-flight, so the counters they share with
+ * the next call are not back at zero, and every later call would both start from
+ * them and carry the flag.  Must be ordered after the call that timed out and
+ * before the next one, like any other call on the context.
+ */
+int tli_reset(tli_ctx *ctx, void *cuda_stream);
 
 /* Vocabulary sizes and number of mapped drafter ids of a context. */
 int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapped);

@@ -2399,6 +2399,8 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
 
 }  // namespace
 
+constexpr size_t kCounterWords = 3 * (TLI_MAX_B + 1) + 8;     // per-sequence tickets (two sets, one spare), sticky error, schedulers
+
 struct tli_ctx {
     int device;
     int32_t V_t, V_d, n_mapped;
@@ -2458,11 +2460,11 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
-        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * kCounterWords)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
         if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
         if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
         if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
-        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * (3 * (TLI_MAX_B + 1) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
+        if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * kCounterWords)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
     } while (0);
     if (rc != TLI_OK) {
         cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
@@ -2740,6 +2742,12 @@ int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, i
     if ((e = cudaStreamSynchronize(stream)) != cudaSuccess) return cuda_fail(e, "cudaStreamSynchronize");
     *gave_up = (h[0] == 1 && h[1] == 1) ? 1 : 0;
     return TLI_OK;
+}
+
+int tli_reset(tli_ctx *ctx, void *cuda_stream) {
+    if (!ctx) return TLI_ERR_ARG;
+    const cudaError_t e = cudaMemsetAsync(ctx->d_counters, 0, sizeof(unsigned) * kCounterWords, reinterpret_cast<cudaStream_t>(cuda_stream));
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "cudaMemsetAsync counters");
 }
 
 int tli_set_tiled(tli_ctx *ctx, int enabled) {

@@ -37,7 +37,7 @@ TLI_MAX_K = 64
 TLI_MAX_V = 1048576
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_selftest_bounded_wait",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_reset", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
            "tli_verify_host_buffer_bytes", "tli_verify_host", "tli_rates_workspace_bytes", "tli_acceptance_rates",
            "tli_ctx_info",
@@ -150,6 +150,8 @@ def load() -> ctypes.CDLL:
         lib.tli_rates_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_acceptance_rates.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_rates_args), ctypes.c_void_p]
         lib.tli_acceptance_rates.restype = ctypes.c_int
+        lib.tli_reset.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        lib.tli_reset.restype = ctypes.c_int
         lib.tli_set_tiled.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_tiled.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
@@ -396,6 +398,15 @@ def tli_set_tiled(ctx: int, enabled: bool) -> None:
     rc = load().tli_set_tiled(ctx, 1 if enabled else 0)
     if rc != TLI_OK:
         raise TLIError(rc, "tli_set_tiled")
+
+
+def tli_reset(ctx: int, stream: Optional[int] = None) -> None:
+    """tli_reset(): the context's counters and its sticky time-out word back to zero, in stream order."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_reset(ctx, ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_reset")
 
 
 def tli_selftest_bounded_wait(ctx: int, polls: int = 2000, stream: Optional[int] = None) -> bool:

@@ -103,16 +103,15 @@ def test_small_and_ragged_vocabularies(dtype, B, R, V_d):
 
 @pytest.mark.parametrize("name", ["cfg0", "cfg1", "cfg2", "cfg3", "cfg4"])
 def test_drafter_rows_of_the_five_workloads(name):
-    """The drafter logits of each workload at full width (all K rows of up to 64 sequences)."""
+    """The drafter logits of each workload at full width and full batch (all K rows of every sequence)."""
     cfg = wl.config_by_name(name)
-    rows = list(range(min(cfg.B, 64)))
-    batch = wl.make_batch(cfg, rows=rows)
+    batch = wl.make_batch(cfg)
     zd = batch["drafter_logits"]
     B, K, _ = zd.shape
     u = batch["uniforms"][:, :K]
     gpu = run_gpu(zd, batch["id_map"], batch["temperature"], u, cfg.V_t)
     excused, orc = compare(zd, batch["id_map"], batch["temperature"], u, gpu)
-    assert excused <= 2
+    assert excused <= 4
     assert (orc["flags"] == 0).all()
 
 

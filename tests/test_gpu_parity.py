@@ -186,6 +186,79 @@ def test_nan_and_plus_infinity_flag_the_row():
         np.testing.assert_array_equal(gpu[k][~flagged], clean[k][~flagged])
 
 
+def test_non_finite_logits_where_the_oracle_and_the_header_say_they_count():
+    """The rule of tli.h, case by case, against the oracle: a NaN in the bonus row counts only when every
+    draft was accepted; at a drafter id outside the intersection it is not examined (the oracle, which
+    forms the softmax over all of D, is given a finite value there); in a temperature-0 row a NaN past
+    the first element is never the arg-max on either side."""
+    cfg = wl.tiny_config(B=6, K=3, V_t=5000, V_d=4000, dtype=wl.F32, f_mapped=0.5, sigma_d=0.3,
+                         temperatures=(1.0,), seed=47)
+    batch = wl.make_batch(cfg)
+    batch["temperature"] = np.array([1.0, 1.0, 1.0, 1.0, 0.0, 0.0], np.float32)
+    clean = run_oracle(batch)
+    K = cfg.K
+    rejected = [b for b in range(4) if clean["accepted"][b] < K]
+    accepted_all = [b for b in range(4) if clean["accepted"][b] == K]
+    zt, zd = batch["target_logits"].copy(), batch["drafter_logits"].copy()
+    unmapped = np.flatnonzero(batch["id_map"] < 0)
+    for b in range(4):
+        zt[b, K, 123] = np.nan                       # bonus row of every sampled sequence
+    zd_orc = zd.copy()
+    zd[0, 0, unmapped[3]] = np.nan                   # outside the intersection: not examined by the GPU
+    zd[1, 1, unmapped[7]] = np.inf
+    zt[4, 1, 2500] = np.nan                          # temperature 0: never the arg-max
+    zt[5, 0, 77] = np.nan
+    gpu = run_gpu(dict(batch, target_logits=zt, drafter_logits=zd))
+    orc = run_oracle(dict(batch, target_logits=zt, drafter_logits=zd_orc))
+    assert rejected, "the case needs a sequence with a rejected draft"
+    for b in rejected:
+        assert orc["flags"][b] == 0 and gpu["row_status"][b] == 0
+    for b in accepted_all:
+        assert orc["flags"][b] == oracle.FLAG_NONFINITE and gpu["row_status"][b] == tli.TLI_ROW_NONFINITE
+    rep = compare(dict(batch, target_logits=zt, drafter_logits=zd_orc), gpu, orc=orc)
+    assert rep.ok(), str(rep)
+    tiled = run_gpu(dict(batch, target_logits=zt, drafter_logits=zd), tiled=True)
+    rep = compare(dict(batch, target_logits=zt, drafter_logits=zd_orc), tiled, orc=orc)
+    assert rep.ok(), "tile kernels: " + str(rep)
+
+
+def test_exactly_zero_residual_falls_back_to_the_target_distribution():
+    """p = q' = 2^-k exactly (identity map, equal logits, power-of-two vocabulary): a draft outside the
+    vocabulary leaves a residual of exactly zero, the fall-back flag, and a token drawn from p --
+    the same on the oracle (pinned on the CPU side) and on both forms of the GPU call."""
+    for dtype in (wl.F32, wl.BF16):
+        V, K, B = 4096, 2, 6
+        zt = np.zeros((B, K + 1, V), np.float32)
+        zd = np.zeros((B, K, V), np.float32)
+        if dtype == wl.BF16:
+            zt, zd = bf16(zt), bf16(zd)
+        batch = {"target_logits": zt, "drafter_logits": zd, "id_map": np.arange(V, dtype=np.int32),
+                 "draft_ids": np.array([[V, 0], [-1, 3], [2, V + 5], [1, 2], [7, -9], [0, 0]], np.int32),
+                 "temperature": np.ones(B, np.float32),
+                 "uniforms": np.array([[0.5, 0.5, 0.30], [0.1, 0.2, 0.99], [0.9, 0.1, 0.0625], [0.3, 0.3, 0.5],
+                                       [0.999, 0.0, 0.124], [0.2, 0.4, 0.9999]], np.float32)}
+        rep = check(batch)
+        assert rep.exact == B and rep.excused_sampler == 0, str(rep)
+        gpu = run_gpu(batch)
+        fb = tli.TLI_ROW_DRAFT_RANGE | tli.TLI_ROW_FALLBACK
+        assert gpu["row_status"].tolist() == [fb, fb, fb, 0, fb, 0]
+        assert gpu["next_token"].tolist() == [int(np.floor(float(v) * V)) for v in batch["uniforms"][:, K]]
+
+
+def test_reset_brings_the_counters_back():
+    """tli_reset() zeroes the context's counters in stream order; calls before and after agree."""
+    cfg = wl.tiny_config(B=4, K=3, V_t=9000, V_d=7000, dtype=wl.BF16, f_mapped=0.5, seed=48)
+    batch = wl.make_batch(cfg)
+    v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+    before = run_gpu(batch, v)
+    tli.tli_reset(v.ctx)
+    after = run_gpu(batch, v)
+    for k in before:
+        np.testing.assert_array_equal(before[k], after[k])
+    assert tli.load().tli_reset(None, None) == tli.TLI_ERR_ARG
+    v.close()
+
+
 def test_bad_temperature_flags_the_row():
     cfg = wl.tiny_config(B=5, K=2, V_t=500, V_d=400, seed=43)
     batch = wl.make_batch(cfg)

@@ -454,8 +454,11 @@ def test_force_accept_and_flags():
         oracle.verify(zt, zd, bad, d, [1.0], u)
 
 
-def test_oracle_catches_a_planted_wrong_denominator():
-    """The enumeration pin is sensitive: using q (not q') as the proposal breaks the identity."""
+def test_enumeration_pin_catches_a_forgotten_renormalisation():
+    """The enumeration pin is sensitive where it matters.  Feed the oracle drafter logits whose softmax is
+    the *unnormalised* q restricted to the intersection (so that its q' is right), then read its
+    thresholds and residual while the drafts are assumed to come from q instead of q': the identity
+    sum_x q(x) [a 1{map x = t} + (1 - a) r(t)] = p(t) must fail, by the mass q puts outside T."""
     rng = np.random.default_rng(41)
     V_t, V_d = 6, 7
     id_map = random_map(rng, V_d, V_t, 4)
@@ -463,18 +466,50 @@ def test_oracle_catches_a_planted_wrong_denominator():
     zd = rng.normal(0, 1.5, V_d).astype(np.float32)
     p = softmax(zt, 1.0)
     q = softmax(zd, 1.0)
-    inside = id_map >= 0
-    # a verifier that forgot the renormalisation would accept with min(1, p/q) while drafting from q'
-    qp = qprime_def(q, id_map)
-    a_wrong = np.minimum(1.0, p[id_map[inside]] / q[inside])
-    qT = np.zeros(V_t)
-    qT[id_map[inside]] = q[inside]
-    r_wrong = np.maximum(0, p - qT)
-    r_wrong /= r_wrong.sum()
-    dist = np.zeros(V_t)
-    np.add.at(dist, id_map[inside], qp[inside] * a_wrong)
-    dist += (qp[inside] * (1 - a_wrong)).sum() * r_wrong
-    assert np.abs(dist - p).max() > 1e-3
+    inside = np.flatnonzero(id_map >= 0)
+    thr = np.zeros(V_d)
+    for x in inside:                                   # the oracle's acceptance probability of every draft
+        o = oracle.verify(zt[None, None].repeat(2, 1), zd[None, None], id_map, np.array([[x]], np.int32),
+                          np.ones(1, np.float32), np.zeros((1, 2), np.float32))
+        thr[x] = o["thr"][0, 0]
+    # the oracle's residual, read off its CDF for a draft it rejects
+    x0 = inside[np.argmin(thr[inside])]
+    assert thr[x0] < 1.0
+    r = np.zeros(V_t)
+    for t in range(V_t):
+        o = oracle.verify(zt[None, None].repeat(2, 1), zd[None, None], id_map, np.array([[x0]], np.int32),
+                          np.ones(1, np.float32), np.array([[0.999999, 0.5]], np.float32),
+                          probe_token=np.array([t], np.int32))
+        assert o["accepted"][0] == 0
+        r[t] = o["probe_w"][0]
+    assert abs(r.sum() - 1) < 1e-12
+    def emitted(proposal):
+        dist = np.zeros(V_t)
+        np.add.at(dist, id_map[inside], proposal[inside] * thr[inside])
+        return dist + (proposal[inside] * (1 - thr[inside])).sum() * r
+    # NB: r is the residual of the one draft position, which is the same for every x (it depends on p, q' only)
+    assert np.abs(emitted(qprime_def(q, id_map)) - p).max() < 1e-12      # drafts from q': lossless
+    assert np.abs(emitted(q) - p).max() > 1e-3                           # drafts from q: not
+
+
+def test_exactly_zero_residual_falls_back_to_the_target_distribution():
+    """Identity map, all logits equal on a power-of-two vocabulary: p = q' = 2^-k and the mass on the
+    intersection is 1, all exactly, so a rejected draft leaves a residual of exactly zero everywhere.
+    Only a draft outside the vocabulary can be rejected there; the oracle must then flag the fall-back
+    and draw from p, i.e. return floor(v * V)."""
+    V = 16
+    K = 2
+    zt = np.zeros((5, K + 1, V), np.float32)
+    zd = np.zeros((5, K, V), np.float32)
+    id_map = np.arange(V, dtype=np.int32)
+    draft = np.array([[V, 0], [-1, 3], [2, V + 5], [1, 2], [7, -9]], np.int32)
+    u = np.array([[0.5, 0.5, 0.30], [0.1, 0.2, 0.99], [0.9, 0.1, 0.0625], [0.3, 0.3, 0.5], [0.999, 0.0, 0.124]], np.float32)
+    o = oracle.verify(zt, zd, id_map, draft, np.ones(5, np.float32), u)
+    assert list(o["accepted"]) == [0, 0, 1, 2, 1]
+    expect_flags = [oracle.FLAG_DRAFT_RANGE | oracle.FLAG_FALLBACK] * 3 + [0, oracle.FLAG_DRAFT_RANGE | oracle.FLAG_FALLBACK]
+    assert list(o["flags"]) == expect_flags
+    assert list(o["next_token"]) == [int(np.floor(float(v) * V)) for v in u[:, K]]
+    assert np.all(o["total"] == 1.0)                   # the sum of sixteen times 2^-4, exactly
 
 
 def test_ragged_draft_counts_equal_truncated_batches():

@@ -3,8 +3,8 @@ allocate device memory when they need it (an inference server whose HBM is alrea
 committed, a decode loop that must not stall on cudaMalloc).
 
 Collected last on purpose: if this addition fails, `pytest -x` has already run everything else.
-The entry point is compared with tli_verify() on two calls in a row -- the second on a different,
-smaller batch, so whatever the first call left in the shared scratch is still there.
+The entry point is compared with tli_verify() and with the CPU oracle on two calls in a row -- the
+second on a different, smaller batch, so whatever the first call left in the shared scratch is still there.
 """
 import ctypes
 import dataclasses
@@ -14,7 +14,7 @@ import pytest
 import torch
 
 from paper_2502_05202_b200 import tli, workload as wl
-from parity_util import to_device
+from parity_util import compare, to_device
 
 pytestmark = pytest.mark.gpu
 
@@ -56,6 +56,8 @@ def test_static_scratch_matches_tli_verify_on_two_calls_in_a_row():
         for k in ("p_draft", "q_draft"):
             np.testing.assert_allclose(got[k], expect[k], rtol=0, atol=1e-5, err_msg=k)
         assert (got["accepted"] >= 0).all() and (got["next_token"] >= 0).all()
+        rep = compare(batch, got)                    # and against the oracle, by the rule of the parity tests
+        assert rep.ok(), str(rep)
     v.close()
 
 
