@@ -86,6 +86,13 @@ struct Params {
     int split_select;    // 1: the CDF inversions run as a kernel of their own
     int seg_vec;         // statistics kernel: 16-byte vectors per segment
     int nst, nsd;        // ... and segments per target / drafter row
+    // vocabulary-sharded calls (all zero otherwise): V_t / V_d above are the widths of this shard's
+    // slices, which hold target ids t_begin .. and drafter ids d_begin ..; map, inv and the mask are
+    // indexed by global ids
+    int t_begin, d_begin;
+    int sh_wd;           // drafter ids per shard (the gathered rows of shard g start at g * sh_stride elements)
+    long long sh_stride;
+    double *tilesum_p;   // tile sums of p beside those of the residual
     int fin_slice;       // cluster kernel: 16-byte vectors of the sampled target row per CTA
     int fin_dvec;        // cluster kernel: 16-byte vectors reserved for the staged drafter row
 };
@@ -662,7 +669,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
 #pragma unroll
                 for (int q = 0; q < CV; ++q) {
                     const int i = q * kSThreads + tid;
-                    bits[q] = (i < nv) ? mask_bits(P.maskbits, rv.first_elem(v0 + i)) : 0u;
+                    bits[q] = (i < nv) ? mask_bits(P.maskbits, rv.first_elem(v0 + i) + P.d_begin) : 0u;
                 }
             }
             uint4 raw[CV];
@@ -696,7 +703,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     int i2 = __shfl_xor_sync(0xffffffffu, best_idx, o);
                     if (b2 > best || (b2 == best && i2 < best_idx)) { best = b2; best_idx = i2; }
                 }
-                px = best; py = __int_as_float(best_idx);
+                px = best; py = __int_as_float(best_idx == INT_MAX ? INT_MAX : best_idx + P.t_begin);     // global id
             } else {
                 // common reference first, then one exact rescale per lane and a plain sum
                 const float c_w = warp_max(c_run);
@@ -968,8 +975,6 @@ __global__ void __launch_bounds__(kThreads) tli_decide_kernel(const Params P) {
 // LEAN: the caller knows that the vector lies wholly inside the row and that its first id is a
 // multiple of four (true for every vector of a tile that is not at an end of an aligned row), which
 // takes the checks and the element-wise loads out of the code.
-// SMEM: zd_row is the shared-memory address (as ld.shared takes it) of element 0 of a staged copy of
-// the drafter row, not a global pointer.
 template <int DT> __device__ __forceinline__ float load_elt_shared(uint32_t row_addr, int i) {
     if (DT == TLI_F32) {
         float v;
@@ -981,9 +986,18 @@ template <int DT> __device__ __forceinline__ float load_elt_shared(uint32_t row_
     return __uint_as_float(static_cast<uint32_t>(h) << 16);
 }
 
-template <int DT, bool LEAN = false, bool SMEM = false>
-__device__ __forceinline__ void vector_weights_from(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
-                                                    const void *zd_row, float (&w)[Elt<DT>::kPerVec]) {
+// Where the drafter logits of row n come from: the row in global memory, a copy of it staged in
+// shared memory (zd_row is then its shared-memory address), or -- vocabulary-sharded calls -- the
+// slices of it gathered from all shards (zd_row is then the slice of shard 0; drafter id x lies
+// x / sh_wd slices further on).
+enum : int { SRC_GLOBAL = 0, SRC_SHARED = 1, SRC_SHARDS = 2 };
+
+// p(t) and q'_T(t) of the elements of one vector of the sampled target row.
+// LEAN: the caller knows that the vector lies wholly inside the row and that the global id of its
+// first element is a multiple of four, which takes the checks and the element-wise loads out.
+template <int DT, bool LEAN, int SRC>
+__device__ __forceinline__ void vector_p_q(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
+                                           const void *zd_row, float (&pt)[Elt<DT>::kPerVec], float (&q)[Elt<DT>::kPerVec]) {
     constexpr int EPV = Elt<DT>::kPerVec;
     float z[EPV];
     unpack<DT>(raw, z);
@@ -991,40 +1005,57 @@ __device__ __forceinline__ void vector_weights_from(const Params &P, const RowSe
 #pragma unroll
     for (int i = 0; i < EPV; ++i) x[i] = -1;
     if (sel.mode == MODE_RESIDUAL) {
-        if (LEAN || (e0 >= 0 && e0 + EPV <= P.V_t && (e0 & 3) == 0)) {
+        const int g0 = e0 + P.t_begin;                         // global target id of the vector's first element
+        if (LEAN || (e0 >= 0 && e0 + EPV <= P.V_t && (g0 & 3) == 0)) {
 #pragma unroll
             for (int i = 0; i < EPV; i += 4) {
-                const int4 q = __ldg(reinterpret_cast<const int4 *>(P.inv + e0 + i));
-                x[i] = q.x; x[i + 1] = q.y; x[i + 2] = q.z; x[i + 3] = q.w;
+                const int4 u = __ldg(reinterpret_cast<const int4 *>(P.inv + g0 + i));
+                x[i] = u.x; x[i + 1] = u.y; x[i + 2] = u.z; x[i + 3] = u.w;
             }
         } else {
 #pragma unroll
             for (int i = 0; i < EPV; ++i) {
                 const int t = e0 + i;
-                x[i] = (t >= 0 && t < P.V_t) ? __ldg(P.inv + t) : -1;
+                x[i] = (t >= 0 && t < P.V_t) ? __ldg(P.inv + g0 + i) : -1;
             }
         }
     }
     const float nct = -sel.c_t, ncd = -sel.c_d;
 #pragma unroll
     for (int i = 0; i < EPV; ++i) {
-        const float et = ex2(__fmaf_rn(z[i], sel.s, nct));
-        float q = 0.f;
+        pt[i] = __fmul_rn(ex2(__fmaf_rn(z[i], sel.s, nct)), sel.rs_t);
+        q[i] = 0.f;
         if (x[i] >= 0) {
-            const float zdv = SMEM ? load_elt_shared<DT>(static_cast<uint32_t>(reinterpret_cast<uintptr_t>(zd_row)), x[i])
-                                   : load_elt<DT>(zd_row, x[i]);
-            q = __fmul_rn(ex2(__fmaf_rn(zdv, sel.s, ncd)), sel.rs_d);
+            float zdv;
+            if (SRC == SRC_SHARED) {
+                zdv = load_elt_shared<DT>(static_cast<uint32_t>(reinterpret_cast<uintptr_t>(zd_row)), x[i]);
+            } else if (SRC == SRC_SHARDS) {
+                const int g = x[i] / P.sh_wd;
+                zdv = load_elt<DT>(zd_row, static_cast<long long>(g) * P.sh_stride + (x[i] - g * P.sh_wd));
+            } else {
+                zdv = load_elt<DT>(zd_row, x[i]);
+            }
+            q[i] = __fmul_rn(ex2(__fmaf_rn(zdv, sel.s, ncd)), sel.rs_d);
         }
-        // p and q' are each rounded before the subtraction, so that equal distributions leave exactly 0
-        w[i] = fmaxf(0.f, __fsub_rn(__fmul_rn(et, sel.rs_t), q));
     }
 }
 
-template <int DT, bool LEAN = false, bool SMEM = false>
+template <int DT, bool LEAN = false, int SRC = SRC_GLOBAL>
+__device__ __forceinline__ void vector_weights_from(const Params &P, const RowSel &sel, const uint4 &raw, int e0,
+                                                    const void *zd_row, float (&w)[Elt<DT>::kPerVec]) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    float pt[EPV], q[EPV];
+    vector_p_q<DT, LEAN, SRC>(P, sel, raw, e0, zd_row, pt, q);
+    // p and q' are each rounded before the subtraction, so that equal distributions leave exactly 0
+#pragma unroll
+    for (int i = 0; i < EPV; ++i) w[i] = fmaxf(0.f, __fsub_rn(pt[i], q[i]));
+}
+
+template <int DT, bool LEAN = false, int SRC = SRC_GLOBAL>
 __device__ __forceinline__ void vector_weights(const Params &P, const RowSel &sel, const RowView<DT> &rt,
                                                const void *zd_row, int v, float (&w)[Elt<DT>::kPerVec]) {
     const uint4 raw = LEAN ? __ldg(rt.vec0 + v) : rt.load(v);
-    vector_weights_from<DT, LEAN, SMEM>(P, sel, raw, rt.first_elem(v), zd_row, w);
+    vector_weights_from<DT, LEAN, SRC>(P, sel, raw, rt.first_elem(v), zd_row, w);
 }
 
 template <int N> __device__ __forceinline__ float ordered_sum(const float (&w)[N]) {
@@ -1043,7 +1074,7 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
     const int nvec = rt.nvec();
     double acc = 0.0;
     const int v_first = tile * kVecPerTile;
-    const bool lean = (rt.head & 3) == 0 && rt.first_elem(v_first) >= 0 &&
+    const bool lean = (rt.head & 3) == 0 && (P.t_begin & 3) == 0 && rt.first_elem(v_first) >= 0 &&
                       rt.first_elem(v_first + kVecPerTile - 1) + EPV <= rt.V;        // the same for the whole CTA
     if (lean) {
 #pragma unroll
@@ -1075,71 +1106,20 @@ __device__ __forceinline__ double tile_weight_sum(const Params &P, const RowSel 
     return tot;
 }
 
-// The CDF inversion for one sequence by one CTA, tile -> vector -> element, from the tile sums in
-// the workspace.  Either the last CTA of the sampling kernel to finish a tile of the sequence runs
-// it, or (large batches) the selection kernel does, one CTA per sequence.
-// KEEP: each thread forms the weights of four consecutive vectors of the chosen tile and keeps them
-// in registers, so that the final walk needs no second trip to memory (the selection kernel, which
-// has the registers); otherwise the vector the target falls into is formed again (inside the
-// sampling kernel, whose 32 registers per thread would spill them).
-template <int DT, bool KEEP = false>
-__device__ void select_sequence(const Params &P, int b, RowSel sel, const RowView<DT> &rt, const void *zd_row) {
+// The last two levels of the CDF inversion by one CTA: the vector of tile T that holds `rem` (the
+// part of v * total that falls into the tile), then the element of that vector.
+// KEEP: each thread forms the weights of four consecutive vectors of the tile and keeps them in
+// registers, so that the final walk needs no second trip to memory (kernels that have the
+// registers); otherwise the vector the target falls into is formed again (inside the sampling
+// kernel, whose 32 registers per thread would spill them).
+template <int DT, bool KEEP, int SRC>
+__device__ void walk_tile(const Params &P, int b, const RowSel &sel, const RowView<DT> &rt, const void *zd_row,
+                          int T, double rem) {
     constexpr int EPV = Elt<DT>::kPerVec;
-    __shared__ double sm_red[kWarps];
-    __shared__ double sm_tiles[kMaxTiles];
     __shared__ float sm_seg[kVecPerTile];
     __shared__ double sm_warp_tot[kWarps];
-    __shared__ int sm_tile, sm_found, sm_lastpos, sm_retry;
-    __shared__ double sm_rem;
+    __shared__ int sm_found, sm_lastpos;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int ntile = P.ntile;
-    // ---- last CTA of the sequence: invert the CDF, tile -> vector -> element ----
-    for (int i = tid; i < ntile; i += kThreads) sm_tiles[i] = __ldcg(P.tilesum + static_cast<size_t>(b) * ntile + i);
-    __syncthreads();
-    for (int attempt = 0; attempt < 2; ++attempt) {
-        if (tid == 0) {
-            double R = 0.0;
-            for (int i = 0; i < ntile; ++i) R += sm_tiles[i];
-            sm_retry = 0;
-            if (!(R > 0.0) || !isfinite(R)) {
-                sm_retry = 1;
-            } else {
-                const double target = static_cast<double>(sel.v) * R;
-                double run = 0.0;
-                int T = -1, lastpos = 0;
-                double before = 0.0;
-                for (int i = 0; i < ntile; ++i) {
-                    const double nx = run + sm_tiles[i];
-                    if (sm_tiles[i] > 0.0) lastpos = i;
-                    if (T < 0 && nx > target) { T = i; before = run; }
-                    run = nx;
-                }
-                if (T < 0) { T = lastpos; before = R - sm_tiles[lastpos]; }
-                sm_tile = T;
-                sm_rem = target - before;
-            }
-        }
-        __syncthreads();
-        if (!sm_retry) break;
-        if (attempt == 1) {                      // no usable mass even from p: give up on the row
-            if (tid == 0) {
-                P.next_token[b] = 0;
-                if (P.status) P.status[b] |= TLI_ROW_NONFINITE;
-            }
-            return;
-        }
-        // zero residual mass: sample from p of the same position instead
-        sel.mode = MODE_TARGET_ONLY;
-        if (tid == 0 && P.status) P.status[b] |= TLI_ROW_FALLBACK;
-        for (int i = 0; i < ntile; ++i) {
-            const double t2 = tile_weight_sum<DT>(P, sel, rt, zd_row, i, sm_red);
-            if (tid == 0) sm_tiles[i] = t2;
-        }
-        __syncthreads();
-    }
-
-    const int T = sm_tile;
-    const double rem = sm_rem;
     const int nvec = rt.nvec();
     // vector sums of tile T; thread i owns vectors 4i .. 4i+3 in the block-wide exclusive prefix (fp64)
     float wv[KEEP ? kVecPerThread : 1][EPV];
@@ -1151,7 +1131,7 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
             const int v = T * kVecPerTile + tid * kVecPerThread + k;
             float sseg = 0.f;
             if (v < nvec) {
-                vector_weights<DT>(P, sel, rt, zd_row, v, wv[k]);
+                vector_weights<DT, false, SRC>(P, sel, rt, zd_row, v, wv[k]);
                 sseg = ordered_sum(wv[k]);
             } else {
 #pragma unroll
@@ -1168,7 +1148,7 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
             float sseg = 0.f;
             if (v < nvec) {
                 float w[EPV];
-                vector_weights<DT>(P, sel, rt, zd_row, v, w);
+                vector_weights<DT, false, SRC>(P, sel, rt, zd_row, v, w);
                 sseg = ordered_sum(w);
             }
             sm_seg[g] = sseg;
@@ -1226,7 +1206,7 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
                     for (int i = 0; i < EPV; ++i) w[i] = wv[k][i];
                 }
         } else {
-            vector_weights<DT>(P, sel, rt, zd_row, v, w);
+            vector_weights<DT, false, SRC>(P, sel, rt, zd_row, v, w);
         }
         float runf = 0.f;
         int pick = -1, lastw = 0;
@@ -1239,8 +1219,67 @@ __device__ void select_sequence(const Params &P, int b, RowSel sel, const RowVie
         if (pick < 0) pick = lastw;
         int token = rt.first_elem(v) + pick;
         token = min(max(token, 0), P.V_t - 1);
-        P.next_token[b] = token;
+        P.next_token[b] = token + P.t_begin;
     }
+}
+
+// The CDF inversion for one sequence by one CTA, tile -> vector -> element, from the tile sums in
+// the workspace.  Either the last CTA of the sampling kernel to finish a tile of the sequence runs
+// it, or (large batches) the selection kernel does, one CTA per sequence.
+template <int DT, bool KEEP = false>
+__device__ void select_sequence(const Params &P, int b, RowSel sel, const RowView<DT> &rt, const void *zd_row) {
+    __shared__ double sm_red[kWarps];
+    __shared__ double sm_tiles[kMaxTiles];
+    __shared__ int sm_tile, sm_retry;
+    __shared__ double sm_rem;
+    const int tid = threadIdx.x;
+    const int ntile = P.ntile;
+    // ---- last CTA of the sequence: invert the CDF, tile -> vector -> element ----
+    for (int i = tid; i < ntile; i += kThreads) sm_tiles[i] = __ldcg(P.tilesum + static_cast<size_t>(b) * ntile + i);
+    __syncthreads();
+    for (int attempt = 0; attempt < 2; ++attempt) {
+        if (tid == 0) {
+            double R = 0.0;
+            for (int i = 0; i < ntile; ++i) R += sm_tiles[i];
+            sm_retry = 0;
+            if (!(R > 0.0) || !isfinite(R)) {
+                sm_retry = 1;
+            } else {
+                const double target = static_cast<double>(sel.v) * R;
+                double run = 0.0;
+                int T = -1, lastpos = 0;
+                double before = 0.0;
+                for (int i = 0; i < ntile; ++i) {
+                    const double nx = run + sm_tiles[i];
+                    if (sm_tiles[i] > 0.0) lastpos = i;
+                    if (T < 0 && nx > target) { T = i; before = run; }
+                    run = nx;
+                }
+                if (T < 0) { T = lastpos; before = R - sm_tiles[lastpos]; }
+                sm_tile = T;
+                sm_rem = target - before;
+            }
+        }
+        __syncthreads();
+        if (!sm_retry) break;
+        if (attempt == 1) {                      // no usable mass even from p: give up on the row
+            if (tid == 0) {
+                P.next_token[b] = 0;
+                if (P.status) P.status[b] |= TLI_ROW_NONFINITE;
+            }
+            return;
+        }
+        // zero residual mass: sample from p of the same position instead
+        sel.mode = MODE_TARGET_ONLY;
+        if (tid == 0 && P.status) P.status[b] |= TLI_ROW_FALLBACK;
+        for (int i = 0; i < ntile; ++i) {
+            const double t2 = tile_weight_sum<DT>(P, sel, rt, zd_row, i, sm_red);
+            if (tid == 0) sm_tiles[i] = t2;
+        }
+        __syncthreads();
+    }
+
+    walk_tile<DT, KEEP, SRC_GLOBAL>(P, b, sel, rt, zd_row, sm_tile, sm_rem);
 }
 
 // The sampling pass: one CTA per 16 KB tile of the target row the extra token is drawn from
@@ -1398,13 +1437,13 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
 #pragma unroll 2
             for (int i = tid; i < count; i += kFinThreads) {
                 float w[EPV];
-                vector_weights<DT, true, true>(P, sel, rt, zd_arg, v_begin + i, w);
+                vector_weights<DT, true, SRC_SHARED>(P, sel, rt, zd_arg, v_begin + i, w);
                 vsum[i] = ordered_sum(w);
             }
         } else {
             for (int i = tid; i < count; i += kFinThreads) {
                 float w[EPV];
-                vector_weights<DT, false, true>(P, sel, rt, zd_arg, v_begin + i, w);
+                vector_weights<DT, false, SRC_SHARED>(P, sel, rt, zd_arg, v_begin + i, w);
                 vsum[i] = ordered_sum(w);
             }
         }
@@ -1488,8 +1527,8 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
             // when rounding left no vector above the target, take the last positive element instead
             const double rem2 = (found != INT_MAX) ? (rem - cand_before) : INFINITY;
             float w[EPV];
-            if (lean) vector_weights<DT, true, true>(P, sel, rt, zd_arg, v_begin + G, w);
-            else vector_weights<DT, false, true>(P, sel, rt, zd_arg, v_begin + G, w);
+            if (lean) vector_weights<DT, true, SRC_SHARED>(P, sel, rt, zd_arg, v_begin + G, w);
+            else vector_weights<DT, false, SRC_SHARED>(P, sel, rt, zd_arg, v_begin + G, w);
             float runf = 0.f;
             int pick = -1, lastw = 0;
 #pragma unroll
@@ -2520,6 +2559,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
         return TLI_ERR_WORKSPACE;
 
     Params P;
+    memset(&P, 0, sizeof P);
     P.B = a->B; P.K = a->K; P.V_t = ctx->V_t; P.V_d = ctx->V_d;
     P.zt = a->target_logits; P.t_sb = a->t_stride_b; P.t_sk = a->t_stride_k;
     P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sk = a->d_stride_k;
