@@ -63,6 +63,7 @@ enum {
 #define TLI_MAX_B 65535    /* sequences per call */
 #define TLI_MAX_K 64       /* drafts per sequence */
 #define TLI_MAX_V 1048576  /* vocabulary size (either side) */
+#define TLI_MAX_SHARDS 64   /* vocabulary shards (tli_shard_create) */
 #define TLI_STATIC_SCRATCH_BYTES 4194304 /* 4 MiB: scratch built into the library for tli_verify_static() */
 
 /*
@@ -368,6 +369,61 @@ size_t tli_rates_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32
  * allocates nothing, uses the context's counters.
  */
 int tli_acceptance_rates(tli_ctx *ctx, const tli_rates_args *args, void *cuda_stream);
+
+/*
+ * Vocabulary-sharded verification: the same Algorithm 4 + Algorithm 5 step when
+ * the logits come from tensor-parallel LM heads, each of G devices holding one
+ * slice of every target row and one slice of every drafter row.  Algorithm 4's
+ * denominator (the drafter mass on the intersection) and Algorithm 5's residual
+ * normaliser are the two sums that cross shards; their partial values are
+ * exchanged by the caller (one all-gather each) between four local calls, and
+ * so is, for every sequence that rejected a draft, the one drafter row the
+ * residual is formed from (a mapped pair may have its drafter id on one shard
+ * and its target id on another).
+ *
+ * Partition: shard g of G holds target ids [g*Wt, min(V_t, (g+1)*Wt)) with
+ * Wt = ceil(V_t / G), and drafter ids [g*Wd, ...) with Wd = ceil(V_d / G)
+ * (tli_shard_info() reports them; trailing shards may hold fewer ids, or none).
+ * The id map is the global one (drafter id -> target id).  draft_ids,
+ * temperature and uniforms are replicated.
+ *
+ * One verification, on every shard, with `args` as for tli_verify() except that
+ * target_logits / drafter_logits are this shard's slices ([B, K+1, >= its target
+ * ids] / [B, K, >= its drafter ids], strides as given), workspace is at least
+ * tli_shard_workspace_bytes(), and draft_lengths must be NULL:
+ *
+ *   tli_shard_stats(ctx, args, record)            record: tli_shard_record_bytes()
+ *       all-gather the records            -> records_all [G][record]
+ *   tli_shard_decide(ctx, args, records_all, rows)  rows: tli_shard_rows_bytes()
+ *       writes accepted, row_status, p_draft, q_draft (identical on every shard),
+ *       next_token of the sequences that need no sample, and this shard's slice
+ *       of drafter row n of every sequence that rejected a draft
+ *       all-gather the rows               -> rows_all [G][rows]
+ *   tli_shard_weights(ctx, args, rows_all, mass)    mass: double[B][2]
+ *       all-gather the masses             -> masses_all [G][B][2]
+ *   tli_shard_select(ctx, args, rows_all, masses_all)
+ *       next_token[b] = the sampled global target id on the one shard that holds
+ *       it, -1 on the others: combine with an element-wise maximum over shards
+ *       (sequences finished by tli_shard_decide carry the same value everywhere).
+ *
+ * All buffers are [device], 16-byte aligned; the gathered ones are the shards'
+ * buffers in shard order.  Every call is asynchronous on the stream, allocates
+ * nothing and touches local memory only; the all-gathers are the caller's (NCCL
+ * or any other transport).  Results equal tli_verify()'s on the unsharded
+ * tensors up to the order in which sums are formed.  A context made here serves
+ * these calls only (tli_verify() refuses it).
+ */
+int tli_shard_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_t *id_map_host,
+                     int32_t n_shards, int32_t shard);
+int tli_shard_info(const tli_ctx *ctx, int32_t *t_begin, int32_t *t_count, int32_t *d_begin, int32_t *d_count,
+                   int32_t *t_width, int32_t *d_width);
+size_t tli_shard_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype);
+size_t tli_shard_record_bytes(const tli_ctx *ctx, int32_t B, int32_t K);
+size_t tli_shard_rows_bytes(const tli_ctx *ctx, int32_t B, int32_t dtype);
+int tli_shard_stats(tli_ctx *ctx, const tli_verify_args *args, void *record_out, void *cuda_stream);
+int tli_shard_decide(tli_ctx *ctx, const tli_verify_args *args, const void *records_all, void *rows_out, void *cuda_stream);
+int tli_shard_weights(tli_ctx *ctx, const tli_verify_args *args, const void *rows_all, void *mass_out, void *cuda_stream);
+int tli_shard_select(tli_ctx *ctx, const tli_verify_args *args, const void *rows_all, const void *masses_all, void *cuda_stream);
 
 /*
  * Measurement hook: tli_verify() with CUDA events recorded on `cuda_stream`

@@ -2315,6 +2315,387 @@ __global__ void __launch_bounds__(kThreads, 6) tli_rate_pairs_kernel(const RateP
     if (P.status) P.status[pair] = status;
 }
 
+// ---------------------------------------------------------------------------
+// vocabulary-sharded verification (the logits of a tensor-parallel LM head)
+// ---------------------------------------------------------------------------
+//
+// Every shard holds a slice of each target row and of each drafter row.  Algorithm 4's
+// denominator (the sum over the intersection) and Algorithm 5's residual normaliser are the two
+// sums that cross shards; everything else is local:
+//   statistics   the statistics kernel on the slices, then one record per sequence: (reference,
+//                sum) of each of its 2K+1 rows over this shard's ids, and the logits of the drafted
+//                tokens that this shard owns.                         -> exchanged (all-gather)
+//   decision     every shard folds the records of all shards (exact powers of two, fp64) and takes
+//                Algorithm 5's decisions: the same on every shard.  It then packs its slice of
+//                drafter row n of every sequence that rejected a draft.  -> exchanged (all-gather)
+//   weights      tile sums of max(0, p - q'_T) and of p over this shard's target ids, q' read from
+//                the gathered drafter row, and their totals.              -> exchanged (all-gather)
+//   selection    every shard adds the totals in shard order; the shard that holds v * total walks
+//                its tiles, the others report -1.                    -> combined (maximum)
+// The exchanges are the caller's (NCCL through torch.distributed); these kernels read and write
+// local memory only.
+
+// doubles per sequence of one shard's record: (reference | max, sum | arg-max) per row, then the
+// target and the drafter logit of every drafted token (0 where another shard owns it)
+__host__ __device__ inline int shard_record_len(int K) { return 2 * (2 * K + 1) + 2 * K; }
+
+struct ShardParams {
+    Params P;
+    int G, g;            // shards, this shard
+    int wt, wd;          // target / drafter ids per shard (the last shards may hold fewer, or none)
+    int V_t_all, V_d_all;
+    double *record;            // this shard's record [B][shard_record_len(K)]
+    const double *records;     // all shards' records [G][B][shard_record_len(K)]
+    void *rows_out;            // this shard's slices of drafter row n [B][row_pitch elements]
+    const void *rows_all;      // all shards' [G][B][row_pitch]
+    int row_pitch;
+    double *mass;              // this shard's totals [B][2]: residual, p
+    const double *masses;      // all shards' [G][B][2]
+};
+
+// One CTA per sequence: the shard's segment partials folded per row into its record, and the
+// logits of the drafted tokens that live on this shard.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_shard_fold_kernel(const ShardParams S) {
+    const Params &P = S.P;
+    const int b = blockIdx.x, tid = threadIdx.x, K = P.K;
+    const float tau = __ldg(P.tau + b);
+    double *rec = S.record + static_cast<size_t>(b) * shard_record_len(K);
+    const bool bad = !(tau >= 0.f) || isinf(tau);
+    const bool greedy = (tau == 0.f);
+    if (tid < K) {                                   // the drafted tokens this shard owns
+        double zt = 0.0, zd = 0.0;
+        const int x = __ldg(P.draft + static_cast<size_t>(b) * K + tid);
+        if (!bad && !greedy && x >= 0 && x < S.V_d_all) {
+            const int t = __ldg(P.map + x);
+            if (t >= P.t_begin && t < P.t_begin + P.V_t)
+                zt = load_elt<DT>(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(tid) * P.t_sk + (t - P.t_begin));
+            if (t >= 0 && x >= P.d_begin && x < P.d_begin + P.V_d)
+                zd = load_elt<DT>(P.zd, static_cast<long long>(b) * P.d_sb + static_cast<long long>(tid) * P.d_sk + (x - P.d_begin));
+        }
+        rec[2 * (2 * K + 1) + tid] = zt;
+        rec[2 * (2 * K + 1) + K + tid] = zd;
+    }
+    const int nrows = 2 * K + 1;
+    for (int r0 = 0; r0 < nrows; r0 += kThreads / 8) {
+        const int r = r0 + (tid >> 3);
+        const int sub = tid & 7;
+        const bool is_t = r <= K;
+        const bool mine = r < nrows && !bad && !(greedy && !is_t);
+        const int nseg = !mine ? 0 : (is_t ? P.nst : P.nsd);
+        const float2 *part = is_t ? P.part_t + (static_cast<size_t>(b) * (K + 1) + r) * P.nst
+                                  : P.part_d + (static_cast<size_t>(b) * K + (r - K - 1)) * P.nsd;
+        if (greedy) {
+            float best = -INFINITY; int idx = INT_MAX;
+            for (int i = sub; i < nseg; i += 8) {
+                float2 pr = __ldcg(part + i);
+                int i2 = __float_as_int(pr.y);
+                if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                float b2 = __shfl_xor_sync(0xffffffffu, best, o);
+                int i2 = __shfl_xor_sync(0xffffffffu, idx, o);
+                if (b2 > best || (b2 == best && i2 < idx)) { best = b2; idx = i2; }
+            }
+            if (sub == 0 && r < nrows) { rec[2 * r] = static_cast<double>(best); rec[2 * r + 1] = static_cast<double>(idx); }
+        } else {
+            float c = kNegBig;
+            double sum = 0.0;
+            for (int i = sub; i < nseg; i += 8) {
+                const float2 pr = __ldcg(part + i);
+                const float cn = fmaxf(c, pr.x);
+                sum = sum * pow2_neg_d(c - cn) + static_cast<double>(pr.y) * pow2_neg_d(pr.x - cn);
+                c = cn;
+            }
+#pragma unroll
+            for (int o = 4; o > 0; o >>= 1) {
+                const float c2 = __shfl_xor_sync(0xffffffffu, c, o);
+                const double s2 = __shfl_xor_sync(0xffffffffu, sum, o);
+                const float cn = fmaxf(c, c2);
+                sum = sum * pow2_neg_d(c - cn) + s2 * pow2_neg_d(c2 - cn);
+                c = cn;
+            }
+            if (sub == 0 && r < nrows) { rec[2 * r] = static_cast<double>(c); rec[2 * r + 1] = sum; }
+        }
+    }
+}
+
+// One CTA per sequence, the same on every shard: the records of all shards folded in shard order,
+// Algorithm 5's acceptance tests and count, the hand-over to the weights pass.
+__global__ void __launch_bounds__(128) tli_shard_decide_kernel(const ShardParams S) {
+    const Params &P = S.P;
+    const int b = blockIdx.x, tid = threadIdx.x, K = P.K, G = S.G;
+    const int len = shard_record_len(K);
+    __shared__ double sm_c[2 * TLI_MAX_K + 1], sm_s[2 * TLI_MAX_K + 1];
+    __shared__ int sm_accept[TLI_MAX_K];
+    __shared__ int sm_flags;
+    const float tau = __ldg(P.tau + b);
+    if (tid == 0) sm_flags = 0;
+    if (!(tau >= 0.f) || isinf(tau)) {
+        if (tid == 0) {
+            P.accepted[b] = 0; P.next_token[b] = 0;
+            if (P.status) P.status[b] = TLI_ROW_BAD_TEMPERATURE;
+            RowSel rs = {0, MODE_SKIP, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+            P.sel[b] = rs;
+        }
+        if (tid < K) {
+            if (P.p_out) P.p_out[static_cast<size_t>(b) * K + tid] = 0.f;
+            if (P.q_out) P.q_out[static_cast<size_t>(b) * K + tid] = 0.f;
+        }
+        return;
+    }
+    const bool greedy = (tau == 0.f);
+    const int nrows = greedy ? K + 1 : 2 * K + 1;
+    for (int r = tid; r < nrows; r += blockDim.x) {
+        if (greedy) {
+            double best = -INFINITY, idx = static_cast<double>(INT_MAX);
+            for (int g = 0; g < G; ++g) {
+                const double *rec = S.records + (static_cast<size_t>(g) * P.B + b) * len;
+                const double m = rec[2 * r], i2 = rec[2 * r + 1];
+                if (m > best || (m == best && i2 < idx)) { best = m; idx = i2; }
+            }
+            sm_c[r] = best; sm_s[r] = (idx == static_cast<double>(INT_MAX)) ? 0.0 : idx;
+        } else {
+            double c = static_cast<double>(kNegBig), sum = 0.0;
+            for (int g = 0; g < G; ++g) {
+                const double *rec = S.records + (static_cast<size_t>(g) * P.B + b) * len;
+                const double c2 = rec[2 * r], s2 = rec[2 * r + 1];
+                const double cn = fmax(c, c2);
+                sum = sum * pow2_neg_d(static_cast<float>(c - cn)) + s2 * pow2_neg_d(static_cast<float>(c2 - cn));
+                c = cn;
+            }
+            sm_c[r] = c; sm_s[r] = sum;
+        }
+    }
+    __syncthreads();
+    const float s_f = 1.4426950408889634f / tau;
+    if (tid < K) {
+        const int j = tid;
+        int ok = 0, fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
+        float pv = 0.f, qv = 0.f;
+        const int x = __ldg(P.draft + static_cast<size_t>(b) * K + j);
+        int t = -1;
+        if (x < 0 || x >= S.V_d_all) fl |= TLI_ROW_DRAFT_RANGE;
+        else { t = __ldg(P.map + x); if (t < 0) fl |= TLI_ROW_DRAFT_UNMAPPED; }
+        if (greedy) {
+            ok = (t >= 0 && t == static_cast<int>(sm_s[j]));
+        } else {
+            const double S_t = sm_s[j], S_d = sm_s[K + 1 + j];
+            if (!(S_t > 0.0) || !isfinite(S_t) || !isfinite(S_d)) fl |= TLI_ROW_NONFINITE;
+            else if (t >= 0) {
+                const int gt = t / S.wt, gd = x / S.wd;                   // the shards that own the two logits
+                const double zt = S.records[(static_cast<size_t>(gt) * P.B + b) * len + 2 * (2 * K + 1) + j];
+                const double zd = S.records[(static_cast<size_t>(gd) * P.B + b) * len + 2 * (2 * K + 1) + K + j];
+                const double sd = static_cast<double>(s_f);
+                const double p = exp2(zt * sd - sm_c[j]) / S_t;
+                const double q = (S_d > 0.0) ? exp2(zd * sd - sm_c[K + 1 + j]) / S_d : 0.0;
+                double thr;
+                if (q > 0.0) thr = fmin(1.0, p / q);
+                else thr = (p > 0.0) ? 1.0 : 0.0;
+                ok = static_cast<double>(__ldg(P.u + static_cast<size_t>(b) * (K + 1) + j)) < thr;
+                pv = static_cast<float>(p); qv = static_cast<float>(q);
+            }
+        }
+        sm_accept[j] = ok;
+        if (fl) atomicOr(&sm_flags, fl);
+        if (P.p_out) P.p_out[static_cast<size_t>(b) * K + j] = pv;
+        if (P.q_out) P.q_out[static_cast<size_t>(b) * K + j] = qv;
+    }
+    __syncthreads();
+    if (tid == 0) {
+        int n = K;
+        for (int j = 0; j < K; ++j) if (!sm_accept[j]) { n = j; break; }
+        int fl = sm_flags;
+        if (!greedy) {
+            const double S_n = sm_s[n];
+            if (!(S_n > 0.0) || !isfinite(S_n)) fl |= TLI_ROW_NONFINITE;
+        }
+        RowSel rs;
+        rs.n = n; rs.mode = MODE_SKIP; rs.s = s_f; rs.c_t = 0.f; rs.rs_t = 0.f; rs.c_d = 0.f; rs.rs_d = 0.f;
+        rs.v = __ldg(P.u + static_cast<size_t>(b) * (K + 1) + K);
+        int token = -1;                            // -1: the selection supplies it
+        if (greedy) {
+            token = static_cast<int>(sm_s[n]);
+        } else if (fl & TLI_ROW_NONFINITE) {
+            n = 0; token = 0;
+        } else {
+            rs.c_t = static_cast<float>(sm_c[n]);
+            rs.rs_t = static_cast<float>(1.0 / sm_s[n]);
+            if (n < K) {
+                const double S_d = sm_s[K + 1 + n];
+                rs.mode = MODE_RESIDUAL;
+                rs.c_d = static_cast<float>(sm_c[K + 1 + n]);
+                rs.rs_d = (S_d > 0.0) ? static_cast<float>(1.0 / S_d) : 0.f;
+            } else {
+                rs.mode = MODE_TARGET_ONLY;
+            }
+        }
+        rs.n = n;
+        P.accepted[b] = n;
+        P.next_token[b] = token;
+        if (P.status) P.status[b] = fl;
+        P.sel[b] = rs;
+    }
+}
+
+// This shard's slice of drafter row n of every sequence that rejected a draft, as 16-byte vectors
+// (ids beyond the slice read -inf).  grid (vectors / 256, B).
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_shard_pack_kernel(const ShardParams S) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const Params &P = S.P;
+    const int b = blockIdx.y;
+    const RowSel sel = P.sel[b];
+    if (sel.mode != MODE_RESIDUAL) return;
+    const int v = blockIdx.x * kThreads + threadIdx.x;
+    if (v * EPV >= S.row_pitch) return;
+    const char *row = reinterpret_cast<const char *>(P.zd) +
+        (static_cast<long long>(b) * P.d_sb + static_cast<long long>(sel.n) * P.d_sk) * Elt<DT>::kBytes;
+    uint32_t w[4] = {Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord, Elt<DT>::kNegInfWord};
+    if constexpr (DT == TLI_F32) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int e = v * 4 + i;
+            if (e < P.V_d) w[i] = __ldg(reinterpret_cast<const uint32_t *>(row) + e);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int e = v * 8 + i;
+            if (e < P.V_d) {
+                const uint32_t h = __ldg(reinterpret_cast<const unsigned short *>(row) + e);
+                w[i >> 1] = (i & 1) ? ((w[i >> 1] & 0x0000ffffu) | (h << 16)) : ((w[i >> 1] & 0xffff0000u) | h);
+            }
+        }
+    }
+    uint4 *dst = reinterpret_cast<uint4 *>(reinterpret_cast<char *>(S.rows_out) +
+                                           static_cast<size_t>(b) * S.row_pitch * Elt<DT>::kBytes);
+    dst[v] = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// One CTA per 16 KB tile of this shard's slice of target row n: the sums of max(0, p - q'_T) and
+// of p over the tile (fp32 per vector, fp64 across).  grid (tiles, B).
+template <int DT>
+__global__ void __launch_bounds__(kThreads, 4) tli_shard_weights_kernel(const ShardParams S) {
+    constexpr int EPV = Elt<DT>::kPerVec;
+    const Params &P = S.P;
+    __shared__ double sm_red[2][kWarps];
+    const int b = blockIdx.y, tile = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const RowSel sel = P.sel[b];
+    if (sel.mode == MODE_SKIP) return;
+    const RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_rows = reinterpret_cast<const char *>(S.rows_all) + static_cast<size_t>(b) * S.row_pitch * Elt<DT>::kBytes;
+    const int nvec = rt.nvec();
+    double acc_r = 0.0, acc_p = 0.0;
+#pragma unroll
+    for (int k = 0; k < kVecPerThread; ++k) {
+        const int v = tile * kVecPerTile + k * kThreads + tid;
+        if (v < nvec) {
+            float pt[EPV], q[EPV], w[EPV];
+            vector_p_q<DT, false, SRC_SHARDS>(P, sel, rt.load(v), rt.first_elem(v), zd_rows, pt, q);
+#pragma unroll
+            for (int i = 0; i < EPV; ++i) w[i] = fmaxf(0.f, __fsub_rn(pt[i], q[i]));
+            acc_r += static_cast<double>(ordered_sum(w));
+            acc_p += static_cast<double>(ordered_sum(pt));
+        }
+    }
+    acc_r = warp_sum(acc_r);
+    acc_p = warp_sum(acc_p);
+    if (lane == 0) { sm_red[0][warp] = acc_r; sm_red[1][warp] = acc_p; }
+    __syncthreads();
+    if (tid == 0) {
+        double tr = 0.0, tp = 0.0;
+#pragma unroll
+        for (int i = 0; i < kWarps; ++i) { tr += sm_red[0][i]; tp += sm_red[1][i]; }
+        __stcg(P.tilesum + static_cast<size_t>(b) * P.ntile + tile, tr);
+        __stcg(P.tilesum_p + static_cast<size_t>(b) * P.ntile + tile, tp);
+    }
+}
+
+// One thread per sequence: this shard's totals, tiles added in order.
+__global__ void __launch_bounds__(128) tli_shard_mass_kernel(const ShardParams S) {
+    const Params &P = S.P;
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= P.B) return;
+    double r = 0.0, p = 0.0;
+    if (P.sel[b].mode != MODE_SKIP) {
+        for (int i = 0; i < P.ntile; ++i) {
+            r += __ldcg(P.tilesum + static_cast<size_t>(b) * P.ntile + i);
+            p += __ldcg(P.tilesum_p + static_cast<size_t>(b) * P.ntile + i);
+        }
+    }
+    S.mass[2 * b] = r;
+    S.mass[2 * b + 1] = p;
+}
+
+// One CTA per sequence, the same arithmetic on every shard: the totals of all shards added in
+// shard order, the shard that holds v * total, and on that shard tile -> vector -> element.
+template <int DT>
+__global__ void __launch_bounds__(kThreads) tli_shard_select_kernel(const ShardParams S) {
+    const Params &P = S.P;
+    __shared__ int sm_tile, sm_mode;
+    __shared__ double sm_rem;
+    const int b = blockIdx.x, tid = threadIdx.x;
+    RowSel sel = P.sel[b];
+    if (sel.mode == MODE_SKIP) return;                   // decided and finished by the decision kernel
+    if (tid == 0) {
+        int kind = (sel.mode == MODE_RESIDUAL) ? 0 : 1;  // which totals: residual, or p
+        double R = 0.0;
+        for (int g = 0; g < S.G; ++g) R += S.masses[(static_cast<size_t>(g) * P.B + b) * 2 + kind];
+        int fl = 0;
+        if (kind == 0 && (!(R > 0.0) || !isfinite(R))) {  // zero residual mass: sample from p of the same position
+            kind = 1; fl |= TLI_ROW_FALLBACK;
+            R = 0.0;
+            for (int g = 0; g < S.G; ++g) R += S.masses[(static_cast<size_t>(g) * P.B + b) * 2 + 1];
+        }
+        sm_mode = -1;
+        if (!(R > 0.0) || !isfinite(R)) {                // no usable mass even from p: give up on the row
+            P.next_token[b] = 0;
+            fl |= TLI_ROW_NONFINITE;
+        } else {
+            const double target = static_cast<double>(sel.v) * R;
+            int owner = -1, lastpos = 0;
+            double before = 0.0, run = 0.0;
+            for (int g = 0; g < S.G; ++g) {
+                const double m = S.masses[(static_cast<size_t>(g) * P.B + b) * 2 + kind];
+                const double nx = run + m;
+                if (m > 0.0) lastpos = g;
+                if (owner < 0 && nx > target) { owner = g; before = run; }
+                run = nx;
+            }
+            if (owner < 0) { owner = lastpos; before = R - S.masses[(static_cast<size_t>(lastpos) * P.B + b) * 2 + kind]; }
+            if (owner == S.g) {
+                // this shard: which of its tiles
+                const double *tiles = (kind == 0 ? P.tilesum : P.tilesum_p) + static_cast<size_t>(b) * P.ntile;
+                const double rem = target - before;
+                double run_t = 0.0, before_t = 0.0;
+                int T = -1, last_t = 0;
+                for (int i = 0; i < P.ntile; ++i) {
+                    const double m = __ldcg(tiles + i);
+                    const double nx = run_t + m;
+                    if (m > 0.0) last_t = i;
+                    if (T < 0 && nx > rem) { T = i; before_t = run_t; }
+                    run_t = nx;
+                }
+                if (T < 0) { T = last_t; before_t = run_t - __ldcg(tiles + last_t); }
+                sm_tile = T;
+                sm_rem = rem - before_t;
+                sm_mode = (kind == 0) ? MODE_RESIDUAL : MODE_TARGET_ONLY;
+            } else {
+                P.next_token[b] = -1;                    // another shard reports it
+            }
+        }
+        if (fl && P.status) P.status[b] |= fl;
+    }
+    __syncthreads();
+    if (sm_mode < 0) return;
+    sel.mode = sm_mode;
+    const RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
+    const void *zd_rows = reinterpret_cast<const char *>(S.rows_all) + static_cast<size_t>(b) * S.row_pitch * Elt<DT>::kBytes;
+    walk_tile<DT, true, SRC_SHARDS>(P, b, sel, rt, zd_rows, sm_tile, sm_rem);
+}
+
 // Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete,
 // with a caller-chosen poll limit, and reports how the wait ended.  The kernel returns normally.
 __global__ void tli_bounded_wait_kernel(unsigned limit, int *result, unsigned *scratch_error) {
@@ -2450,7 +2831,27 @@ struct tli_ctx {
     unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
+    // vocabulary-sharded contexts (tli_shard_create); one shard holding everything otherwise
+    int n_shards, shard;
+    int32_t wt, wd;             // ids per shard
+    int32_t t_begin, t_count, d_begin, d_count;
 };
+
+namespace {
+
+cudaError_t launch_stats(const Params &P, const Layout &L, int dtype, cudaStream_t stream) {
+    const dim3 g1(L.grid), b1(kSThreads + 32);
+#define TLI_LAUNCH_STATS(DT, CV) tli_stats_kernel<DT, CV><<<g1, b1, kStatsSmemBytes, stream>>>(P)
+    if (dtype == TLI_F32) {
+        if (L.cv == 4) TLI_LAUNCH_STATS(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_F32, 2); else TLI_LAUNCH_STATS(TLI_F32, 1);
+    } else {
+        if (L.cv == 4) TLI_LAUNCH_STATS(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_BF16, 2); else TLI_LAUNCH_STATS(TLI_BF16, 1);
+    }
+#undef TLI_LAUNCH_STATS
+    return cudaGetLastError();
+}
+
+}  // namespace
 
 extern "C" {
 
@@ -2484,6 +2885,8 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
     c->tiled = 0;
+    c->n_shards = 1; c->shard = 0; c->wt = V_t; c->wd = V_d;
+    c->t_begin = 0; c->t_count = V_t; c->d_begin = 0; c->d_count = V_d;
     int rc = TLI_OK;
     do {
         if ((e = cudaDeviceGetAttribute(&c->num_sms, cudaDevAttrMultiProcessorCount, device)) != cudaSuccess) { rc = cuda_fail(e, "cudaDeviceGetAttribute"); break; }
@@ -2543,6 +2946,7 @@ int tli_ctx_info(const tli_ctx *ctx, int32_t *V_t, int32_t *V_d, int32_t *n_mapp
 
 static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, cudaEvent_t *ev) {
     if (!ctx || !a) return TLI_ERR_ARG;
+    if (ctx->n_shards != 1) return TLI_ERR_ARG;                 // a shard's context serves the tli_shard_* calls only
     if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
     if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
     if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
@@ -2586,17 +2990,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
     const dim3 grid2(static_cast<unsigned>(L.ntile), static_cast<unsigned>(a->B));
-    {
-        const dim3 g1(L.grid), b1(kSThreads + 32);
-#define TLI_LAUNCH_STATS(DT, CV) tli_stats_kernel<DT, CV><<<g1, b1, kStatsSmemBytes, stream>>>(P)
-        if (a->dtype == TLI_F32) {
-            if (L.cv == 4) TLI_LAUNCH_STATS(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_F32, 2); else TLI_LAUNCH_STATS(TLI_F32, 1);
-        } else {
-            if (L.cv == 4) TLI_LAUNCH_STATS(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_BF16, 2); else TLI_LAUNCH_STATS(TLI_BF16, 1);
-        }
-#undef TLI_LAUNCH_STATS
-    }
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e = launch_stats(P, L, a->dtype, stream);
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
     if (ev) cudaEventRecord(ev[1], stream);
 
@@ -2765,6 +3159,187 @@ int tli_slem_verify(tli_ctx *ctx, const tli_slem_args *a, void *cuda_stream) {
     const cudaError_t e = cudaLaunchKernelEx(&cfg, tli_slem_match_kernel, Q);
     if (e != cudaSuccess) return cuda_fail(e, "launch tli_slem_match_kernel");
     return TLI_OK;
+}
+
+// ---- vocabulary-sharded verification ----
+
+namespace {
+
+struct ShardLayout { Layout L; size_t tilesum_p, total; int row_pitch; };
+
+ShardLayout make_shard_layout(const tli_ctx *ctx, int B, int K, int dtype) {
+    ShardLayout SL;
+    SL.L = make_layout(B, K, ctx->t_count, ctx->d_count, dtype, ctx->num_sms);
+    SL.tilesum_p = SL.L.total;
+    SL.total = align_up(SL.tilesum_p + sizeof(double) * static_cast<size_t>(B) * SL.L.ntile, 256);
+    const int epv = dtype == TLI_F32 ? 4 : 8;
+    SL.row_pitch = (ctx->wd + epv - 1) / epv * epv;
+    return SL;
+}
+
+// Argument checks and kernel parameters shared by the four sharded calls.
+int shard_params(tli_ctx *ctx, const tli_verify_args *a, ShardParams &S, ShardLayout &SL) {
+    if (!ctx || !a) return TLI_ERR_ARG;
+    if (a->B < 1 || a->K < 1) return TLI_ERR_ARG;
+    if (a->B > TLI_MAX_B || a->K > TLI_MAX_K) return TLI_ERR_UNSUPPORTED;
+    if (a->dtype != TLI_F32 && a->dtype != TLI_BF16) return TLI_ERR_ARG;
+    if (!a->target_logits || !a->drafter_logits || !a->draft_ids || !a->temperature || !a->uniforms ||
+        !a->accepted || !a->next_token)
+        return TLI_ERR_ARG;
+    const size_t elt = a->dtype == TLI_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
+        return TLI_ERR_ARG;
+    if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
+    if (a->draft_lengths) return TLI_ERR_UNSUPPORTED;
+    SL = make_shard_layout(ctx, a->B, a->K, a->dtype);
+    if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < SL.total)
+        return TLI_ERR_WORKSPACE;
+    memset(&S, 0, sizeof S);
+    Params &P = S.P;
+    const Layout &L = SL.L;
+    P.B = a->B; P.K = a->K; P.V_t = ctx->t_count; P.V_d = ctx->d_count;
+    P.zt = a->target_logits; P.t_sb = a->t_stride_b; P.t_sk = a->t_stride_k;
+    P.zd = a->drafter_logits; P.d_sb = a->d_stride_b; P.d_sk = a->d_stride_k;
+    P.map = ctx->d_map; P.inv = ctx->d_inv; P.maskbits = ctx->d_mask; P.n_mapped = ctx->n_mapped;
+    P.draft = a->draft_ids; P.tau = a->temperature; P.u = a->uniforms;
+    P.accepted = a->accepted; P.next_token = a->next_token; P.status = a->row_status;
+    P.p_out = a->p_draft; P.q_out = a->q_draft;
+    char *ws = reinterpret_cast<char *>(a->workspace);
+    P.part_t = reinterpret_cast<float2 *>(ws + L.part_t);
+    P.part_d = reinterpret_cast<float2 *>(ws + L.part_d);
+    P.sel = reinterpret_cast<RowSel *>(ws + L.sel);
+    P.tilesum = reinterpret_cast<double *>(ws + L.tilesum);
+    P.tilesum_p = reinterpret_cast<double *>(ws + SL.tilesum_p);
+    P.cnt_stats = ctx->d_counters;
+    P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
+    P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
+    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
+    P.ntile = L.ntile;
+    P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
+    P.t_begin = ctx->t_begin; P.d_begin = ctx->d_begin;
+    P.sh_wd = ctx->wd; P.sh_stride = static_cast<long long>(a->B) * SL.row_pitch;
+    S.G = ctx->n_shards; S.g = ctx->shard; S.wt = ctx->wt; S.wd = ctx->wd;
+    S.V_t_all = ctx->V_t; S.V_d_all = ctx->V_d;
+    S.row_pitch = SL.row_pitch;
+    return TLI_OK;
+}
+
+}  // namespace
+
+int tli_shard_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_t *id_map_host,
+                     int32_t n_shards, int32_t shard) {
+    if (out) *out = nullptr;
+    if (n_shards < 1 || n_shards > TLI_MAX_SHARDS || shard < 0 || shard >= n_shards) return TLI_ERR_ARG;
+    const int rc = tli_create(out, device, V_t, V_d, id_map_host);
+    if (rc != TLI_OK) return rc;
+    tli_ctx *c = *out;
+    c->n_shards = n_shards; c->shard = shard;
+    c->wt = (V_t + n_shards - 1) / n_shards;
+    c->wd = (V_d + n_shards - 1) / n_shards;
+    auto clip = [](long long x, int32_t hi) { return static_cast<int32_t>(x < hi ? x : hi); };
+    c->t_begin = clip(static_cast<long long>(shard) * c->wt, V_t);
+    c->t_count = clip(static_cast<long long>(shard + 1) * c->wt, V_t) - c->t_begin;
+    c->d_begin = clip(static_cast<long long>(shard) * c->wd, V_d);
+    c->d_count = clip(static_cast<long long>(shard + 1) * c->wd, V_d) - c->d_begin;
+    return TLI_OK;
+}
+
+int tli_shard_info(const tli_ctx *ctx, int32_t *t_begin, int32_t *t_count, int32_t *d_begin, int32_t *d_count,
+                   int32_t *t_width, int32_t *d_width) {
+    if (!ctx) return TLI_ERR_ARG;
+    if (t_begin) *t_begin = ctx->t_begin;
+    if (t_count) *t_count = ctx->t_count;
+    if (d_begin) *d_begin = ctx->d_begin;
+    if (d_count) *d_count = ctx->d_count;
+    if (t_width) *t_width = ctx->wt;
+    if (d_width) *d_width = ctx->wd;
+    return TLI_OK;
+}
+
+size_t tli_shard_workspace_bytes(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype) {
+    if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return 0;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return 0;
+    return make_shard_layout(ctx, B, K, dtype).total;
+}
+
+size_t tli_shard_record_bytes(const tli_ctx *ctx, int32_t B, int32_t K) {
+    if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return 0;
+    return sizeof(double) * static_cast<size_t>(B) * shard_record_len(K);
+}
+
+size_t tli_shard_rows_bytes(const tli_ctx *ctx, int32_t B, int32_t dtype) {
+    if (!ctx || B < 1 || B > TLI_MAX_B || (dtype != TLI_F32 && dtype != TLI_BF16)) return 0;
+    const size_t epv = dtype == TLI_F32 ? 4 : 8;
+    return static_cast<size_t>(B) * ((ctx->wd + epv - 1) / epv) * 16;
+}
+
+int tli_shard_stats(tli_ctx *ctx, const tli_verify_args *a, void *record_out, void *cuda_stream) {
+    ShardParams S; ShardLayout SL;
+    const int rc = shard_params(ctx, a, S, SL);
+    if (rc != TLI_OK) return rc;
+    if (!record_out || reinterpret_cast<uintptr_t>(record_out) % 8) return TLI_ERR_ARG;
+    S.record = reinterpret_cast<double *>(record_out);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    cudaError_t e = launch_stats(S.P, SL.L, a->dtype, stream);
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_stats_kernel");
+    if (a->dtype == TLI_F32) tli_shard_fold_kernel<TLI_F32><<<a->B, kThreads, 0, stream>>>(S);
+    else tli_shard_fold_kernel<TLI_BF16><<<a->B, kThreads, 0, stream>>>(S);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "launch tli_shard_fold_kernel");
+}
+
+int tli_shard_decide(tli_ctx *ctx, const tli_verify_args *a, const void *records_all, void *rows_out, void *cuda_stream) {
+    ShardParams S; ShardLayout SL;
+    const int rc = shard_params(ctx, a, S, SL);
+    if (rc != TLI_OK) return rc;
+    if (!records_all || !rows_out || reinterpret_cast<uintptr_t>(records_all) % 8 || reinterpret_cast<uintptr_t>(rows_out) % 16)
+        return TLI_ERR_ARG;
+    S.records = reinterpret_cast<const double *>(records_all);
+    S.rows_out = rows_out;
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    tli_shard_decide_kernel<<<a->B, 128, 0, stream>>>(S);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_shard_decide_kernel");
+    const int epv = a->dtype == TLI_F32 ? 4 : 8;
+    const dim3 grid(static_cast<unsigned>((SL.row_pitch / epv + kThreads - 1) / kThreads), static_cast<unsigned>(a->B));
+    if (a->dtype == TLI_F32) tli_shard_pack_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(S);
+    else tli_shard_pack_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(S);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "launch tli_shard_pack_kernel");
+}
+
+int tli_shard_weights(tli_ctx *ctx, const tli_verify_args *a, const void *rows_all, void *mass_out, void *cuda_stream) {
+    ShardParams S; ShardLayout SL;
+    const int rc = shard_params(ctx, a, S, SL);
+    if (rc != TLI_OK) return rc;
+    if (!rows_all || !mass_out || reinterpret_cast<uintptr_t>(rows_all) % 16 || reinterpret_cast<uintptr_t>(mass_out) % 8)
+        return TLI_ERR_ARG;
+    S.rows_all = rows_all;
+    S.mass = reinterpret_cast<double *>(mass_out);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    const dim3 grid(static_cast<unsigned>(SL.L.ntile), static_cast<unsigned>(a->B));
+    if (a->dtype == TLI_F32) tli_shard_weights_kernel<TLI_F32><<<grid, kThreads, 0, stream>>>(S);
+    else tli_shard_weights_kernel<TLI_BF16><<<grid, kThreads, 0, stream>>>(S);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_shard_weights_kernel");
+    tli_shard_mass_kernel<<<(a->B + 127) / 128, 128, 0, stream>>>(S);
+    e = cudaGetLastError();
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "launch tli_shard_mass_kernel");
+}
+
+int tli_shard_select(tli_ctx *ctx, const tli_verify_args *a, const void *rows_all, const void *masses_all, void *cuda_stream) {
+    ShardParams S; ShardLayout SL;
+    const int rc = shard_params(ctx, a, S, SL);
+    if (rc != TLI_OK) return rc;
+    if (!rows_all || !masses_all || reinterpret_cast<uintptr_t>(rows_all) % 16 || reinterpret_cast<uintptr_t>(masses_all) % 8)
+        return TLI_ERR_ARG;
+    S.rows_all = rows_all;
+    S.masses = reinterpret_cast<const double *>(masses_all);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    if (a->dtype == TLI_F32) tli_shard_select_kernel<TLI_F32><<<a->B, kThreads, 0, stream>>>(S);
+    else tli_shard_select_kernel<TLI_BF16><<<a->B, kThreads, 0, stream>>>(S);
+    const cudaError_t e = cudaGetLastError();
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "launch tli_shard_select_kernel");
 }
 
 int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up) {
