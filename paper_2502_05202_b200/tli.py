@@ -35,12 +35,15 @@ TLI_ROW_BAD_TEMPERATURE = 32
 TLI_MAX_B = 65535
 TLI_MAX_K = 64
 TLI_MAX_V = 1048576
+TLI_MAX_SHARDS = 64
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
 EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_reset", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
            "tli_verify_host_buffer_bytes", "tli_verify_host", "tli_rates_workspace_bytes", "tli_acceptance_rates",
            "tli_ctx_info",
+           "tli_shard_create", "tli_shard_info", "tli_shard_workspace_bytes", "tli_shard_record_bytes", "tli_shard_rows_bytes",
+           "tli_shard_stats", "tli_shard_decide", "tli_shard_weights", "tli_shard_select",
            "tli_status_string", "tli_last_cuda_error")
 
 
@@ -150,6 +153,25 @@ def load() -> ctypes.CDLL:
         lib.tli_rates_workspace_bytes.restype = ctypes.c_size_t
         lib.tli_acceptance_rates.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_rates_args), ctypes.c_void_p]
         lib.tli_acceptance_rates.restype = ctypes.c_int
+        lib.tli_shard_create.argtypes = [ctypes.POINTER(ctypes.c_void_p), ctypes.c_int, ctypes.c_int32, ctypes.c_int32,
+                                         ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_shard_create.restype = ctypes.c_int
+        lib.tli_shard_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 6
+        lib.tli_shard_info.restype = ctypes.c_int
+        lib.tli_shard_workspace_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_shard_workspace_bytes.restype = ctypes.c_size_t
+        lib.tli_shard_record_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_shard_record_bytes.restype = ctypes.c_size_t
+        lib.tli_shard_rows_bytes.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32]
+        lib.tli_shard_rows_bytes.restype = ctypes.c_size_t
+        lib.tli_shard_stats.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p, ctypes.c_void_p]
+        lib.tli_shard_stats.restype = ctypes.c_int
+        lib.tli_shard_decide.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.tli_shard_decide.restype = ctypes.c_int
+        lib.tli_shard_weights.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.tli_shard_weights.restype = ctypes.c_int
+        lib.tli_shard_select.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.tli_shard_select.restype = ctypes.c_int
         lib.tli_reset.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         lib.tli_reset.restype = ctypes.c_int
         lib.tli_set_tiled.argtypes = [ctypes.c_void_p, ctypes.c_int]
@@ -398,6 +420,58 @@ def tli_set_tiled(ctx: int, enabled: bool) -> None:
     rc = load().tli_set_tiled(ctx, 1 if enabled else 0)
     if rc != TLI_OK:
         raise TLIError(rc, "tli_set_tiled")
+
+
+def tli_shard_create(device: int, V_t: int, V_d: int, id_map, n_shards: int, shard: int) -> int:
+    """tli_shard_create(): the context of shard ``shard`` of ``n_shards``; returns the handle (an int)."""
+    m = np.ascontiguousarray(id_map, dtype=np.int32)
+    if m.shape != (V_d,):
+        raise ValueError("id_map must have V_d entries")
+    ctx = ctypes.c_void_p()
+    rc = load().tli_shard_create(ctypes.byref(ctx), device, V_t, V_d, m.ctypes.data_as(ctypes.c_void_p), n_shards, shard)
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_shard_create")
+    return ctx.value
+
+
+def tli_shard_info(ctx: int) -> Dict[str, int]:
+    """tli_shard_info(): the id ranges of a shard's context."""
+    v = [ctypes.c_int32() for _ in range(6)]
+    rc = load().tli_shard_info(ctx, *[ctypes.byref(x) for x in v])
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_shard_info")
+    return dict(zip(("t_begin", "t_count", "d_begin", "d_count", "t_width", "d_width"), (x.value for x in v)))
+
+
+def _shard_call(name: str, ctx: int, args: tli_verify_args, *buffers: torch.Tensor, stream: Optional[int] = None) -> None:
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = getattr(load(), name)(ctx, ctypes.byref(args), *[ctypes.c_void_p(b.data_ptr()) for b in buffers], ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, name)
+
+
+def tli_shard_stats(ctx: int, args: tli_verify_args, record: torch.Tensor, stream: Optional[int] = None) -> None:
+    """tli_shard_stats(): this shard's statistics record."""
+    _shard_call("tli_shard_stats", ctx, args, record, stream=stream)
+
+
+def tli_shard_decide(ctx: int, args: tli_verify_args, records_all: torch.Tensor, rows: torch.Tensor,
+                     stream: Optional[int] = None) -> None:
+    """tli_shard_decide(): the decisions from all shards' records; packs this shard's slices of drafter row n."""
+    _shard_call("tli_shard_decide", ctx, args, records_all, rows, stream=stream)
+
+
+def tli_shard_weights(ctx: int, args: tli_verify_args, rows_all: torch.Tensor, mass: torch.Tensor,
+                      stream: Optional[int] = None) -> None:
+    """tli_shard_weights(): tile sums and totals of the extra token's weights over this shard's target ids."""
+    _shard_call("tli_shard_weights", ctx, args, rows_all, mass, stream=stream)
+
+
+def tli_shard_select(ctx: int, args: tli_verify_args, rows_all: torch.Tensor, masses_all: torch.Tensor,
+                     stream: Optional[int] = None) -> None:
+    """tli_shard_select(): the extra token on the shard that holds it, -1 elsewhere."""
+    _shard_call("tli_shard_select", ctx, args, rows_all, masses_all, stream=stream)
 
 
 def tli_reset(ctx: int, stream: Optional[int] = None) -> None:
