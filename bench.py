@@ -3,12 +3,12 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--config cfg3] [--impl reference]
 
-A step is one tli_verify() call on one synthetic batch: both kernels, all
+A step is one tli_verify() call on one synthetic batch: all kernels, all
 sequences.  The headline workload is the largest of the five (cfg3: B=256, K=4,
 V_t=256000, V_d=128256, fp32 logits, 1.8 GB per call, larger than L2).  With N>1
-(under torchrun) every rank verifies its own copy of the batch -- sequences are
-independent, there is no collective on the data path -- and the value is the sum
-over ranks divided by the slowest rank's time.
+(under torchrun) the batch is split into contiguous blocks of sequences, one per
+rank -- sequences are independent, there is no collective on the data path -- and
+the value is the whole batch divided by the slowest rank's time (strong scaling).
 
 Prints ONE JSON line.  `--impl reference` times the CPU oracle instead.
 """
@@ -30,6 +30,9 @@ if ROOT not in sys.path:
 METRIC = "draft positions verified/s"
 UNIT = "positions/s"
 L2_ROTATE_BYTES = 400 << 20          # distinct input bytes cycled through when one batch fits in L2
+NOMINAL_HBM_GBS = 8000.0             # the nominal peak the target is worded against; fractions are given of both
+KERNEL_SOURCE = os.path.join(ROOT, "paper_2502_05202_b200", "csrc", "tli.cu")
+COUNTERS_FILE = os.path.join(ROOT, "profiles", "stats_kernel_counters.json")
 
 
 def load_peaks():
@@ -173,23 +176,30 @@ def reference_arm(args):
     }))
 
 
-def stats_kernel_traffic(cfg):
-    """DRAM bytes (read + write) of one tli_stats_kernel launch from the committed ncu capture
-    (kept as a summary beside the other profiles): cfg3 with B=64 moved 459 066 112 + 4 182 016 bytes;
-    traffic is proportional to B, so the full batch is 4 x that.  None for the other workloads and
-    to be set back to None whenever the kernel changes."""
-    if cfg.name == "cfg3" and cfg.B % 64 == 0:
-        return (459066112 + 4182016) * (cfg.B // 64)
-    if cfg.name == "cfg2" and cfg.B == 64:
-        return 207997952 + 3759872
-    return None
+def source_digest():
+    import hashlib
+    with open(KERNEL_SOURCE, "rb") as f:
+        return hashlib.sha256(f.read()).hexdigest()
 
 
-def kernels_per_call(cfg) -> int:
-    """statistics + decision + sampling, plus the separate selection kernel for large batches."""
-    epv = 4 if cfg.elt == 4 else 8
-    ntile = -(-(cfg.V_t + epv - 1) // (epv * 1024))
-    return 4 if cfg.B * ntile >= 4096 else 3
+def stats_kernel_counters(cfg):
+    """ncu counters of one tli_stats_kernel launch on this workload, from the summary kept beside the
+    other profiles: {"dram_bytes": read + write, "warp_instructions": ...} scaled to the batch by the
+    sequences it holds (traffic and instruction count grow in proportion to B).  None when there is no
+    capture of this workload, or when the kernel source has changed since the capture was taken."""
+    try:
+        with open(COUNTERS_FILE) as f:
+            data = json.load(f)
+    except (OSError, ValueError):
+        return None
+    if data.get("source_sha256") != source_digest():
+        return None
+    c = data.get("workloads", {}).get(cfg.name)
+    if not c or cfg.B % c["B"]:
+        return None
+    k = cfg.B // c["B"]
+    return {"dram_bytes": (c["dram_bytes_read"] + c["dram_bytes_write"]) * k,
+            "warp_instructions": c["warp_instructions"] * k}
 
 
 def workload_config(cfg, l2_note):
@@ -208,9 +218,14 @@ def workload_config(cfg, l2_note):
 class GpuCase:
     """One workload resident on the device: enough copies of the inputs to defeat L2, outputs, scratch."""
 
-    def __init__(self, cfg, device, torch, tli, wl, want_host=False):
+    def __init__(self, cfg, device, torch, tli, wl, want_host=False, rows=None):
         self.cfg, self.torch, self.tli = cfg, torch, tli
-        self.batch = wl.make_batch(cfg)
+        if rows is not None:                         # a block of the batch's sequences (one rank of several)
+            import dataclasses
+            self.batch = wl.make_batch(cfg, rows=list(rows))
+            cfg = self.cfg = dataclasses.replace(cfg, B=len(rows))
+        else:
+            self.batch = wl.make_batch(cfg)
         self.bytes = algorithmic_bytes(cfg, self.batch)
         l2 = torch.cuda.get_device_properties(device).L2_cache_size
         self.copies = 1 if cfg.logit_bytes > 2 * l2 else max(2, -(-L2_ROTATE_BYTES // cfg.logit_bytes))
@@ -241,7 +256,9 @@ class GpuCase:
         self.out = torch.empty(2, cfg.B, dtype=torch.int32, device=device)      # accepted, next_token
         self.status = torch.empty(cfg.B, dtype=torch.int32, device=device)
         self.ver = tli.Verifier(cfg.V_t, cfg.V_d, b["id_map"], device=device.index)
-        self.ws = self.ver.workspace(cfg.B, cfg.K, tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16)
+        self.dt = tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16
+        self.plan = tli.tli_verify_plan(self.ver.ctx, cfg.B, cfg.K, self.dt)
+        self.ws = self.ver.workspace(cfg.B, cfg.K, self.dt)
         self.args = [tli.make_args(self.zt[i], self.zd[i], self.draft, self.tau, self.u, self.out[0], self.out[1],
                                    self.ws, self.status) for i in range(self.copies)]
         self.stream = torch.cuda.current_stream().cuda_stream
@@ -258,6 +275,37 @@ class GpuCase:
     def step(self):
         self.tli.tli_verify(self.ver.ctx, self.args[self.calls % self.copies], self.stream)
         self.calls += 1
+
+    def probe(self):
+        """The launches of one call with kernels that do nothing."""
+        self.tli.tli_launch_probe(self.ver.ctx, self.cfg.B, self.cfg.K, self.dt, self.stream)
+
+    def touched_bytes(self):
+        """Bytes a call reads in all: every logit once, plus the second pass over target row n of every
+        sampled sequence and, where a draft was rejected, over drafter row n."""
+        import numpy as np
+        acc = self.out[0].cpu().numpy()
+        tau = np.asarray(self.batch["temperature"])
+        sampled = tau > 0
+        extra = int(sampled.sum()) * self.cfg.V_t + int((sampled & (acc < self.cfg.K)).sum()) * self.cfg.V_d
+        return self.bytes + self.cfg.elt * extra
+
+    def sustained(self, seconds, sampler_index):
+        """Back-to-back calls for `seconds`: ms per call under a sustained load, with the SM clock seen."""
+        torch = self.torch
+        for _ in range(3):
+            self.step()
+        torch.cuda.synchronize()
+        probe_ms = timed(torch, None, 50, self.step, 1) / 50
+        calls = max(50, int(seconds / (probe_ms * 1e-3)))
+        sampler = ClockSampler(sampler_index)
+        sampler.start()
+        ms = timed(torch, None, calls, self.step, 1) / calls
+        clocks = sampler.stop()
+        mhz = clocks.get("sm_mhz")
+        return {"seconds": ms * calls * 1e-3, "calls": calls, "ms_per_call": ms, "sm_mhz_median": mhz,
+                "ms_times_mhz": (ms * mhz) if mhz else None, "reasons": clocks.get("reasons"),
+                "path_frac_of_peak": None}
 
     def step_e2e(self):
         """tli_verify_host(): pinned host buffers in, host results out -- H2D of every input, the kernels,
@@ -447,7 +495,59 @@ def gpu_arm(args):
         cfg = dataclasses.replace(cfg, B=args.batch)
     if args.kernels_only:
         args.no_per_config = True
-    case = GpuCase(cfg, device, torch, tli, wl, want_host=not args.kernels_only)
+    rows = None
+    if world > 1:
+        from paper_2502_05202_b200 import shard
+        b0, b1 = shard.row_block(cfg.B, rank, world)            # this rank's sequences; nothing is exchanged
+        rows = range(b0, b1)
+    case = GpuCase(cfg, device, torch, tli, wl, want_host=not args.kernels_only, rows=rows)
+    sms = torch.cuda.get_device_properties(device).multi_processor_count
+
+    def describe(c, ms_step, with_extras):
+        """Figures of one workload from a device-timed loop of `ms_step` per call."""
+        gbs = c.bytes / (ms_step * 1e-3) / 1e9
+        c.profile(3)
+        ms_stats, ms_decide, ms_sample = c.profile(min(max(args.steps, 20), 50))
+        counters = stats_kernel_counters(c.cfg)
+        stats_gbs = c.bytes / (ms_stats * 1e-3) / 1e9
+        d = {"workload": c.cfg.name, "ms_per_step": ms_step, "value": c.cfg.positions / (ms_step * 1e-3),
+             "path_gbs": gbs, "path_frac_of_peak": gbs / peak, "path_frac_of_nominal": gbs / NOMINAL_HBM_GBS,
+             "roofline_ms_at_peak": c.bytes / (peak * 1e9) * 1e3,
+             "call_traffic_ratio": c.touched_bytes() / c.bytes,
+             "plan": c.plan, "launches_per_call": c.plan["launches"],
+             "ms_stats_kernel": ms_stats, "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample,
+             "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm", "achieved": stats_gbs, "peak": peak,
+                          "peak_kind": peak_kind, "unit": "GB/s", "frac": stats_gbs / peak,
+                          "frac_of_nominal": stats_gbs / NOMINAL_HBM_GBS,
+                          "traffic": counters["dram_bytes"] if counters else None,
+                          "algorithmic_bytes": c.bytes, "path_frac": gbs / peak,
+                          "note": ("frac above 1: the peak is a copy's read+write rate, a read-only stream can exceed it"
+                                   if stats_gbs > peak else None)},
+             "l2": c.l2_note}
+        if with_extras:
+            d.update(call_timings(c, torch, args.steps))
+            # the floor of a call: its launches with kernels that do nothing
+            for _ in range(5):
+                c.probe()
+            n = max(args.steps, 100)
+            d["launch_floor_ms"] = timed(torch, None, n, c.probe, 1) / n
+            sus = c.sustained(args.sustain_seconds, local)
+            sus["path_frac_of_peak"] = c.bytes / (sus["ms_per_call"] * 1e-3) / 1e9 / peak
+            d["sustained"] = sus
+            if counters and sus.get("sm_mhz_median"):
+                # every issue slot of the GPU busy with this kernel's instructions: its floor whatever memory does
+                d["roofline"]["issue_floor_ms"] = counters["warp_instructions"] / (4 * sms * sus["sm_mhz_median"] * 1e6) * 1e3
+            # the other form of the sampling pass
+            tli.tli_set_tiled(c.ver.ctx, True)
+            for _ in range(3 + c.copies):
+                c.step()
+            n = max(args.steps, 2 * c.copies)
+            d["ms_per_step_tile_kernels"] = timed(torch, None, n, c.step, 1) / n
+            tli.tli_set_tiled(c.ver.ctx, False)
+            d["draft_sample"] = c.draft_timing(max(args.steps, 20))
+            d["slem_verify"] = c.slem_timing(max(args.steps, 20))
+            d["acceptance_rates"] = c.rates_timing(max(args.steps, 20))
+        return d
 
     for _ in range(max(args.warmup, 3)):
         case.step()
@@ -455,14 +555,9 @@ def gpu_arm(args):
     if rank == 0:
         sampler.start()
     ms = timed(torch, dist, args.steps, case.step, world)
-    # the dominant kernel alone, with events around it, on the same stream and workload
-    case.profile(3)
-    ms_stats, ms_decide, ms_sample = case.profile(args.steps)
-    calls = call_timings(case, torch, args.steps)
-    draft = case.draft_timing(max(args.steps, 20)) if world == 1 else None
-    slem = case.slem_timing(max(args.steps, 20)) if world == 1 else None
-    rates = case.rates_timing(max(args.steps, 20)) if world == 1 else None
     clocks = sampler.stop() if rank == 0 else None
+    ms_step = ms / args.steps
+    head = describe(case, ms_step, with_extras=(world == 1 and not args.kernels_only))
     case.check()
     # end to end: host buffers in, host results out
     e2e_steps = max(3, min(args.steps, 10))
@@ -473,31 +568,35 @@ def gpu_arm(args):
             case.step_e2e()
         ms_e2e = timed(torch, dist, e2e_steps, case.step_e2e, world)
         h2d, d2h = case.e2e_bytes()
+    total_bytes = case.bytes
+    if world > 1:
+        t = torch.tensor([h2d, d2h, total_bytes], dtype=torch.int64, device="cuda")
+        dist.all_reduce(t)
+        h2d, d2h, total_bytes = int(t[0]), int(t[1]), int(t[2])
 
-    ms_step = ms / args.steps
-    value = world * cfg.positions / (ms_step * 1e-3)
+    value = cfg.positions / (ms_step * 1e-3)             # the whole batch, all ranks, over the slowest rank's time
+    path_gbs = total_bytes / (ms_step * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True,
+        "scaling": "strong" if world > 1 else "weak",
         "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-        "config": dict(workload_config(cfg, case.l2_note), parallelism="sequences replicated per GPU, no collective"),
+        "config": dict(workload_config(cfg, case.l2_note),
+                       parallelism=("sequences split into %d contiguous blocks, one per GPU, no collective" % world)
+                       if world > 1 else "one GPU"),
         "clocks": clocks,
-        "e2e": {"value": world * cfg.positions / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
+        "e2e": {"value": cfg.positions / (ms_e2e / e2e_steps * 1e-3), "unit": UNIT,
                 "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / e2e_steps},
-        "gpu_launches": kernels_per_call(cfg) * args.steps,
-        "path_gbs": case.bytes / (ms_step * 1e-3) / 1e9,
-        "path_frac_of_peak": case.bytes / (ms_step * 1e-3) / 1e9 / peak,
-        "per_call": calls,
-        "draft_sample": draft,
-        "slem_verify": slem,
-        "acceptance_rates": rates,
-        "roofline": {"kernel": "tli_stats_kernel", "bound": "hbm",
-                     "achieved": case.bytes / (ms_stats * 1e-3) / 1e9, "peak": peak, "peak_kind": peak_kind,
-                     "unit": "GB/s", "frac": case.bytes / (ms_stats * 1e-3) / 1e9 / peak,
-                     "traffic": stats_kernel_traffic(cfg), "algorithmic_bytes": case.bytes,
-                     "ms_stats_kernel": ms_stats, "ms_decide_kernel": ms_decide,
-                     "ms_sample_kernel": ms_sample},
+        "gpu_launches": case.plan["launches"] * args.steps,
+        "path_gbs": path_gbs,
+        "path_frac_of_peak": path_gbs / (peak * world),
+        "path_frac_of_nominal": path_gbs / (NOMINAL_HBM_GBS * world),
+        "roofline": head["roofline"],
     }
+    if "ms_call_median" in head:
+        out["per_call"] = {k: head[k] for k in ("ms_call_median", "ms_call_min", "ms_call_graph_replay")}
+    for k in ("draft_sample", "slem_verify", "acceptance_rates", "sustained", "launch_floor_ms"):
+        out[k] = head.get(k)
     headline_batch = case.batch
     case.close()
     del case
@@ -507,26 +606,15 @@ def gpu_arm(args):
         per = []
         for c in wl.CONFIGS:
             if c.name == cfg.name:
-                per.append({"workload": c.name, "ms_per_step": ms_step, "value": value, "path_gbs": out["path_gbs"],
-                            "path_frac_of_peak": out["path_frac_of_peak"], "ms_stats_kernel": ms_stats,
-                            "ms_decide_kernel": ms_decide, "ms_sample_kernel": ms_sample, **calls,
-                            "draft_sample": draft, "slem_verify": slem, "acceptance_rates": rates})
+                per.append(head)
                 continue
             k = GpuCase(c, device, torch, tli, wl)
             for _ in range(max(args.warmup, 3) + k.copies):
                 k.step()
             steps = max(args.steps, 2 * k.copies)
             m = timed(torch, None, steps, k.step, 1) / steps
-            k.profile(3)
-            a, d, b = k.profile(min(steps, 50))
-            kc = call_timings(k, torch, steps)
-            kc["draft_sample"] = k.draft_timing(steps)
-            kc["slem_verify"] = k.slem_timing(steps)
-            kc["acceptance_rates"] = k.rates_timing(steps)
+            per.append(describe(k, m, with_extras=True))
             k.check()
-            per.append({"workload": c.name, "ms_per_step": m, "value": c.positions / (m * 1e-3),
-                        "path_gbs": k.bytes / (m * 1e-3) / 1e9, "path_frac_of_peak": k.bytes / (m * 1e-3) / 1e9 / peak,
-                        "ms_stats_kernel": a, "ms_decide_kernel": d, "ms_sample_kernel": b, "l2": k.l2_note, **kc})
             k.close()
             del k
             torch.cuda.empty_cache()
@@ -555,6 +643,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-per-config", action="store_true", help="skip the four other workloads")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU time given to the oracle baseline leg")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0,
+                    help="length of the sustained leg per workload (back-to-back calls, clocks sampled)")
     ap.add_argument("--batch", type=int, default=0, help="override the workload's B (profiling on a smaller case)")
     ap.add_argument("--kernels-only", action="store_true",
                     help="only the device-timed loop: no per-config, end-to-end or CPU legs (for profiler runs)")

@@ -426,6 +426,24 @@ int tli_shard_weights(tli_ctx *ctx, const tli_verify_args *args, const void *row
 int tli_shard_select(tli_ctx *ctx, const tli_verify_args *args, const void *rows_all, const void *masses_all, void *cuda_stream);
 
 /*
+ * How tli_verify() will run a batch of this shape on this context: [host]
+ * plan[8] = { kernel launches per call, CTAs per sequence of the cluster
+ * kernel (0: the tile kernels draw the extra token), CTAs of the statistics
+ * kernel, bytes per stage of its ring, bytes per segment, segments per target
+ * row, segments per drafter row, shared memory of a cluster CTA }.
+ */
+int tli_verify_plan(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, int32_t *plan);
+
+/*
+ * Measurement hook: the launches of one tli_verify() call of this shape with
+ * kernels that do nothing -- the same grids, block sizes, shared memory, the
+ * programmatic dependent launch and the cluster barrier -- so that the time a
+ * call spends on getting through the stream can be told from the time it
+ * spends on its work (the floor of a small batch).  Asynchronous.
+ */
+int tli_launch_probe(tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, void *cuda_stream);
+
+/*
  * Measurement hook: tli_verify() with CUDA events recorded on `cuda_stream`
  * around each kernel.  Blocks until the call has finished and writes three
  * durations in milliseconds to [host] ms[3]: ms[0] the statistics pass over

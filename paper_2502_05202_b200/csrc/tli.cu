@@ -2696,6 +2696,21 @@ __global__ void __launch_bounds__(kThreads) tli_shard_select_kernel(const ShardP
     walk_tile<DT, true, SRC_SHARDS>(P, b, sel, rt, zd_rows, sm_tile, sm_rem);
 }
 
+// Kernels that do nothing, for tli_launch_probe(): the cost of getting a call's launches through
+// the stream (launch, scheduling of the CTAs, the dependent launch, the cluster barrier) without any
+// of its work.
+__global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_probe_first_kernel(int dummy) {
+    extern __shared__ __align__(128) unsigned char probe_smem[];
+    if (dummy < 0) probe_smem[threadIdx.x] = 0;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__global__ void __launch_bounds__(kFinThreads, 2) tli_probe_second_kernel(int dummy) {
+    extern __shared__ __align__(16) unsigned char probe_smem2[];
+    if (dummy < 0) probe_smem2[threadIdx.x] = 0;
+    cluster_barrier();
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
 // Self-test of the bounded wait: one thread waits on a barrier that nothing will ever complete,
 // with a caller-chosen poll limit, and reports how the wait ended.  The kernel returns normally.
 __global__ void tli_bounded_wait_kernel(unsigned limit, int *result, unsigned *scratch_error) {
@@ -3369,6 +3384,50 @@ int tli_set_tiled(tli_ctx *ctx, int enabled) {
     if (!ctx) return TLI_ERR_ARG;
     ctx->tiled = enabled ? 1 : 0;
     return TLI_OK;
+}
+
+int tli_verify_plan(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, int32_t *plan) {
+    if (!ctx || !plan || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return TLI_ERR_ARG;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return TLI_ERR_ARG;
+    Layout L = make_layout(B, K, ctx->t_count, ctx->d_count, dtype, ctx->num_sms);
+    if (ctx->tiled || ctx->n_shards != 1) L.fin_cluster = 0;
+    const int split = (static_cast<long long>(B) * L.ntile >= 4096) ? 1 : 0;
+    plan[0] = L.fin_cluster ? 2 : 3 + split;         // kernel launches per call
+    plan[1] = L.fin_cluster;                         // CTAs per sequence of the cluster kernel, 0: tile kernels
+    plan[2] = static_cast<int32_t>(L.grid);          // CTAs of the statistics kernel
+    plan[3] = L.cv * kSThreads * 16;                 // bytes per stage
+    plan[4] = L.seg_vec * 16;                        // bytes per segment
+    plan[5] = L.nst; plan[6] = L.nsd;                // segments per target / drafter row
+    plan[7] = static_cast<int32_t>(L.fin_smem);      // shared memory of a cluster CTA
+    return TLI_OK;
+}
+
+int tli_launch_probe(tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, void *cuda_stream) {
+    if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return TLI_ERR_ARG;
+    if (dtype != TLI_F32 && dtype != TLI_BF16) return TLI_ERR_ARG;
+    Layout L = make_layout(B, K, ctx->V_t, ctx->V_d, dtype, ctx->num_sms);
+    cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+    static std::once_flag once;
+    std::call_once(once, [] {
+        cudaFuncSetAttribute(tli_probe_first_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes);
+        cudaFuncSetAttribute(tli_probe_second_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kFinSmemOnePerSm));
+    });
+    tli_probe_first_kernel<<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(0);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "launch tli_probe_first_kernel");
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    const int C = L.fin_cluster ? L.fin_cluster : 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(C); attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr; cfg.numAttrs = 2; cfg.stream = stream;
+    cfg.blockDim = dim3(kFinThreads); cfg.dynamicSmemBytes = L.fin_cluster ? L.fin_smem : 0;
+    cfg.gridDim = dim3(static_cast<unsigned>(C), static_cast<unsigned>(B));
+    e = cudaLaunchKernelEx(&cfg, tli_probe_second_kernel, 0);
+    return e == cudaSuccess ? TLI_OK : cuda_fail(e, "launch tli_probe_second_kernel");
 }
 
 int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream, float *ms) {

@@ -44,6 +44,7 @@ EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tl
            "tli_ctx_info",
            "tli_shard_create", "tli_shard_info", "tli_shard_workspace_bytes", "tli_shard_record_bytes", "tli_shard_rows_bytes",
            "tli_shard_stats", "tli_shard_decide", "tli_shard_weights", "tli_shard_select",
+           "tli_verify_plan", "tli_launch_probe",
            "tli_status_string", "tli_last_cuda_error")
 
 
@@ -172,6 +173,10 @@ def load() -> ctypes.CDLL:
         lib.tli_shard_weights.restype = ctypes.c_int
         lib.tli_shard_select.argtypes = [ctypes.c_void_p, ctypes.POINTER(tli_verify_args), ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
         lib.tli_shard_select.restype = ctypes.c_int
+        lib.tli_verify_plan.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32)]
+        lib.tli_verify_plan.restype = ctypes.c_int
+        lib.tli_launch_probe.argtypes = [ctypes.c_void_p, ctypes.c_int32, ctypes.c_int32, ctypes.c_int32, ctypes.c_void_p]
+        lib.tli_launch_probe.restype = ctypes.c_int
         lib.tli_reset.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
         lib.tli_reset.restype = ctypes.c_int
         lib.tli_set_tiled.argtypes = [ctypes.c_void_p, ctypes.c_int]
@@ -472,6 +477,25 @@ def tli_shard_select(ctx: int, args: tli_verify_args, rows_all: torch.Tensor, ma
                      stream: Optional[int] = None) -> None:
     """tli_shard_select(): the extra token on the shard that holds it, -1 elsewhere."""
     _shard_call("tli_shard_select", ctx, args, rows_all, masses_all, stream=stream)
+
+
+def tli_verify_plan(ctx: int, B: int, K: int, dtype: int) -> Dict[str, int]:
+    """tli_verify_plan(): how a batch of this shape will be run."""
+    plan = (ctypes.c_int32 * 8)()
+    rc = load().tli_verify_plan(ctx, B, K, dtype, plan)
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_verify_plan")
+    return dict(zip(("launches", "cluster", "stats_ctas", "stage_bytes", "segment_bytes", "segments_per_target_row",
+                     "segments_per_drafter_row", "cluster_smem_bytes"), plan))
+
+
+def tli_launch_probe(ctx: int, B: int, K: int, dtype: int, stream: Optional[int] = None) -> None:
+    """tli_launch_probe(): the launches of one call with kernels that do nothing."""
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    rc = load().tli_launch_probe(ctx, B, K, dtype, ctypes.c_void_p(stream))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_launch_probe")
 
 
 def tli_reset(ctx: int, stream: Optional[int] = None) -> None:
