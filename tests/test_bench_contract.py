@@ -30,7 +30,7 @@ def test_gpu_arm_prints_the_contract_keys():
     assert d["e2e"]["value"] < d["value"]
     r = d["roofline"]
     assert r["bound"] == "hbm" and r["unit"] == "GB/s" and abs(r["frac"] - r["achieved"] / r["peak"]) < 1e-9
-    assert d["gpu_launches"] == 3 * 5
+    assert d["gpu_launches"] == 2 * 5 and d["config"]["workload"] == "cfg1"
     c = d["cpu_baseline"]
     assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0
 
