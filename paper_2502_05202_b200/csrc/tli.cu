@@ -70,6 +70,14 @@ struct __align__(16) RowSel {   // what the sampling pass needs for one sequence
     float v;             // uniforms[b, K]
 };
 
+// Division of a 32-bit number by a divisor fixed on the host: q = (mulhi(n, m) + n) >> s with
+// s = ceil(log2 d) and m = floor(2^32 (2^s - d) / d) + 1, exact for every 32-bit n (the sum is
+// formed in 64 bits).  The producer thread of the statistics kernel decodes every segment number
+// with three of these instead of three hardware-less divisions of ~100 instructions.
+struct FastDiv {
+    unsigned m, s, d;
+};
+
 struct Params {
     int B, K, V_t, V_d;
     const void *zt; long long t_sb, t_sk;
@@ -86,6 +94,7 @@ struct Params {
     int split_select;    // 1: the CDF inversions run as a kernel of their own
     int seg_vec;         // statistics kernel: 16-byte vectors per segment
     int nst, nsd;        // ... and segments per target / drafter row
+    FastDiv div_per_b, div_nst, div_nsd;   // by the segments of a sequence, of a target row, of a drafter row
     // vocabulary-sharded calls (all zero otherwise): V_t / V_d above are the widths of this shard's
     // slices, which hold target ids t_begin .. and drafter ids d_begin ..; map, inv and the mask are
     // indexed by global ids
@@ -297,25 +306,27 @@ struct Segment {
     int m;            // drafts of the sequence that count
 };
 
-__device__ __forceinline__ long long segment_count(const Params &P) {
-    return static_cast<long long>(P.B) * ((P.K + 1) * P.nst + P.K * P.nsd);
+__device__ __forceinline__ unsigned segment_count(const Params &P) {       // the host made sure it fits 32 bits
+    return static_cast<unsigned>(P.B) * static_cast<unsigned>((P.K + 1) * P.nst + P.K * P.nsd);
+}
+__device__ __forceinline__ unsigned fast_div(unsigned n, const FastDiv &f) {
+    return static_cast<unsigned>((static_cast<unsigned long long>(__umulhi(n, f.m)) + n) >> f.s);
 }
 
 // The index arithmetic of a segment, and the loads of its sequence's temperature and draft count:
 // issued here, used by finish_segment(), so that their latency passes while the producer is still
 // streaming the segment before.
-__device__ __forceinline__ Segment decode_segment(const Params &P, long long id) {
+__device__ __forceinline__ Segment decode_segment(const Params &P, unsigned id) {
     Segment g;
-    const int per_b = (P.K + 1) * P.nst + P.K * P.nsd;
-    g.b = static_cast<int>(id / per_b);
-    int item = static_cast<int>(id - static_cast<long long>(g.b) * per_b);
+    g.b = static_cast<int>(fast_div(id, P.div_per_b));
+    int item = static_cast<int>(id - static_cast<unsigned>(g.b) * P.div_per_b.d);
     g.tau = __ldg(P.tau + g.b);
     g.m = P.draft_len ? __ldg(P.draft_len + g.b) : P.K;
     if (item < (P.K + 1) * P.nst) {
-        g.row = item / P.nst; g.seg = item - g.row * P.nst;
+        g.row = static_cast<int>(fast_div(static_cast<unsigned>(item), P.div_nst)); g.seg = item - g.row * P.nst;
     } else {
         item -= (P.K + 1) * P.nst;
-        const int j = item / P.nsd;
+        const int j = static_cast<int>(fast_div(static_cast<unsigned>(item), P.div_nsd));
         g.row = P.K + 1 + j; g.seg = item - j * P.nsd;
     }
     g.v0 = g.seg * P.seg_vec;
@@ -562,7 +573,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
-    const long long nseg_total = segment_count(P);
+    const unsigned nseg_total = segment_count(P);
 
     if (threadIdx.x < 32) {
         // ---------------- producer ----------------
@@ -572,14 +583,16 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             bool ok = true;
             // every CTA starts on the segment of its own number (so that a small batch spreads over all
             // CTAs however unevenly they start); the rest come from the counter
-            long long id = blockIdx.x;
+            // (segment numbers beyond the last may wrap around 32 bits only after 2^32 - nseg_total fetches
+            // by CTAs that have found the queue empty: each CTA fetches at most two such numbers)
+            unsigned id = blockIdx.x;
             Segment g = decode_segment(P, id);
-            long long id_next = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);
+            unsigned id_next = gridDim.x + atomicAdd(P.seg_counter, 1u);
             while (ok) {
                 if (id >= nseg_total) break;
                 Segment g_next = g;
                 if (id_next < nseg_total) g_next = decode_segment(P, id_next);
-                const long long id_after = static_cast<long long>(gridDim.x) + atomicAdd(P.seg_counter, 1u);
+                const unsigned id_after = gridDim.x + atomicAdd(P.seg_counter, 1u);
                 finish_segment(P, g);
                 const Segment gc = g;
                 g = g_next; id = id_next; id_next = id_after;
@@ -2739,6 +2752,15 @@ int cuda_fail(cudaError_t e, const char *what) {
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
+FastDiv make_fast_div(unsigned d) {
+    FastDiv f;
+    f.d = d;
+    f.s = 0;
+    while ((1ull << f.s) < d) ++f.s;
+    f.m = static_cast<unsigned>((((1ull << f.s) - d) << 32) / d + 1);
+    return f;
+}
+
 int chunks_per_row(int V, int dtype, int vec_per_chunk) {
     const long long epv = dtype == TLI_F32 ? 4 : 8;
     return static_cast<int>((static_cast<long long>(V) + epv - 1 + epv * vec_per_chunk - 1) / (epv * vec_per_chunk));
@@ -2749,6 +2771,7 @@ struct Layout {
     int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
     int ntile;
     int seg_vec, nst, nsd;      // segments of the statistics kernel, see Params
+    long long nseg;             // ... in all (the kernel numbers them in 32 bits)
     unsigned grid;
     int fin_cluster;     // CTAs per sequence of the cluster kernel; 0: the tile kernels draw the extra token
     int fin_slice;       // vectors of the target row per CTA of the cluster
@@ -2820,6 +2843,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.nst = per_row(nvec_t, L.seg_vec);
     L.nsd = per_row(nvec_d, L.seg_vec);
     const long long nseg = count(L.seg_vec);
+    L.nseg = nseg;
     const long long grid = nseg < ctas ? nseg : ctas;
     L.grid = static_cast<unsigned>(grid);
     size_t off = 0;
@@ -2974,6 +2998,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
     Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
     if (ctx->tiled) L.fin_cluster = 0;
+    if (L.nseg >= (1ll << 32) - 4 * L.grid) return TLI_ERR_UNSUPPORTED;
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
         return TLI_ERR_WORKSPACE;
 
@@ -3001,6 +3026,8 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.ntile = L.ntile;
     P.fin_slice = L.fin_slice; P.fin_dvec = L.fin_dvec;
     P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
+    P.div_per_b = make_fast_div(static_cast<unsigned>((P.K + 1) * L.nst + P.K * L.nsd));
+    P.div_nst = make_fast_div(static_cast<unsigned>(L.nst)); P.div_nsd = make_fast_div(static_cast<unsigned>(L.nsd));
 
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     if (ev) cudaEventRecord(ev[0], stream);
@@ -3207,6 +3234,7 @@ int shard_params(tli_ctx *ctx, const tli_verify_args *a, ShardParams &S, ShardLa
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
     if (a->draft_lengths) return TLI_ERR_UNSUPPORTED;
     SL = make_shard_layout(ctx, a->B, a->K, a->dtype);
+    if (SL.L.nseg >= (1ll << 32) - 4 * SL.L.grid) return TLI_ERR_UNSUPPORTED;
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < SL.total)
         return TLI_ERR_WORKSPACE;
     memset(&S, 0, sizeof S);
@@ -3231,6 +3259,8 @@ int shard_params(tli_ctx *ctx, const tli_verify_args *a, ShardParams &S, ShardLa
     P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
     P.ntile = L.ntile;
     P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
+    P.div_per_b = make_fast_div(static_cast<unsigned>((P.K + 1) * L.nst + P.K * L.nsd));
+    P.div_nst = make_fast_div(static_cast<unsigned>(L.nst)); P.div_nsd = make_fast_div(static_cast<unsigned>(L.nsd));
     P.t_begin = ctx->t_begin; P.d_begin = ctx->d_begin;
     P.sh_wd = ctx->wd; P.sh_stride = static_cast<long long>(a->B) * SL.row_pitch;
     S.G = ctx->n_shards; S.g = ctx->shard; S.wt = ctx->wt; S.wd = ctx->wd;
