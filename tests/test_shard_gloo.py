@@ -174,3 +174,27 @@ def test_two_vocabulary_shards_agree_with_the_unsharded_oracle(tmp_path):
     np.testing.assert_array_equal(got[:, 0], o["accepted"])
     np.testing.assert_array_equal(got[:, 1], o["next_token"])
     assert 0 < o["accepted"].min() + 1 and o["accepted"].max() >= 1
+
+
+def test_the_benchmark_split_covers_the_headline_batch_once():
+    """bench.py --gpus N gives rank r the sequences shard.row_block(B, r, N) of the headline workload and
+    builds only those (make_batch(rows=...)): the blocks partition the batch, and a block generated on
+    its own holds the same bits as the same rows of the whole batch."""
+    cfg = wl.tiny_config(B=11, K=3, V_t=900, V_d=700, dtype=wl.BF16, f_mapped=0.6, temperatures=(0.7, 1.0),
+                         greedy_rows="interleaved", seed=95)
+    full = wl.make_batch(cfg)
+    for world in (2, 4, 8):
+        seen = []
+        for rank in range(world):
+            b0, b1 = shard.row_block(cfg.B, rank, world)
+            seen += list(range(b0, b1))
+            if b1 > b0:
+                part = wl.make_batch(cfg, rows=list(range(b0, b1)))
+                for k in ("target_logits", "drafter_logits", "draft_ids", "temperature", "uniforms"):
+                    np.testing.assert_array_equal(part[k], full[k][b0:b1], err_msg=k)
+                np.testing.assert_array_equal(part["id_map"], full["id_map"])
+        assert seen == list(range(cfg.B))
+    big = wl.config_by_name("cfg3")
+    for world in (1, 2, 4, 8):
+        sizes = [e - b for b, e in shard.row_blocks(big.B, world)]
+        assert sum(sizes) * big.K == big.positions and max(sizes) - min(sizes) <= 1
