@@ -1,7 +1,8 @@
 // TLI verification for sm_100a: kernels and the C ABI declared in include/tli.h.
 //
-// A call is three launches (four for large batches).  The first and the third stream logits and
-// are HBM-bound; there is no dense contraction on this path, hence no tensor cores.
+// A call is two launches (four for vocabularies or batches too large for the cluster kernel).
+// The passes over logits are HBM-bound; there is no dense contraction on this path, hence no
+// tensor cores.
 //
 //   tli_stats_kernel   persistent grid, two CTAs per SM, each one producer warp and sixteen
 //                      consumer warps around a 96 KB ring of shared-memory stages filled by
@@ -11,19 +12,21 @@
 //                      full-softmax denominator cancels in q' = q / sum_{T cap D} q);
 //                      temperature-0 rows: (max, lowest index).  One pair per segment of a row
 //                      goes to the workspace.
-//   tli_decide_kernel  one CTA per sequence: fp64 combination of the pairs, Algorithm 5's
-//                      acceptance tests and count of accepted drafts, which row the extra token
-//                      is drawn from.
-//   tli_sample_kernel  one CTA per 16 KB tile of that one target row: tile sums of
-//                      max(0, p - q'_T) (or of p for the bonus row); the last CTA of a sequence
-//                      walks tile -> 16-byte vector -> element to invert the CDF.
-//   tli_select_kernel  large batches only: those inversions as a kernel of their own.
-//   tli_fused_kernel   all of the above in one persistent grid (tli_set_fused; not the default).
+//   tli_finish_kernel  one thread-block cluster per sequence: fp64 combination of the pairs,
+//                      Algorithm 5's acceptance tests and count of accepted drafts, then the extra
+//                      token: the drafter row staged in shared memory, weights max(0, p - q'_T)
+//                      (or p for the bonus row) over the CTAs' slices of the one target row, the
+//                      CDF inverted through distributed shared memory.
+//   tli_decide_kernel, tli_sample_kernel, tli_select_kernel
+//                      the same in three kernels for rows that do not fit a cluster's shared
+//                      memory: decision per sequence, one CTA per 16 KB tile of the target row
+//                      (q'_T gathered through the inverse map), inversion tile -> vector -> element.
 //
 // Beside the verification call: tli_draft_kernel / tli_draft_select_kernel draw one id per row of
 // logits by inverse CDF (the drafts from q' for tli_draft_sample; with no mask, the target tokens
-// of Algorithm 2 for tli_slem_verify, compared by tli_slem_match_kernel), and tli_rate_*_kernel
-// form the paper's expected acceptance rates per draft position (tli_acceptance_rates).
+// of Algorithm 2 for tli_slem_verify, compared by tli_slem_match_kernel), tli_rate_*_kernel form
+// the paper's expected acceptance rates per draft position (tli_acceptance_rates), and
+// tli_shard_*_kernel are the local steps of the verification over vocabulary shards.
 //
 // Softmax terms are formed as ex2(fma(z, s, -c)) with an integer-valued reference c in log2
 // units: the only per-term rounding is the one in the fma, and every change or combination of
@@ -230,11 +233,12 @@ __device__ __forceinline__ float reference_for(float ms) { return fmaxf(ceilf(ms
 // pass 1: statistics of every row, persistent and pipelined
 // ---------------------------------------------------------------------------
 //
-// Work unit: a segment = up to `cps` consecutive 16 KB chunks of one logit row.  Segments are
-// numbered sequence-major and dealt round-robin to a fixed grid of CTAs.  In each CTA one thread
-// (the producer) streams the chunks into a ring of shared-memory stages with cp.async.bulk,
-// completion counted on an mbarrier per stage; eight consumer warps reduce a stage from shared
-// memory and hand it back through a second mbarrier as soon as its bytes are in registers.
+// Work unit: a segment = a run of consecutive 16-byte vectors of one logit row (up to 128 KB).
+// Segments are numbered sequence-major and handed out by an atomic counter to a fixed grid of CTAs.
+// In each CTA one thread (the producer) streams the vectors into a ring of shared-memory stages
+// with cp.async.bulk, completion counted on an mbarrier per stage; sixteen consumer warps reduce a
+// stage from shared memory and hand it back through a second mbarrier as soon as its bytes are in
+// registers.
 
 // ---- mbarrier and bulk-copy primitives ----
 
@@ -888,7 +892,7 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
     }
     __syncthreads();
 
-    const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the chunks used
+    const float s_f = 1.4426950408889634f / tau;       // the same rounded scale the statistics used
     if (tid < Kb) {
         const int j = tid;
         int ok = 0, fl = g_fl;
@@ -2768,7 +2772,7 @@ int chunks_per_row(int V, int dtype, int vec_per_chunk) {
 
 struct Layout {
     size_t part_t, part_d, sel, tilesum, total;
-    int cv;              // vectors per consumer thread per chunk of the statistics kernel (1, 2 or 4)
+    int cv;              // vectors per consumer thread per stage of the statistics kernel (1, 2 or 4)
     int ntile;
     int seg_vec, nst, nsd;      // segments of the statistics kernel, see Params
     long long nseg;             // ... in all (the kernel numbers them in 32 bits)
