@@ -92,7 +92,9 @@ struct Params {
     float2 *part_t; float2 *part_d; RowSel *sel; double *tilesum;
     unsigned *cnt_stats; unsigned *cnt_sample;
     unsigned *error;     // sticky: set when a bounded wait ran out
-    unsigned *seg_counter, *cta_done;   // segment scheduler of the statistics kernel; zero between calls
+    unsigned long long *seg_counter;    // segment scheduler of the statistics kernel: segments taken from the front (low
+                                        // half) and from the back (high half); zero between calls
+    unsigned *cta_done;                 // ... and the CTAs that have left
     int ntile;           // 16 KB tiles per target row (sampling pass)
     int split_select;    // 1: the CDF inversions run as a kernel of their own
     int seg_vec;         // statistics kernel: 16-byte vectors per segment
@@ -533,11 +535,28 @@ __device__ __forceinline__ void softmax_chunk(const uint4 (&raw)[CV], const uint
 
 // Temperature-0 rows: (largest value, lowest index attaining it) over the first nq vectors.
 // bf16: a running pair of packed maxima (even and odd positions) tells in five instructions
-// whether a vector can raise the maximum at all; only then are its eight elements compared.
+// whether a vector can raise the maximum at all; only then are its eight elements compared.  After
+// every stage the pair is raised to the largest value the whole warp has seen (all of it at lower
+// indices than anything the warp reads later), so that from the second stage of a segment on the
+// element-wise path is rare for the warp as a whole and not just for each lane.
+// In the first stage of a segment there is no such value yet: the warp first takes the largest value
+// of the whole stage (packed maxima only) and lets through what reaches it -- the pair starts one
+// bf16 step below it, because an equal value may be the one with the lowest index.
 template <int DT, int CV, bool FULL>
-__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], int nq, const RowView<DT> &rv, int v_first,
-                                             uint32_t &mm, float &best, int &best_idx) {
+__device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], int nq, bool first_stage, const RowView<DT> &rv,
+                                             int v_first, uint32_t &mm, float &best, int &best_idx) {
     constexpr int EPV = Elt<DT>::kPerVec;
+    if constexpr (DT == TLI_BF16) {
+        if (first_stage) {
+            uint32_t sm = bf16x2_max(raw[0]);
+#pragma unroll
+            for (int q = 1; q < CV; ++q)
+                if (FULL || q < nq) sm = bf16x2_max(sm, bf16x2_max(raw[q]));
+            const float m_w = warp_max(fmaxf(bf16_lo(sm), bf16_hi(sm)));
+            const uint32_t h = __float_as_uint(order_float(float_order(m_w) - 0x10000)) >> 16;    // one step below
+            mm = h | (h << 16);
+        }
+    }
 #pragma unroll
     for (int q = 0; q < CV; ++q) {                        // increasing index order, strict > keeps the lowest
         if (!FULL && q >= nq) continue;
@@ -552,6 +571,11 @@ __device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], int nq, con
 #pragma unroll
         for (int i = 0; i < EPV; ++i)
             if (z[i] > best) { best = z[i]; best_idx = e0 + i; }
+    }
+    if constexpr (DT == TLI_BF16) {
+        const float m_w = warp_max(fmaxf(bf16_lo(mm), bf16_hi(mm)));       // a bf16 value, or -inf
+        const uint32_t h = __float_as_uint(m_w) >> 16;
+        mm = bf16x2_max(mm, h | (h << 16));
     }
 }
 
@@ -587,16 +611,27 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             bool ok = true;
             // every CTA starts on the segment of its own number (so that a small batch spreads over all
             // CTAs however unevenly they start); the rest come from the counter
-            // (segment numbers beyond the last may wrap around 32 bits only after 2^32 - nseg_total fetches
-            // by CTAs that have found the queue empty: each CTA fetches at most two such numbers)
-            unsigned id = blockIdx.x;
+            // Half the CTAs take segments from the front of the (sequence-major) list, half from the back,
+            // until the two meet.  CTAs i and i + gridDim/2 share an SM under round-robin placement, so
+            // when cost varies along the batch (temperature-0 sequences stream at memory speed, the others
+            // are held by the exponentials) every SM gets both kinds at once.
+            const unsigned n_front = (gridDim.x + 1) / 2, n_back = gridDim.x - n_front;
+            const bool back = blockIdx.x >= n_front;
+            const unsigned long long one = back ? (1ull << 32) : 1ull;
+            auto take = [&]() -> unsigned {               // the next segment number for this CTA, or nseg_total when none is left
+                const unsigned long long old = atomicAdd(P.seg_counter, one);
+                const unsigned long long f = n_front + (old & 0xffffffffull), k = n_back + (old >> 32);
+                if (f + k >= nseg_total) return nseg_total;
+                return back ? nseg_total - 1u - static_cast<unsigned>(k) : static_cast<unsigned>(f);
+            };
+            unsigned id = back ? nseg_total - 1u - (blockIdx.x - n_front) : blockIdx.x;
             Segment g = decode_segment(P, id);
-            unsigned id_next = gridDim.x + atomicAdd(P.seg_counter, 1u);
+            unsigned id_next = take();
             while (ok) {
                 if (id >= nseg_total) break;
                 Segment g_next = g;
                 if (id_next < nseg_total) g_next = decode_segment(P, id_next);
-                const unsigned id_after = gridDim.x + atomicAdd(P.seg_counter, 1u);
+                const unsigned id_after = take();
                 finish_segment(P, g);
                 const Segment gc = g;
                 g = g_next; id = id_next; id_next = id_after;
@@ -701,11 +736,11 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             }
             constexpr bool kMaskInSum = (DT != TLI_BF16);          // fp32 drafter rows apply the mask element by element
             if (nq == CV) {
-                if (greedy) argmax_chunk<DT, CV, true>(raw, nq, rv, v0 + tid, best_mm, best, best_idx);
+                if (greedy) argmax_chunk<DT, CV, true>(raw, nq, (meta.flags & META_FIRST) != 0, rv, v0 + tid, best_mm, best, best_idx);
                 else if (masked && kMaskInSum) softmax_chunk<DT, CV, true, true>(raw, bits, nq, s, c_run, acc);
                 else softmax_chunk<DT, CV, false, true>(raw, bits, nq, s, c_run, acc);
             } else if (nq > 0) {
-                if (greedy) argmax_chunk<DT, CV, false>(raw, nq, rv, v0 + tid, best_mm, best, best_idx);
+                if (greedy) argmax_chunk<DT, CV, false>(raw, nq, (meta.flags & META_FIRST) != 0, rv, v0 + tid, best_mm, best, best_idx);
                 else if (masked && kMaskInSum) softmax_chunk<DT, CV, true, false>(raw, bits, nq, s, c_run, acc);
                 else softmax_chunk<DT, CV, false, false>(raw, bits, nq, s, c_run, acc);
             }
@@ -774,7 +809,7 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         if (clean_exit && tid == 0) {
             __threadfence();
             const unsigned t = atomicAdd(P.cta_done, 1u);
-            if (t == gridDim.x - 1) { *P.seg_counter = 0u; *P.cta_done = 0u; __threadfence(); }
+            if (t == gridDim.x - 1) { *P.seg_counter = 0ull; *P.cta_done = 0u; __threadfence(); }
         }
     }
 }
@@ -3024,7 +3059,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
     P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
-    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
+    P.seg_counter = reinterpret_cast<unsigned long long *>(P.error + 4); P.cta_done = P.error + 2;
     // many tiles: a fence and a ticket per tile CTA cost more than one more small kernel
     P.split_select = (static_cast<long long>(a->B) * L.ntile >= 4096) ? 1 : 0;
     P.ntile = L.ntile;
@@ -3260,7 +3295,7 @@ int shard_params(tli_ctx *ctx, const tli_verify_args *a, ShardParams &S, ShardLa
     P.cnt_stats = ctx->d_counters;
     P.cnt_sample = ctx->d_counters + (TLI_MAX_B + 1);
     P.error = ctx->d_counters + 3 * (TLI_MAX_B + 1);
-    P.seg_counter = P.error + 1; P.cta_done = P.error + 2;
+    P.seg_counter = reinterpret_cast<unsigned long long *>(P.error + 4); P.cta_done = P.error + 2;
     P.ntile = L.ntile;
     P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
     P.div_per_b = make_fast_div(static_cast<unsigned>((P.K + 1) * L.nst + P.K * L.nsd));
