@@ -601,6 +601,10 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     __syncthreads();
+    // Launched as a programmatic dependent: when the kernel before it in the stream is the last one
+    // of an earlier call (they let their dependents start at once), the CTAs of this grid are set
+    // up while that call is still finishing; nothing is read or written before it has completed.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
     const unsigned nseg_total = segment_count(P);
 
     if (threadIdx.x < 32) {
@@ -1343,6 +1347,7 @@ __global__ void __launch_bounds__(kThreads, 8) tli_sample_kernel(const Params P)
     __shared__ int sm_last;
     const int b = blockIdx.y, tile = blockIdx.x;
     const int tid = threadIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the selection kernel, or the next call's first kernel
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const RowSel sel = P.sel[b];
     if (sel.mode == MODE_SKIP) return;
@@ -1373,6 +1378,7 @@ __global__ void __launch_bounds__(kThreads, 8) tli_sample_kernel(const Params P)
 template <int DT>
 __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
     const int b = blockIdx.x;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next call's first kernel may be set up meanwhile
     asm volatile("griddepcontrol.wait;" ::: "memory");
     const RowSel sel = P.sel[b];
     if (sel.mode == MODE_SKIP) return;
@@ -1437,6 +1443,7 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
     const int b = blockIdx.y;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const unsigned rank = cluster_cta_rank(), C = cluster_cta_count();
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");     // the next call's first kernel may be set up meanwhile
     const int slice = P.fin_slice;                           // vectors of the target row per CTA
     uint4 *drow = reinterpret_cast<uint4 *>(fin_smem);       // drafter row n on its 16-byte vector grid
     float *vsum = reinterpret_cast<float *>(fin_smem + static_cast<size_t>(P.fin_dvec) * 16);
@@ -2918,15 +2925,22 @@ struct tli_ctx {
 namespace {
 
 cudaError_t launch_stats(const Params &P, const Layout &L, int dtype, cudaStream_t stream) {
-    const dim3 g1(L.grid), b1(kSThreads + 32);
-#define TLI_LAUNCH_STATS(DT, CV) tli_stats_kernel<DT, CV><<<g1, b1, kStatsSmemBytes, stream>>>(P)
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof cfg);
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1; cfg.stream = stream;
+    cfg.gridDim = dim3(L.grid); cfg.blockDim = dim3(kSThreads + 32); cfg.dynamicSmemBytes = kStatsSmemBytes;
+    cudaError_t e = cudaSuccess;
+#define TLI_LAUNCH_STATS(DT, CV) e = cudaLaunchKernelEx(&cfg, tli_stats_kernel<DT, CV>, P)
     if (dtype == TLI_F32) {
         if (L.cv == 4) TLI_LAUNCH_STATS(TLI_F32, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_F32, 2); else TLI_LAUNCH_STATS(TLI_F32, 1);
     } else {
         if (L.cv == 4) TLI_LAUNCH_STATS(TLI_BF16, 4); else if (L.cv == 2) TLI_LAUNCH_STATS(TLI_BF16, 2); else TLI_LAUNCH_STATS(TLI_BF16, 1);
     }
 #undef TLI_LAUNCH_STATS
-    return cudaGetLastError();
+    return e;
 }
 
 }  // namespace
