@@ -190,7 +190,7 @@ int tli_verify(tli_ctx *ctx, const tli_verify_args *args, void *cuda_stream);
  *     process exits, used or not;
  *   - a batch whose scratch need (tli_workspace_bytes()) exceeds the array is
  *     refused with TLI_ERR_STATIC_SCRATCH and nothing is launched; the five
- *     benchmark workloads need at most about 1.3 MiB;
+ *     benchmark workloads need at most about 0.3 MiB;
  *   - the first call on each device looks up the array's device address (the
  *     context's device must be current, as for tli_verify()).  Make that first
  *     call outside any stream capture;
