@@ -218,9 +218,11 @@ def workload_config(cfg, l2_note):
 class GpuCase:
     """One workload resident on the device: enough copies of the inputs to defeat L2, outputs, scratch."""
 
-    def __init__(self, cfg, device, torch, tli, wl, want_host=False, rows=None):
+    def __init__(self, cfg, device, torch, tli, wl, want_host=False, rows=None, batch=None):
         self.cfg, self.torch, self.tli = cfg, torch, tli
-        if rows is not None:                         # a block of the batch's sequences (one rank of several)
+        if batch is not None:                        # host arrays of a case that exists already
+            self.batch = batch
+        elif rows is not None:                       # a block of the batch's sequences (one rank of several)
             import dataclasses
             self.batch = wl.make_batch(cfg, rows=list(rows))
             cfg = self.cfg = dataclasses.replace(cfg, B=len(rows))
@@ -460,6 +462,44 @@ def timed(torch, dist, steps, fn, world):
     return ms
 
 
+def independent_streams(case, device, torch, tli, wl, nstreams, steps):
+    """Per-call time when `nstreams` independent batches of this workload (own context, inputs, outputs and
+    scratch each) are verified in turn on as many CUDA streams: the dependent tail of one call then runs
+    under the streaming of the next.  What a server with several batches in flight sees; the figures of a
+    single stream of calls stay the headline."""
+    cases = [case] + [GpuCase(case.cfg, device, torch, tli, wl, batch=case.batch) for _ in range(nstreams - 1)]
+    streams = [torch.cuda.Stream() for _ in range(nstreams)]
+    saved = case.stream
+    for c, st in zip(cases, streams):
+        c.stream = st.cuda_stream
+
+    def run(n):
+        for i in range(n):
+            cases[i % nstreams].step()
+    run(4 * nstreams)
+    torch.cuda.synchronize()
+    n = max(steps, 4 * case.copies) // nstreams * nstreams
+    best = float("inf")
+    for _ in range(3):
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for st in streams:
+            st.wait_event(e0)
+        run(n)
+        for st in streams:
+            torch.cuda.current_stream().wait_stream(st)
+        e1.record()
+        torch.cuda.synchronize()
+        best = min(best, e0.elapsed_time(e1) / n)
+    for c in cases:
+        c.check()
+    for c in cases[1:]:
+        c.close()
+    case.stream = saved
+    return best
+
+
 def call_timings(case, torch, steps):
     """Per-call figures beside the K-step loop: events around single calls, and a CUDA-graph replay."""
     med, mn = case.per_call_ms(min(max(steps, 20), 200))
@@ -544,6 +584,10 @@ def gpu_arm(args):
             n = max(args.steps, 2 * c.copies)
             d["ms_per_step_tile_kernels"] = timed(torch, None, n, c.step, 1) / n
             tli.tli_set_tiled(c.ver.ctx, False)
+            d["independent_streams"] = {}
+            for ns in (2, 3):
+                m = independent_streams(c, device, torch, tli, wl, ns, max(args.steps, 100))
+                d["independent_streams"][str(ns)] = {"ms_per_call": m, "path_frac_of_peak": c.bytes / (m * 1e-3) / 1e9 / peak}
             d["draft_sample"] = c.draft_timing(max(args.steps, 20))
             d["slem_verify"] = c.slem_timing(max(args.steps, 20))
             d["acceptance_rates"] = c.rates_timing(max(args.steps, 20))
