@@ -491,3 +491,23 @@ def test_a_wait_that_nothing_completes_gives_up_and_leaves_the_context_usable():
     with pytest.raises(tli.TLIError):
         tli.tli_selftest_bounded_wait(v.ctx, polls=0)
     v.close()
+
+
+def test_the_plan_follows_the_size_rule():
+    """tli_verify_plan(): two launches (one cluster per sequence) where the drafter row fits a CTA's shared
+    memory and the batch is moderate, the tile kernels otherwise; tli_set_tiled forces the latter."""
+    expect = {"cfg0": (2, 8), "cfg1": (2, 8), "cfg2": (2, 4), "cfg3": (4, 0), "cfg4": (2, 4)}
+    for name, (launches, cluster) in expect.items():
+        cfg = wl.config_by_name(name)
+        v = tli.Verifier(cfg.V_t, cfg.V_d, wl.make_id_map(cfg))
+        dt = tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16
+        plan = tli.tli_verify_plan(v.ctx, cfg.B, cfg.K, dt)
+        assert (plan["launches"], plan["cluster"]) == (launches, cluster), (name, plan)
+        assert plan["stats_ctas"] >= 1 and plan["segment_bytes"] % plan["stage_bytes"] in (0, plan["segment_bytes"])
+        big = tli.tli_verify_plan(v.ctx, 4096, cfg.K, dt)                # far more CTAs than eight per SM
+        assert big["cluster"] == 0 and big["launches"] >= 3
+        tli.tli_set_tiled(v.ctx, True)
+        assert tli.tli_verify_plan(v.ctx, cfg.B, cfg.K, dt)["cluster"] == 0
+        v.close()
+    with pytest.raises(tli.TLIError):
+        tli.tli_verify_plan(0, 1, 1, 0)
