@@ -298,9 +298,11 @@ __device__ __forceinline__ float2 ld_shared_pair(const float2 *p) {     // a pai
 // A row is seen as 16-byte vectors on the aligned address grid (RowView).  A segment is a run of
 // consecutive vectors of one row and leaves one partial result; a stage of the ring holds up to
 // 512*CV vectors of it.  Segments are numbered sequence-major and handed out in that order.
-// (Shorter segments for the sequences handed out last, so that the CTAs run dry together, were
-// measured and dropped: what a CTA still holds when the queue runs dry is its ring of stages and
-// the two segments it works ahead, whatever the length of the segments.)
+// A CTA asks for its next segment only when every stage of the one before has been issued: what it
+// holds when the list runs out is then its ring of stages and nothing else.  (Asking one or two
+// segments ahead hides the latency of the counter and of the temperature load, but the slower CTA
+// of an SM then sits on up to two more segments at the end while the others are idle: measured,
+// 3 to 5 us longer on batches of a few hundred MB.)
 
 struct Segment {
     int b;            // sequence
@@ -319,9 +321,8 @@ __device__ __forceinline__ unsigned fast_div(unsigned n, const FastDiv &f) {
     return static_cast<unsigned>((static_cast<unsigned long long>(__umulhi(n, f.m)) + n) >> f.s);
 }
 
-// The index arithmetic of a segment, and the loads of its sequence's temperature and draft count:
-// issued here, used by finish_segment(), so that their latency passes while the producer is still
-// streaming the segment before.
+// The index arithmetic of a segment, and the loads of its sequence's temperature and draft count
+// (used by finish_segment()).
 __device__ __forceinline__ Segment decode_segment(const Params &P, unsigned id) {
     Segment g;
     g.b = static_cast<int>(fast_div(id, P.div_per_b));
@@ -580,8 +581,8 @@ __device__ __forceinline__ void argmax_chunk(const uint4 (&raw)[CV], int nq, boo
 }
 
 // Segments are handed out by an atomic counter: a CTA that is slow simply takes fewer of them.
-// The producer thread works two segments ahead (see above), streams the vectors through the stage
-// ring and labels every stage for the consumers.
+// The producer thread streams the vectors of its segment through the stage ring, labels every stage
+// for the consumers, and then asks for the next segment (see above).
 // CV = 16-byte vectors per consumer thread per stage: a stage is kSThreads*CV*16 bytes and the
 // ring holds kRingBytes / that many stages.  Large batches use large stages (less bookkeeping per
 // byte), small ones small stages (more parallelism across CTAs).
@@ -630,16 +631,11 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
             };
             unsigned id = back ? nseg_total - 1u - (blockIdx.x - n_front) : blockIdx.x;
             Segment g = decode_segment(P, id);
-            unsigned id_next = take();
             while (ok) {
                 if (id >= nseg_total) break;
-                Segment g_next = g;
-                if (id_next < nseg_total) g_next = decode_segment(P, id_next);
-                const unsigned id_after = take();
                 finish_segment(P, g);
                 const Segment gc = g;
-                g = g_next; id = id_next; id_next = id_after;
-                if (gc.skip) continue;                   // bad temperature, or drafter row at temperature 0
+                if (gc.skip) { id = take(); if (id < nseg_total) g = decode_segment(P, id); continue; }
                 const RowView<DT> rv = segment_row<DT>(P, gc);
                 const int v_end = min(gc.v1, rv.nvec());
                 int v0 = gc.v0;
@@ -664,6 +660,8 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
                     if (++st == NST) { st = 0; par ^= 1u; }
                     v0 += CVEC;
                 } while (v0 < v_end);
+                id = take();
+                if (id < nseg_total) g = decode_segment(P, id);
             }
             // nothing more to start: the next kernel of the stream may be made resident as CTAs of this
             // one leave (it still waits for all of this grid before it reads the partials).  Triggering
