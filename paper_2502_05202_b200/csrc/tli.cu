@@ -153,8 +153,9 @@ __device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w 
 __device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
 
 template <int DT> __device__ __forceinline__ float load_elt(const void *row, long long i) {
-    if (DT == TLI_F32) return __ldg(reinterpret_cast<const float *>(row) + i);
-    return __uint_as_float(static_cast<uint32_t>(__ldg(reinterpret_cast<const unsigned short *>(row) + i)) << 16);
+    // (single elements are gathered: they go past L1, which the coalesced loads of the same kernels need)
+    if (DT == TLI_F32) return __ldcg(reinterpret_cast<const float *>(row) + i);
+    return __uint_as_float(static_cast<uint32_t>(__ldcg(reinterpret_cast<const unsigned short *>(row) + i)) << 16);
 }
 
 template <int DT> __device__ __forceinline__ void unpack(const uint4 &r, float (&z)[Elt<DT>::kPerVec]) {
