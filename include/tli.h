@@ -428,7 +428,8 @@ int tli_shard_select(tli_ctx *ctx, const tli_verify_args *args, const void *rows
 /*
  * How tli_verify() will run a batch of this shape on this context: [host]
  * plan[8] = { kernel launches per call, CTAs per sequence of the cluster
- * kernel (0: the tile kernels draw the extra token), CTAs of the statistics
+ * kernel (0: the tile kernels draw the extra token; up to 16 where the device
+ * places thread-block clusters of that size, else up to 8), CTAs of the statistics
  * kernel, bytes per stage of its ring, bytes per segment, segments per target
  * row, segments per drafter row, shared memory of a cluster CTA }.
  */

@@ -1407,7 +1407,7 @@ __global__ void __launch_bounds__(kThreads) tli_select_kernel(const Params P) {
 
 constexpr int kFinThreads = 512;                   // 1024 threads where one CTA has an SM to itself: measured slower (64 registers)
 constexpr int kFinWarps = kFinThreads / 32;
-constexpr int kFinMaxCluster = 8;
+constexpr int kFinMaxCluster = 16;                 // beyond 8 CTAs a cluster is not portable: the context asks the driver once
 
 __device__ __forceinline__ unsigned cluster_cta_rank() {
     unsigned r;
@@ -2831,19 +2831,19 @@ struct Layout {
 // share the one row.
 constexpr size_t kFinSmemTwoPerSm = 100 * 1024;
 constexpr size_t kFinSmemOnePerSm = 200 * 1024;
-void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms) {
+void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms, int max_cluster) {
     L.fin_cluster = 0; L.fin_slice = 0; L.fin_dvec = 0; L.fin_smem = 0;
     const int nvec = chunks_per_row(V_t, dtype, 1);                 // vectors of a row, whatever its alignment
     const int dvec = chunks_per_row(V_d, dtype, 1);
     auto need = [&](int c) { return static_cast<size_t>(dvec) * 16 + static_cast<size_t>((nvec + c - 1) / c) * 4; };
     int C = 0;
-    for (int c = 1; c <= kFinMaxCluster; c *= 2)
+    for (int c = 1; c <= max_cluster; c *= 2)
         if (need(c) <= kFinSmemTwoPerSm) { C = c; break; }
     if (C) {
-        while (C < kFinMaxCluster && static_cast<long long>(B) * C * 2 <= 2LL * num_sms) C *= 2;
+        while (C < max_cluster && static_cast<long long>(B) * C * 2 <= 2LL * num_sms) C *= 2;
         if (static_cast<long long>(B) * C > 8LL * num_sms) return;
     } else {
-        for (int c = kFinMaxCluster; c >= 1; c /= 2)
+        for (int c = max_cluster; c >= 1; c /= 2)
             if (need(c) <= kFinSmemOnePerSm && static_cast<long long>(B) * c <= num_sms) { C = c; break; }
         if (C == 0) return;
     }
@@ -2859,7 +2859,7 @@ void plan_finish(Layout &L, int B, int V_t, int V_d, int dtype, int num_sms) {
 // about four per CTA (long enough to amortise the per-segment reduction; longer ones interleave the
 // rows of a large batch worse).  A small batch is cut into the shortest segments that still number
 // no more than the CTAs.
-Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
+Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms, int max_cluster = 8) {
     Layout L;
     const long long elt = dtype == TLI_F32 ? 4 : 2;
     const long long bytes = elt * B * (static_cast<long long>(K + 1) * V_t + static_cast<long long>(K) * V_d);
@@ -2897,7 +2897,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms) {
     L.sel = off;    off = align_up(off + sizeof(RowSel) * static_cast<size_t>(B), 256);
     L.tilesum = off; off = align_up(off + sizeof(double) * static_cast<size_t>(B) * L.ntile, 256);
     L.total = off;
-    plan_finish(L, B, V_t, V_d, dtype, num_sms);
+    plan_finish(L, B, V_t, V_d, dtype, num_sms, max_cluster);
     return L;
 }
 
@@ -2912,6 +2912,7 @@ struct tli_ctx {
     int *d_inv;
     uint32_t *d_mask;
     int tiled;                  // option: the extra token always by the tile kernels (default 0: by size)
+    int max_cluster;            // widest cluster the device takes for the cluster kernel (16 where the driver allows it, else 8)
     unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
@@ -2976,6 +2977,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
     c->tiled = 0;
+    c->max_cluster = 8;
     c->n_shards = 1; c->shard = 0; c->wt = V_t; c->wd = V_d;
     c->t_begin = 0; c->t_count = V_t; c->d_begin = 0; c->d_count = V_d;
     int rc = TLI_OK;
@@ -2990,6 +2992,27 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_F32>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemOnePerSm);
         if (e == cudaSuccess) e = cudaFuncSetAttribute(tli_finish_kernel<TLI_BF16>, cudaFuncAttributeMaxDynamicSharedMemorySize, kFinSmemOnePerSm);
         if (e != cudaSuccess) { rc = cuda_fail(e, "cudaFuncSetAttribute"); break; }
+        {
+            // clusters of 16 are not portable: take them only if the driver places at least one with the
+            // largest shared memory the kernel is ever given
+            bool wide = true;
+            for (int dt = 0; dt < 2 && wide; ++dt) {
+                const void *fn = dt == 0 ? reinterpret_cast<const void *>(tli_finish_kernel<TLI_F32>)
+                                         : reinterpret_cast<const void *>(tli_finish_kernel<TLI_BF16>);
+                if (cudaFuncSetAttribute(fn, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) != cudaSuccess) { wide = false; break; }
+                cudaLaunchConfig_t qc;
+                memset(&qc, 0, sizeof qc);
+                cudaLaunchAttribute qa[1];
+                qa[0].id = cudaLaunchAttributeClusterDimension;
+                qa[0].val.clusterDim.x = kFinMaxCluster; qa[0].val.clusterDim.y = 1; qa[0].val.clusterDim.z = 1;
+                qc.attrs = qa; qc.numAttrs = 1;
+                qc.gridDim = dim3(kFinMaxCluster); qc.blockDim = dim3(kFinThreads); qc.dynamicSmemBytes = kFinSmemOnePerSm;
+                int n_clusters = 0;
+                if (cudaOccupancyMaxActiveClusters(&n_clusters, fn, &qc) != cudaSuccess || n_clusters < 1) wide = false;
+            }
+            cudaGetLastError();                              // a refusal above is an answer, not an error of this call
+            c->max_cluster = wide ? kFinMaxCluster : 8;
+        }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
@@ -3048,7 +3071,7 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     if (reinterpret_cast<uintptr_t>(a->target_logits) % elt || reinterpret_cast<uintptr_t>(a->drafter_logits) % elt)
         return TLI_ERR_ARG;
     if (a->t_stride_b < 0 || a->t_stride_k < 0 || a->d_stride_b < 0 || a->d_stride_k < 0) return TLI_ERR_ARG;
-    Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms);
+    Layout L = make_layout(a->B, a->K, ctx->V_t, ctx->V_d, a->dtype, ctx->num_sms, ctx->max_cluster);
     if (ctx->tiled) L.fin_cluster = 0;
     if (L.nseg >= (1ll << 32) - 4 * L.grid) return TLI_ERR_UNSUPPORTED;
     if (!a->workspace || reinterpret_cast<uintptr_t>(a->workspace) % 256 || a->workspace_bytes < L.total)
@@ -3471,7 +3494,7 @@ int tli_set_tiled(tli_ctx *ctx, int enabled) {
 int tli_verify_plan(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, int32_t *plan) {
     if (!ctx || !plan || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return TLI_ERR_ARG;
     if (dtype != TLI_F32 && dtype != TLI_BF16) return TLI_ERR_ARG;
-    Layout L = make_layout(B, K, ctx->t_count, ctx->d_count, dtype, ctx->num_sms);
+    Layout L = make_layout(B, K, ctx->t_count, ctx->d_count, dtype, ctx->num_sms, ctx->max_cluster);
     if (ctx->tiled || ctx->n_shards != 1) L.fin_cluster = 0;
     const int split = (static_cast<long long>(B) * L.ntile >= 4096) ? 1 : 0;
     plan[0] = L.fin_cluster ? 2 : 3 + split;         // kernel launches per call
@@ -3487,12 +3510,13 @@ int tli_verify_plan(const tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, int
 int tli_launch_probe(tli_ctx *ctx, int32_t B, int32_t K, int32_t dtype, void *cuda_stream) {
     if (!ctx || B < 1 || K < 1 || B > TLI_MAX_B || K > TLI_MAX_K) return TLI_ERR_ARG;
     if (dtype != TLI_F32 && dtype != TLI_BF16) return TLI_ERR_ARG;
-    Layout L = make_layout(B, K, ctx->V_t, ctx->V_d, dtype, ctx->num_sms);
+    Layout L = make_layout(B, K, ctx->V_t, ctx->V_d, dtype, ctx->num_sms, ctx->max_cluster);
     cudaStream_t stream = reinterpret_cast<cudaStream_t>(cuda_stream);
     static std::once_flag once;
     std::call_once(once, [] {
         cudaFuncSetAttribute(tli_probe_first_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kStatsSmemBytes);
         cudaFuncSetAttribute(tli_probe_second_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kFinSmemOnePerSm));
+        cudaFuncSetAttribute(tli_probe_second_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
     });
     tli_probe_first_kernel<<<L.grid, kSThreads + 32, kStatsSmemBytes, stream>>>(0);
     cudaError_t e = cudaGetLastError();
