@@ -469,6 +469,17 @@ int tli_verify_profile(tli_ctx *ctx, const tli_verify_args *args, void *cuda_str
 int tli_set_tiled(tli_ctx *ctx, int enabled);
 
 /*
+ * Widest thread-block cluster the cluster kernel may use on this context.
+ * Clusters of more than 8 CTAs are not portable: tli_create() asks the driver
+ * once and allows 16 where it places them, 8 otherwise.  ctas = 8 narrows a
+ * context to the portable size, ctas = 16 widens it again if the device has it
+ * (TLI_ERR_UNSUPPORTED if not); other values: TLI_ERR_ARG.  Results do not
+ * depend on it beyond the order of the fp64 additions across CTAs.  For tests
+ * and measurements.                                                    [host]
+ */
+int tli_set_max_cluster(tli_ctx *ctx, int ctas);
+
+/*
  * Self-test of the kernels' bounded waits.  Every wait inside the kernels (on a
  * shared-memory barrier that a bulk copy or another warp completes) gives up
  * after a fixed number of polls, records the fact and lets the kernel finish;

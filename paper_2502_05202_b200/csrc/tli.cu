@@ -2913,6 +2913,7 @@ struct tli_ctx {
     uint32_t *d_mask;
     int tiled;                  // option: the extra token always by the tile kernels (default 0: by size)
     int max_cluster;            // widest cluster the device takes for the cluster kernel (16 where the driver allows it, else 8)
+    int device_max_cluster;     // ... what tli_create() found; max_cluster can be narrowed by tli_set_max_cluster()
     unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
@@ -2977,7 +2978,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
     c->num_sms = 0;
     c->tiled = 0;
-    c->max_cluster = 8;
+    c->max_cluster = 8; c->device_max_cluster = 8;
     c->n_shards = 1; c->shard = 0; c->wt = V_t; c->wd = V_d;
     c->t_begin = 0; c->t_count = V_t; c->d_begin = 0; c->d_count = V_d;
     int rc = TLI_OK;
@@ -3012,6 +3013,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
             }
             cudaGetLastError();                              // a refusal above is an answer, not an error of this call
             c->max_cluster = wide ? kFinMaxCluster : 8;
+            c->device_max_cluster = c->max_cluster;
         }
         if ((e = cudaMalloc(&c->d_map, sizeof(int32_t) * V_d)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc map"); break; }
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
@@ -3488,6 +3490,13 @@ int tli_reset(tli_ctx *ctx, void *cuda_stream) {
 int tli_set_tiled(tli_ctx *ctx, int enabled) {
     if (!ctx) return TLI_ERR_ARG;
     ctx->tiled = enabled ? 1 : 0;
+    return TLI_OK;
+}
+
+int tli_set_max_cluster(tli_ctx *ctx, int ctas) {
+    if (!ctx || (ctas != 8 && ctas != kFinMaxCluster)) return TLI_ERR_ARG;
+    if (ctas > ctx->device_max_cluster) return TLI_ERR_UNSUPPORTED;
+    ctx->max_cluster = ctas;
     return TLI_OK;
 }
 

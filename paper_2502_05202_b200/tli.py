@@ -38,7 +38,7 @@ TLI_MAX_V = 1048576
 TLI_MAX_SHARDS = 64
 TLI_STATIC_SCRATCH_BYTES = 4194304
 
-EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_reset", "tli_selftest_bounded_wait",
+EXPORTS = ("tli_create", "tli_destroy", "tli_workspace_bytes", "tli_verify", "tli_verify_static", "tli_verify_profile", "tli_set_tiled", "tli_set_max_cluster", "tli_reset", "tli_selftest_bounded_wait",
            "tli_draft_workspace_bytes", "tli_draft_sample", "tli_slem_workspace_bytes", "tli_slem_verify",
            "tli_verify_host_buffer_bytes", "tli_verify_host", "tli_rates_workspace_bytes", "tli_acceptance_rates",
            "tli_ctx_info",
@@ -181,6 +181,8 @@ def load() -> ctypes.CDLL:
         lib.tli_reset.restype = ctypes.c_int
         lib.tli_set_tiled.argtypes = [ctypes.c_void_p, ctypes.c_int]
         lib.tli_set_tiled.restype = ctypes.c_int
+        lib.tli_set_max_cluster.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        lib.tli_set_max_cluster.restype = ctypes.c_int
         lib.tli_selftest_bounded_wait.argtypes = [ctypes.c_void_p, ctypes.c_void_p, ctypes.c_uint, ctypes.POINTER(ctypes.c_int)]
         lib.tli_selftest_bounded_wait.restype = ctypes.c_int
         lib.tli_ctx_info.argtypes = [ctypes.c_void_p] + [ctypes.POINTER(ctypes.c_int32)] * 3
@@ -418,6 +420,13 @@ def tli_verify_profile(ctx: int, args: tli_verify_args, stream: Optional[int] = 
     if rc != TLI_OK:
         raise TLIError(rc, "tli_verify_profile")
     return ms[0], ms[1], ms[2]
+
+
+def tli_set_max_cluster(ctx: int, ctas: int) -> None:
+    """tli_set_max_cluster(): widest cluster of the cluster kernel, 8 (portable) or 16 (where the device places it)."""
+    rc = load().tli_set_max_cluster(ctx, int(ctas))
+    if rc != TLI_OK:
+        raise TLIError(rc, "tli_set_max_cluster")
 
 
 def tli_set_tiled(ctx: int, enabled: bool) -> None:

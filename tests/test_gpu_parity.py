@@ -89,6 +89,36 @@ def test_full_size_workloads(name):
     assert rep.exact >= cfg.B - max(2, cfg.B // 16)
 
 
+@pytest.mark.parametrize("name", ["cfg0", "cfg1"])
+def test_small_batches_with_the_portable_and_the_wide_cluster(name):
+    """Clusters of 8 CTAs (portable) and, where the device places them, of 16: both against the oracle."""
+    cfg = wl.config_by_name(name)
+    batch = wl.make_batch(cfg)
+    dt = tli.TLI_F32 if cfg.elt == 4 else tli.TLI_BF16
+    widths = []
+    for ctas in (8, 16):
+        v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+        try:
+            tli.tli_set_max_cluster(v.ctx, ctas)
+        except tli.TLIError as e:
+            assert ctas == 16 and e.code == tli.TLI_ERR_UNSUPPORTED
+            v.close()
+            continue
+        plan = tli.tli_verify_plan(v.ctx, cfg.B, cfg.K, dt)
+        assert plan["cluster"] == ctas, plan
+        rep = check(batch, verifier=v)
+        assert rep.rows == cfg.B
+        widths.append(ctas)
+        v.close()
+    assert 8 in widths
+    with pytest.raises(tli.TLIError):
+        v = tli.Verifier(cfg.V_t, cfg.V_d, batch["id_map"])
+        try:
+            tli.tli_set_max_cluster(v.ctx, 12)
+        finally:
+            v.close()
+
+
 def test_interleaved_greedy_rows_and_raw_drafts_on_cfg4_shape():
     cfg = dataclasses.replace(wl.config_by_name("cfg4"), B=8, K=6, greedy_rows="interleaved", seed=77)
     rep = check(wl.make_batch(cfg, draft_mode="raw"))
