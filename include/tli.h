@@ -81,9 +81,13 @@ enum {
  *                        before any CUDA call is made.
  *
  * The context owns device copies of the map, its inverse (target id -> drafter
- * id), a bit mask of mapped drafter ids, and per-sequence completion counters.
- * Because of those counters a context serves one tli_verify() at a time: calls
- * on the same context must be ordered on one stream (or by events).
+ * id), a bit mask of mapped drafter ids, per-sequence completion counters and
+ * an 8 MiB buffer for the per-row partial results of moderate batches (kept
+ * "empty" between calls, so that the kernel that reads them can tell a result
+ * that has been stored from one that has not without waiting for the whole
+ * kernel that stores them; larger batches keep theirs in the workspace).
+ * Because of the counters and that buffer a context serves one tli_verify() at
+ * a time: calls on the same context must be ordered on one stream (or by events).
  */
 int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_t *id_map_host);
 
@@ -492,12 +496,13 @@ int tli_set_max_cluster(tli_ctx *ctx, int ctas);
 int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, int *gave_up);
 
 /*
- * Put the context's device-side counters back to their initial state (a
- * stream-ordered memset): the completion tickets, the segment scheduler and the
- * sticky time-out word.  Needed only after a call reported TLI_ROW_TIMEOUT: the
- * kernels of that call gave up in mid-flight, so the counters they share with
- * the next call are not back at zero, and every later call would both start from
- * them and carry the flag.  Must be ordered after the call that timed out and
+ * Put the context's device-side state back to its initial value (stream-ordered
+ * memsets): the completion tickets, the segment scheduler, the sticky time-out
+ * word, and the context's 8 MiB buffer of partial results, which the kernels
+ * leave "empty" after every call that ends normally.  Needed only after a call
+ * reported TLI_ROW_TIMEOUT: the kernels of that call gave up in mid-flight, so
+ * what they share with the next call is not back at its initial value, and every
+ * later call would both start from it and carry the flag.  Must be ordered after the call that timed out and
  * before the next one, like any other call on the context.
  */
 int tli_reset(tli_ctx *ctx, void *cuda_stream);

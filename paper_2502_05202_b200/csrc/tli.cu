@@ -107,6 +107,9 @@ struct Params {
     int sh_wd;           // drafter ids per shard (the gathered rows of shard g start at g * sh_stride elements)
     long long sh_stride;
     double *tilesum_p;   // tile sums of p beside those of the residual
+    int poll_parts;      // cluster kernel: the partials lie in the context's own buffer, which holds kPartEmpty wherever no
+                         // call is under way, and are waited for one by one (see tli_finish_kernel)
+    int early_trigger;   // ... and the statistics grid leaves SMs free: the cluster kernel may become resident at once
     int fin_slice;       // cluster kernel: 16-byte vectors of the sampled target row per CTA
     int fin_dvec;        // cluster kernel: 16-byte vectors reserved for the staged drafter row
 };
@@ -287,6 +290,20 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, unsigned parity, int *s
 __device__ __forceinline__ void bulk_load(void *dst, const void *src, unsigned bytes, uint64_t *bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
                  ::"r"(smem_addr(dst)), "l"(src), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// A partial result in the context's own buffer: both words are all ones until the statistics kernel
+// has stored the pair (a reference is never NaN, a sum that is NaN is the canonical positive one, an
+// index is never -1).  Returns false if the pair has not arrived after kWaitLimit polls or the
+// statistics kernel has given up.
+constexpr uint32_t kPartEmpty = 0xffffffffu;
+__device__ __forceinline__ bool load_partial_when_stored(const float2 *p, const unsigned *g_error, float2 &v) {
+    for (unsigned i = 0; i < kWaitLimit; ++i) {
+        asm volatile("ld.relaxed.gpu.global.v2.f32 {%0, %1}, [%2];" : "=f"(v.x), "=f"(v.y) : "l"(p) : "memory");
+        if (__float_as_uint(v.x) != kPartEmpty && __float_as_uint(v.y) != kPartEmpty) return true;
+        if ((i & 31u) == 31u && *reinterpret_cast<const volatile unsigned *>(g_error)) break;
+        if (i > 4) __nanosleep(40);
+    }
+    return false;
 }
 __device__ __forceinline__ float2 ld_shared_pair(const float2 *p) {     // a pair another warp wrote: not from a register copy
     float2 v;
@@ -607,6 +624,11 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
     // of an earlier call (they let their dependents start at once), the CTAs of this grid are set
     // up while that call is still finishing; nothing is read or written before it has completed.
     asm volatile("griddepcontrol.wait;" ::: "memory");
+    // A small batch leaves room on the SMs: the cluster kernel, which waits for single partials and not
+    // for this grid, is let in right away and has its prologue behind it when the partials arrive.
+    // (With two CTAs of this grid on every SM it could only come in as they leave, and what it does then
+    // slows the last of them down: measured, see the trigger below.)
+    if (P.early_trigger) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const unsigned nseg_total = segment_count(P);
 
     if (threadIdx.x < 32) {
@@ -830,7 +852,9 @@ __global__ void __launch_bounds__(kSThreads + 32, kCtasPerSm) tli_stats_kernel(c
 // sequence is finished here: invalid temperature, temperature 0, non-finite logits).
 // Returns true when the extra token is still to be drawn (sel.mode is MODE_RESIDUAL or
 // MODE_TARGET_ONLY).
-template <int DT, int NT>
+// POLL: the caller's grid did not wait for the statistics grid; the partials come from the context's
+// buffer and each is waited for where it is read (load_partial_when_stored).
+template <int DT, int NT, bool POLL = false>
 __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool writer, RowSel &sel, int &flags) {
     const int tid = threadIdx.x;
     // loads that depend on nothing go out together: temperature, this thread's uniform, (below) its draft id
@@ -846,7 +870,7 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
     sel.n = 0; sel.mode = MODE_SKIP; sel.s = 0.f; sel.c_t = 0.f; sel.rs_t = 0.f; sel.c_d = 0.f; sel.rs_d = 0.f; sel.v = 0.f;
     if (!(tau >= 0.f) || isinf(tau)) {             // negative, NaN or infinite temperature
         flags = TLI_ROW_BAD_TEMPERATURE;
-        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (!POLL) asm volatile("griddepcontrol.wait;" ::: "memory");
         if (writer) {
             if (tid == 0) {
                 P.accepted[b] = 0; P.next_token[b] = 0;
@@ -876,12 +900,13 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
     if (tid == K) sm_sel.v = u_mine;
 
     // everything below reads what the statistics kernel wrote (its partials, its time-out word)
-    asm volatile("griddepcontrol.wait;" ::: "memory");
+    if (!POLL) asm volatile("griddepcontrol.wait;" ::: "memory");
     if (tid == 0) {
         int fl = (P.n_mapped == 0 && !greedy) ? TLI_ROW_FALLBACK : 0;
-        if (*reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
+        if (!POLL && *reinterpret_cast<volatile unsigned *>(P.error)) fl |= TLI_ROW_TIMEOUT;
         sm_flags = fl;
     }
+    if (POLL) __syncthreads();                       // sm_flags is in place before a wait that expires ORs into it
     // Eight lanes per row, one pass: every lane folds its share of the row's partials into a running
     // pair (changes of reference are exact powers of two), then the eight lanes are folded together.
     // (the loop bound is the same for all lanes of a warp: lanes beyond the last row run along with
@@ -897,7 +922,12 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
         if (greedy) {
             float best = -INFINITY; int idx = INT_MAX;
             for (int i = sub; i < nseg; i += 8) {
-                float2 pr = __ldcg(part + i);
+                float2 pr;
+                if (!POLL) pr = __ldcg(part + i);
+                else if (!load_partial_when_stored(part + i, P.error, pr)) {
+                    atomicOr(&sm_flags, TLI_ROW_TIMEOUT);
+                    pr = make_float2(-INFINITY, __int_as_float(INT_MAX));
+                }
                 int i2 = __float_as_int(pr.y);
                 if (pr.x > best || (pr.x == best && i2 < idx)) { best = pr.x; idx = i2; }
             }
@@ -912,7 +942,12 @@ __device__ __forceinline__ bool decide_sequence(const Params &P, int b, bool wri
             float c = kNegBig;
             double sum = 0.0;
             for (int i = sub; i < nseg; i += 8) {
-                const float2 pr = __ldcg(part + i);
+                float2 pr;
+                if (!POLL) pr = __ldcg(part + i);
+                else if (!load_partial_when_stored(part + i, P.error, pr)) {
+                    atomicOr(&sm_flags, TLI_ROW_TIMEOUT);
+                    pr = make_float2(kNegBig, 0.f);
+                }
                 const float cn = fmaxf(c, pr.x);
                 sum = sum * pow2_neg_d(c - cn) + static_cast<double>(pr.y) * pow2_neg_d(pr.x - cn);
                 c = cn;
@@ -1432,7 +1467,7 @@ __device__ __forceinline__ void st_cluster_f64(uint32_t addr, double v) {
 }
 
 template <int DT>
-__global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params P) {
+__device__ __forceinline__ void finish_sequence(const Params &P) {
     constexpr int EPV = Elt<DT>::kPerVec;
     extern __shared__ __align__(16) unsigned char fin_smem[];
     __shared__ double sm_warp_tot[kFinWarps];
@@ -1452,11 +1487,33 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
         sm_error = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    cluster_barrier();            // every CTA of the cluster is running before anybody stores into a neighbour
-
     RowSel sel;
     int flags;
-    if (!decide_sequence<DT, kFinThreads>(P, b, rank == 0, sel, flags)) return;
+    bool draw;
+    if (P.poll_parts) {
+        // The partials lie in the context's own buffer and are waited for one by one: this grid does not
+        // wait for the statistics grid as a whole (whose end reaches a waiting grid only 2.5 us after its
+        // last CTA has left).  When every CTA of the cluster has read them, the first one puts the
+        // slots back to "empty" for the next call.
+        draw = decide_sequence<DT, kFinThreads, true>(P, b, rank == 0, sel, flags);
+        cluster_barrier();        // ... and every CTA of the cluster is running before anybody stores into a neighbour
+        if (rank == 0) {
+            const float tau = __ldg(P.tau + b);
+            if (tau >= 0.f && !isinf(tau)) {
+                const int Kb = P.draft_len ? min(max(__ldg(P.draft_len + b), 0), P.K) : P.K;
+                const int n_t = (Kb + 1) * P.nst, n_d = (tau == 0.f) ? 0 : Kb * P.nsd;
+                float2 *pt = P.part_t + static_cast<size_t>(b) * (P.K + 1) * P.nst;
+                float2 *pd = P.part_d + static_cast<size_t>(b) * P.K * P.nsd;
+                const float2 empty = make_float2(__uint_as_float(kPartEmpty), __uint_as_float(kPartEmpty));
+                for (int i = tid; i < n_t; i += kFinThreads) __stcg(pt + i, empty);
+                for (int i = tid; i < n_d; i += kFinThreads) __stcg(pd + i, empty);
+            }
+        }
+    } else {
+        cluster_barrier();        // every CTA of the cluster is running before anybody stores into a neighbour
+        draw = decide_sequence<DT, kFinThreads>(P, b, rank == 0, sel, flags);
+    }
+    if (!draw) return;
 
     const RowView<DT> rt(P.zt, static_cast<long long>(b) * P.t_sb + static_cast<long long>(sel.n) * P.t_sk, P.V_t);
     const int nvec = rt.nvec();
@@ -1601,6 +1658,19 @@ __global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params
             P.next_token[b] = token;
         }
         return;
+    }
+}
+
+template <int DT>
+__global__ void __launch_bounds__(kFinThreads, 2) tli_finish_kernel(const Params P) {
+    finish_sequence<DT>(P);
+    if (P.poll_parts) {
+        // This grid did not wait for the statistics grid; it must not be over before that grid is (whose
+        // last CTA puts the segment counter back), or the kernel after this one could overtake it.  By
+        // now the wait returns at once.  A time-out anywhere in that grid marks the row as it always did.
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (threadIdx.x == 0 && cluster_cta_rank() == 0 && P.status && *reinterpret_cast<volatile unsigned *>(P.error))
+            P.status[blockIdx.y] |= TLI_ROW_TIMEOUT;
     }
 }
 
@@ -2903,6 +2973,7 @@ Layout make_layout(int B, int K, int V_t, int V_d, int dtype, int num_sms, int m
 
 }  // namespace
 
+constexpr size_t kCtxPartsBytes = 8u << 20;
 constexpr size_t kCounterWords = 3 * (TLI_MAX_B + 1) + 8;     // per-sequence tickets (two sets, one spare), sticky error, schedulers
 
 struct tli_ctx {
@@ -2914,6 +2985,7 @@ struct tli_ctx {
     int tiled;                  // option: the extra token always by the tile kernels (default 0: by size)
     int max_cluster;            // widest cluster the device takes for the cluster kernel (16 where the driver allows it, else 8)
     int device_max_cluster;     // ... what tli_create() found; max_cluster can be narrowed by tli_set_max_cluster()
+    float2 *d_parts;            // kCtxPartsBytes of partial results for the cluster form: all ones (kPartEmpty) between calls
     unsigned *d_counters;       // [3 * (TLI_MAX_B + 1) + 8], zero between calls: tickets, tickets, sequence states,
                                 // sticky error, schedulers
     int num_sms;
@@ -2975,7 +3047,7 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
     tli_ctx *c = new (std::nothrow) tli_ctx();
     if (!c) { cudaSetDevice(prev); return TLI_ERR_ARG; }
     c->device = device; c->V_t = V_t; c->V_d = V_d; c->n_mapped = n_mapped;
-    c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr;
+    c->d_map = nullptr; c->d_inv = nullptr; c->d_mask = nullptr; c->d_counters = nullptr; c->d_parts = nullptr;
     c->num_sms = 0;
     c->tiled = 0;
     c->max_cluster = 8; c->device_max_cluster = 8;
@@ -3019,13 +3091,15 @@ int tli_create(tli_ctx **out, int device, int32_t V_t, int32_t V_d, const int32_
         if ((e = cudaMalloc(&c->d_inv, sizeof(int32_t) * (static_cast<size_t>(V_t) + 8))) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc inverse map"); break; }
         if ((e = cudaMalloc(&c->d_mask, sizeof(uint32_t) * mask_words)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc mask"); break; }
         if ((e = cudaMalloc(&c->d_counters, sizeof(unsigned) * kCounterWords)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc counters"); break; }
+        if ((e = cudaMalloc(&c->d_parts, kCtxPartsBytes)) != cudaSuccess) { rc = cuda_fail(e, "cudaMalloc partials"); break; }
+        if ((e = cudaMemset(c->d_parts, 0xff, kCtxPartsBytes)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset partials"); break; }
         if ((e = cudaMemcpy(c->d_map, id_map_host, sizeof(int32_t) * V_d, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy map"); break; }
         if ((e = cudaMemcpy(c->d_inv, inv.data(), sizeof(int32_t) * V_t, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy inverse map"); break; }
         if ((e = cudaMemcpy(c->d_mask, mask.data(), sizeof(uint32_t) * mask_words, cudaMemcpyHostToDevice)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemcpy mask"); break; }
         if ((e = cudaMemset(c->d_counters, 0, sizeof(unsigned) * kCounterWords)) != cudaSuccess) { rc = cuda_fail(e, "cudaMemset counters"); break; }
     } while (0);
     if (rc != TLI_OK) {
-        cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters);
+        cudaFree(c->d_map); cudaFree(c->d_inv); cudaFree(c->d_mask); cudaFree(c->d_counters); cudaFree(c->d_parts);
         delete c;
         cudaSetDevice(prev);
         return rc;
@@ -3040,7 +3114,7 @@ int tli_destroy(tli_ctx *ctx) {
     int prev = -1;
     cudaGetDevice(&prev);
     cudaSetDevice(ctx->device);
-    cudaFree(ctx->d_map); cudaFree(ctx->d_inv); cudaFree(ctx->d_mask); cudaFree(ctx->d_counters);
+    cudaFree(ctx->d_map); cudaFree(ctx->d_inv); cudaFree(ctx->d_mask); cudaFree(ctx->d_counters); cudaFree(ctx->d_parts);
     if (prev >= 0) cudaSetDevice(prev);
     delete ctx;
     return TLI_OK;
@@ -3102,6 +3176,16 @@ static int verify_impl(tli_ctx *ctx, const tli_verify_args *a, void *cuda_stream
     P.split_select = (static_cast<long long>(a->B) * L.ntile >= 4096) ? 1 : 0;
     P.ntile = L.ntile;
     P.fin_slice = L.fin_slice; P.fin_dvec = L.fin_dvec;
+    {
+        // cluster form: partials in the context's own buffer, where "not yet stored" can be told from the data
+        const size_t n_t = static_cast<size_t>(a->B) * (a->K + 1) * L.nst, n_d = static_cast<size_t>(a->B) * a->K * L.nsd;
+        if (L.fin_cluster && (n_t + n_d) * sizeof(float2) <= kCtxPartsBytes) {
+            P.part_t = ctx->d_parts;
+            P.part_d = ctx->d_parts + n_t;
+            P.poll_parts = 1;
+            P.early_trigger = L.grid < static_cast<unsigned>(kCtasPerSm * ctx->num_sms) ? 1 : 0;
+        }
+    }
     P.seg_vec = L.seg_vec; P.nst = L.nst; P.nsd = L.nsd;
     P.div_per_b = make_fast_div(static_cast<unsigned>((P.K + 1) * L.nst + P.K * L.nsd));
     P.div_nst = make_fast_div(static_cast<unsigned>(L.nst)); P.div_nsd = make_fast_div(static_cast<unsigned>(L.nsd));
@@ -3483,7 +3567,8 @@ int tli_selftest_bounded_wait(tli_ctx *ctx, void *cuda_stream, unsigned polls, i
 
 int tli_reset(tli_ctx *ctx, void *cuda_stream) {
     if (!ctx) return TLI_ERR_ARG;
-    const cudaError_t e = cudaMemsetAsync(ctx->d_counters, 0, sizeof(unsigned) * kCounterWords, reinterpret_cast<cudaStream_t>(cuda_stream));
+    cudaError_t e = cudaMemsetAsync(ctx->d_counters, 0, sizeof(unsigned) * kCounterWords, reinterpret_cast<cudaStream_t>(cuda_stream));
+    if (e == cudaSuccess) e = cudaMemsetAsync(ctx->d_parts, 0xff, kCtxPartsBytes, reinterpret_cast<cudaStream_t>(cuda_stream));
     return e == cudaSuccess ? TLI_OK : cuda_fail(e, "cudaMemsetAsync counters");
 }
 

@@ -507,6 +507,30 @@ def test_per_sequence_draft_counts(dtype):
         assert (gpu["p_draft"][b, m:] == 0).all() and (gpu["q_draft"][b, m:] == 0).all()
 
 
+def test_one_context_through_changing_shapes():
+    """Calls of different batch sizes, draft counts and temperature mixes on one context, in turn and again:
+    the context's buffer of partial results is back in its empty state after every call, whatever rows the
+    call before used (temperature 0 sequences have no drafter rows, short sequences fewer rows)."""
+    V_t, V_d = 40013, 33001
+    base = wl.tiny_config(B=9, K=5, V_t=V_t, V_d=V_d, dtype=wl.BF16, f_mapped=0.6, sigma_d=0.4,
+                          temperatures=(0.0, 0.7, 1.0), seed=91)
+    first = wl.make_batch(base)
+    v = tli.Verifier(V_t, V_d, first["id_map"])
+    shapes = [dict(B=9, K=5), dict(B=3, K=2), dict(B=14, K=7), dict(B=1, K=1), dict(B=9, K=5)]      # the id map comes from the seed alone
+    for rnd in range(2):
+        for i, sh in enumerate(shapes):
+            cfg = dataclasses.replace(base, **sh)
+            batch = wl.make_batch(cfg)
+            np.testing.assert_array_equal(batch["id_map"], first["id_map"])
+            if i % 2 == 1:
+                batch["draft_lengths"] = (np.arange(cfg.B, dtype=np.int32) * 3) % (cfg.K + 1)
+            rep = check(batch, verifier=v)
+            assert rep.rows == cfg.B, (rnd, sh, rep)
+    plan = tli.tli_verify_plan(v.ctx, 9, 5, tli.TLI_BF16)
+    assert plan["launches"] == 2 and plan["cluster"] >= 1         # the form that uses that buffer
+    v.close()
+
+
 def test_a_wait_that_nothing_completes_gives_up_and_leaves_the_context_usable():
     """The kernels' waits are bounded: run the same wait code on a barrier nobody will complete."""
     cfg = wl.tiny_config(B=3, K=2, V_t=9000, V_d=7000, dtype=wl.F32, f_mapped=0.5, seed=83)
